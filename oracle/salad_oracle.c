@@ -1,0 +1,251 @@
+/*
+ * CPU oracle for the SALAD attention forward pass.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the plain, slow definition of what the GPU library must compute.  It is
+ * called from the tests, from the smoke check and from the CPU-baseline leg of the
+ * benchmark, never from the product path, and it shares no code with the CUDA kernels.
+ *
+ * Everything is evaluated in fp64 on inputs that were already rounded to bf16 and
+ * widened to fp32 by the caller, so the oracle and the GPU see identical operands.
+ * The only "optimisation" is an OpenMP parallel-for over independent outputs; there is
+ * no blocking, no online softmax, no reordering of the sums beyond what the equations
+ * themselves state.
+ *
+ * Layout: Q, K, V are [B, H, N, d] row-major (d fastest).  Tokens of the latent grid
+ * are numbered n = (t*Hs + h)*Ws + w, time slowest (Appendix A.1, token flattening).
+ *
+ * Mask representation: block-granular.  Query block i covers tokens [i*Bq, min(N,(i+1)*Bq)),
+ * key block j covers [j*Bk, min(N,(j+1)*Bk)).  A CSR list per (mask head, query block)
+ * names the kept key blocks; token pair (n, m) is allowed iff block(m) is in the list of
+ * block(n).  This is the matrix M of Eq. 2 with entries 0 on kept blocks, -inf elsewhere.
+ *
+ * Pins (see tests): dense masked softmax written as an N x N matrix (Eq. 2 literally),
+ * the library routine torch SDPA, the un-reordered N x N form of Eq. 3, closed forms
+ * (constant V, zero K, homogeneity in K), hand-counted window masks.
+ *
+ * Parity unpinned: nothing ties these functions to the authors' own implementation (the
+ * paper prints no worked numeric example); the 3-D window reading of the ST-SWA mask and
+ * the per-head scalar reading of the static projection are this build's readings.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_API __attribute__((visibility("default")))
+
+static int iabs(int x) { return x < 0 ? -x : x; }
+
+/* Does any (query token in block i, key token in block j) pair lie inside the 3-D window?
+ * Direct enumeration of all token pairs; the block mask is the "any" over the token mask
+ * (static sliding-window mask of Sec. 3 on the un-permuted t,h,w token order). */
+static int block_pair_kept(int i, int j, int N, int Hs, int Ws, int Bq, int Bk,
+                           int wt, int wh, int ww)
+{
+    int q0 = i * Bq, q1 = q0 + Bq; if (q1 > N) q1 = N;
+    int k0 = j * Bk, k1 = k0 + Bk; if (k1 > N) k1 = N;
+    for (int n = q0; n < q1; ++n) {
+        int tq = n / (Hs * Ws), hq = (n / Ws) % Hs, wq = n % Ws;
+        for (int m = k0; m < k1; ++m) {
+            int tk = m / (Hs * Ws), hk = (m / Ws) % Hs, wk = m % Ws;
+            if (iabs(tq - tk) <= wt && iabs(hq - hk) <= wh && iabs(wq - wk) <= ww) return 1;
+        }
+    }
+    return 0;
+}
+
+/*
+ * oracle_mask_build: CSR lists of kept key blocks for a 3-D sliding-window block mask.
+ *   windows  [Hm][3] = (wt, wh, ww) per mask head.
+ *   row_ptr  [Hm*nQb + 1] out, global offsets; row of (hm, i) is hm*nQb + i.
+ *   col_idx  [capacity] out, ascending key-block ids per row; may be NULL to count only.
+ * Returns nnz (even when capacity is too small; then col_idx holds only the first
+ * `capacity` entries).
+ */
+ORACLE_API int64_t oracle_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm,
+                                     const int32_t* windows, int32_t* row_ptr,
+                                     int32_t* col_idx, int64_t capacity)
+{
+    int N = T * Hs * Ws;
+    int nQb = (N + Bq - 1) / Bq, nKb = (N + Bk - 1) / Bk;
+    int64_t rows = (int64_t)Hm * nQb;
+    unsigned char* keep = (unsigned char*)malloc((size_t)rows * nKb);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < rows; ++r) {
+        int hm = (int)(r / nQb), i = (int)(r % nQb);
+        for (int j = 0; j < nKb; ++j)
+            keep[r * nKb + j] = (unsigned char)block_pair_kept(
+                i, j, N, Hs, Ws, Bq, Bk, windows[3 * hm], windows[3 * hm + 1], windows[3 * hm + 2]);
+    }
+    int64_t nnz = 0;
+    for (int64_t r = 0; r < rows; ++r) {
+        row_ptr[r] = (int32_t)nnz;
+        for (int j = 0; j < nKb; ++j)
+            if (keep[r * nKb + j]) {
+                if (col_idx && nnz < capacity) col_idx[nnz] = j;
+                ++nnz;
+            }
+    }
+    row_ptr[rows] = (int32_t)nnz;
+    free(keep);
+    return nnz;
+}
+
+/* Decode a selected output row.  sel == NULL means "all rows", identity order. */
+static void decode_row(const int64_t* sel, int64_t s, int N, int64_t* bh, int* n)
+{
+    int64_t flat = sel ? sel[s] : s;
+    *bh = flat / N;
+    *n = (int)(flat % N);
+}
+
+/*
+ * oracle_sparse_attn: Eq. 2 with the block-granular mask.
+ * For each selected query row n of head (b,h):
+ *     x_m = scale * <Q_n, K_m>   for every key token m < N in every kept key block
+ *     O_s[n] = sum_m softmax(x)_m V_m ,   lse[n] = log sum_m exp(x_m)
+ * A row whose list is empty gives O_s = 0 and lse = -inf.
+ *   sel   [nsel] flat indices (b*H + h)*N + n, or NULL for all B*H*N rows.
+ *   o     [nsel][d] out (fp64).   lse [nsel] out, may be NULL.
+ */
+ORACLE_API void oracle_sparse_attn(const float* q, const float* k, const float* v,
+                                   int B, int H, int N, int d, int Bq, int Bk,
+                                   const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                   double scale, const int64_t* sel, int64_t nsel,
+                                   double* o, double* lse)
+{
+    int nQb = (N + Bq - 1) / Bq;
+    if (!sel) nsel = (int64_t)B * H * N;
+#pragma omp parallel
+    {
+        double* x = (double*)malloc(sizeof(double) * (size_t)N);
+        int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)N);
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t s = 0; s < nsel; ++s) {
+            int64_t bh; int n;
+            decode_row(sel, s, N, &bh, &n);
+            int h = (int)(bh % H);
+            int hm = (Hm == 1) ? 0 : h;
+            int64_t r = (int64_t)hm * nQb + n / Bq;
+            const float* qn = q + (bh * N + n) * (int64_t)d;
+            const float* kb = k + bh * (int64_t)N * d;
+            const float* vb = v + bh * (int64_t)N * d;
+            /* scores over all kept key tokens */
+            int64_t cnt = 0;
+            double mx = -INFINITY;
+            for (int32_t e = row_ptr[r]; e < row_ptr[r + 1]; ++e) {
+                int j = col_idx[e];
+                int m1 = (j + 1) * Bk; if (m1 > N) m1 = N;
+                for (int m = j * Bk; m < m1; ++m) {
+                    double acc = 0.0;
+                    const float* km = kb + (int64_t)m * d;
+                    for (int c = 0; c < d; ++c) acc += (double)qn[c] * (double)km[c];
+                    acc *= scale;
+                    x[cnt] = acc; idx[cnt] = m; ++cnt;
+                    if (acc > mx) mx = acc;
+                }
+            }
+            double* on = o + s * (int64_t)d;
+            for (int c = 0; c < d; ++c) on[c] = 0.0;
+            if (cnt == 0) { if (lse) lse[s] = -INFINITY; continue; }
+            double l = 0.0;
+            for (int64_t e = 0; e < cnt; ++e) { x[e] = exp(x[e] - mx); l += x[e]; }
+            for (int64_t e = 0; e < cnt; ++e) {
+                double p = x[e] / l;
+                const float* vm = vb + (int64_t)idx[e] * d;
+                for (int c = 0; c < d; ++c) on[c] += p * (double)vm[c];
+            }
+            if (lse) lse[s] = mx + log(l);
+        }
+        free(x); free(idx);
+    }
+}
+
+static double relu(double a) { return a > 0.0 ? a : 0.0; }
+
+/*
+ * oracle_linear_state: the two reductions of Eq. 3,
+ *     KV[b,h] = sum_j ReLU(K_j)^T V_j   (d x d, row = key channel, column = value channel)
+ *     Z[b,h]  = sum_j ReLU(K_j)         (d)
+ */
+ORACLE_API void oracle_linear_state(const float* k, const float* v, int B, int H, int N, int d,
+                                    double* kv, double* z)
+{
+    int64_t BH = (int64_t)B * H;
+#pragma omp parallel for schedule(dynamic, 1) collapse(2)
+    for (int64_t bh = 0; bh < BH; ++bh) {
+        for (int a = 0; a < d; ++a) {
+            const float* kb = k + bh * (int64_t)N * d;
+            const float* vb = v + bh * (int64_t)N * d;
+            double* row = kv + (bh * d + a) * (int64_t)d;
+            for (int c = 0; c < d; ++c) row[c] = 0.0;
+            double zs = 0.0;
+            for (int j = 0; j < N; ++j) {
+                double f = relu((double)kb[(int64_t)j * d + a]);
+                zs += f;
+                const float* vj = vb + (int64_t)j * d;
+                for (int c = 0; c < d; ++c) row[c] += f * (double)vj[c];
+            }
+            z[bh * d + a] = zs;
+        }
+    }
+}
+
+/*
+ * oracle_linear_attn: Eq. 3 for selected rows, from the state,
+ *     O_l[n] = ReLU(Q_n) KV / (ReLU(Q_n) . Z + eps).
+ * The paper's denominator has no eps; eps > 0 only defines the 0/0 case (all ReLU(Q_n)
+ * zero gives O_l = 0).
+ */
+ORACLE_API void oracle_linear_attn(const float* q, const double* kv, const double* z,
+                                   int B, int H, int N, int d, double eps,
+                                   const int64_t* sel, int64_t nsel, double* o_l)
+{
+    if (!sel) nsel = (int64_t)B * H * N;
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        int64_t bh; int n;
+        decode_row(sel, s, N, &bh, &n);
+        const float* qn = q + (bh * N + n) * (int64_t)d;
+        const double* kvb = kv + bh * (int64_t)d * d;
+        const double* zb = z + bh * (int64_t)d;
+        double den = 0.0;
+        for (int a = 0; a < d; ++a) den += relu((double)qn[a]) * zb[a];
+        double* on = o_l + s * (int64_t)d;
+        for (int c = 0; c < d; ++c) {
+            double num = 0.0;
+            for (int a = 0; a < d; ++a) num += relu((double)qn[a]) * kvb[(int64_t)a * d + c];
+            on[c] = num / (den + eps);
+        }
+    }
+}
+
+/*
+ * oracle_salad_fused: Algorithm 1, residual integration, with the static projection read
+ * as one scalar per head (lambda of Eq. 5 folded in) and the dynamic scale s one scalar
+ * per batch item:
+ *     O[b,h,n] = O_s[b,h,n] + s[b] * lambda[h] * O_l[b,h,n].
+ */
+ORACLE_API void oracle_salad_fused(const float* q, const float* k, const float* v,
+                                   int B, int H, int N, int d, int Bq, int Bk,
+                                   const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                   const double* lambda_h, const double* s_b,
+                                   double scale, double eps,
+                                   const int64_t* sel, int64_t nsel, double* o)
+{
+    if (!sel) nsel = (int64_t)B * H * N;
+    int64_t BH = (int64_t)B * H;
+    double* kv = (double*)malloc(sizeof(double) * (size_t)(BH * d * d));
+    double* z = (double*)malloc(sizeof(double) * (size_t)(BH * d));
+    double* ol = (double*)malloc(sizeof(double) * (size_t)(nsel * d));
+    oracle_sparse_attn(q, k, v, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, scale, sel, nsel, o, NULL);
+    oracle_linear_state(k, v, B, H, N, d, kv, z);
+    oracle_linear_attn(q, kv, z, B, H, N, d, eps, sel, nsel, ol);
+    for (int64_t s = 0; s < nsel; ++s) {
+        int64_t bh; int n;
+        decode_row(sel, s, N, &bh, &n);
+        double c = s_b[bh / H] * lambda_h[bh % H];
+        for (int a = 0; a < d; ++a) o[s * d + a] += c * ol[s * d + a];
+    }
+    free(kv); free(z); free(ol);
+}

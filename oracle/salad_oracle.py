@@ -1,0 +1,156 @@
+"""ctypes front end of the CPU oracle (``salad_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the CPU-baseline leg of the benchmark may import this
+module.  It never touches the GPU library and the GPU library never touches it.
+
+All array arguments are numpy arrays; Q, K, V are float32 arrays holding bf16-representable
+values, shape [B, H, N, d].  Outputs are float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "salad_oracle.c")
+_LIB = os.path.join(_HERE, "libsalad_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP only parallelises independent output rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-fvisibility=hidden",
+             "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i32, i64, f64 = ctypes.c_int32, ctypes.c_int64, ctypes.c_double
+        p = ctypes.c_void_p
+        lib.oracle_mask_build.restype = i64
+        lib.oracle_mask_build.argtypes = [i32] * 6 + [p, p, p, i64]
+        lib.oracle_sparse_attn.restype = None
+        lib.oracle_sparse_attn.argtypes = [p, p, p] + [i32] * 6 + [p, p, i32, f64, p, i64, p, p]
+        lib.oracle_linear_state.restype = None
+        lib.oracle_linear_state.argtypes = [p, p] + [i32] * 4 + [p, p]
+        lib.oracle_linear_attn.restype = None
+        lib.oracle_linear_attn.argtypes = [p, p, p] + [i32] * 4 + [f64, p, i64, p]
+        lib.oracle_salad_fused.restype = None
+        lib.oracle_salad_fused.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64,
+                                                                    p, i64, p])
+        _lib = lib
+    return _lib
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data
+
+
+def _i32(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data
+
+
+def _sel(sel):
+    if sel is None:
+        return None, None, 0
+    s = np.ascontiguousarray(sel, dtype=np.int64)
+    return s, s.ctypes.data, int(s.size)
+
+
+def num_threads() -> int:
+    """Threads the OpenMP runtime will use (OMP_NUM_THREADS or all visible cores)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env.split(",")[0])
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def mask_build(T, Hs, Ws, Bq, Bk, windows):
+    """3-D sliding-window block mask -> (row_ptr[Hm*nQb+1], col_idx[nnz]) int32."""
+    lib = _load()
+    w, wp = _i32(np.asarray(windows).reshape(-1, 3))
+    Hm = w.shape[0]
+    N = T * Hs * Ws
+    nQb = -(-N // Bq)
+    row_ptr = np.zeros(Hm * nQb + 1, dtype=np.int32)
+    nnz = lib.oracle_mask_build(T, Hs, Ws, Bq, Bk, Hm, wp, row_ptr.ctypes.data, None, 0)
+    col_idx = np.zeros(max(nnz, 1), dtype=np.int32)
+    lib.oracle_mask_build(T, Hs, Ws, Bq, Bk, Hm, wp, row_ptr.ctypes.data, col_idx.ctypes.data, nnz)
+    return row_ptr, col_idx[:nnz]
+
+
+def sparse_attn(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, scale=None, sel=None):
+    """Eq. 2 on the block mask.  Returns (O_s [rows, d] float64, lse [rows] float64)."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = q.shape
+    rp, rpp = _i32(row_ptr); ci, cip = _i32(col_idx if len(col_idx) else np.zeros(1, np.int32))
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    lse = np.empty(rows, dtype=np.float64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    lib.oracle_sparse_attn(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, float(scale),
+                           sp, nsel, o.ctypes.data, lse.ctypes.data)
+    return o, lse
+
+
+def linear_state(k, v):
+    """Returns (KV [B,H,d,d], Z [B,H,d]) float64."""
+    lib = _load()
+    k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = k.shape
+    kv = np.empty((B, H, d, d), dtype=np.float64)
+    z = np.empty((B, H, d), dtype=np.float64)
+    lib.oracle_linear_state(kp, vp, B, H, N, d, kv.ctypes.data, z.ctypes.data)
+    return kv, z
+
+
+def linear_attn(q, k, v, eps=1e-6, sel=None, state=None):
+    """Eq. 3.  Returns O_l [rows, d] float64."""
+    lib = _load()
+    q, qp = _f32(q)
+    B, H, N, d = q.shape
+    kv, z = state if state is not None else linear_state(k, v)
+    kv = np.ascontiguousarray(kv, dtype=np.float64); z = np.ascontiguousarray(z, dtype=np.float64)
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    lib.oracle_linear_attn(qp, kv.ctypes.data, z.ctypes.data, B, H, N, d, float(eps),
+                           sp, nsel, o.ctypes.data)
+    return o
+
+
+def salad_fused(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, scale=None, eps=1e-6,
+                sel=None):
+    """Algorithm 1 residual integration: O_s + s_b * lambda_h * O_l.  [rows, d] float64."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = q.shape
+    rp, rpp = _i32(row_ptr); ci, cip = _i32(col_idx if len(col_idx) else np.zeros(1, np.int32))
+    lam = np.ascontiguousarray(lambda_h, dtype=np.float64); sb = np.ascontiguousarray(s_b, dtype=np.float64)
+    assert lam.size == H and sb.size == B
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    lib.oracle_salad_fused(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
+                           sb.ctypes.data, float(scale), float(eps), sp, nsel, o.ctypes.data)
+    return o

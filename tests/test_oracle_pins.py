@@ -1,0 +1,306 @@
+"""Pins of the CPU oracle against things other than itself: the equations written out as
+dense N x N matrices in numpy, torch's SDPA routine, closed forms and hand-counted masks.
+CPU only."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import salad_oracle as orc
+from paper_2601_16515_b200 import workloads as wlmod
+
+
+def bf16_round(a):
+    return torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).float().numpy()
+
+
+def rand_qkv(B, H, N, d, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return tuple(bf16_round(rng.standard_normal((B, H, N, d)) * scale) for _ in range(3))
+
+
+def token_mask_from_csr(N, Bq, Bk, row_ptr, col_idx, hm, nQb):
+    """Matrix M of Eq. 2 as a boolean 'allowed' matrix [N, N]."""
+    allowed = np.zeros((N, N), dtype=bool)
+    for i in range(nQb):
+        r = hm * nQb + i
+        for j in col_idx[row_ptr[r]:row_ptr[r + 1]]:
+            allowed[i * Bq:min(N, (i + 1) * Bq), j * Bk:min(N, (j + 1) * Bk)] = True
+    return allowed
+
+
+def dense_masked_softmax(q, k, v, allowed):
+    """Eq. 2 literally: softmax((Q K^T + M)/sqrt(d)) V with M in {-inf, 0}."""
+    d = q.shape[-1]
+    M = np.where(allowed, 0.0, -np.inf)
+    s = (q.astype(np.float64) @ k.astype(np.float64).T + M) / np.sqrt(d)
+    s = s - s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    p /= p.sum(axis=1, keepdims=True)
+    return p @ v.astype(np.float64)
+
+
+# ----------------------------------------------------------------------------- mask
+
+def window_mask_vectorised(T, Hs, Ws, Bq, Bk, win):
+    """Token-level window mask by broadcasting, then 'any' over blocks."""
+    N = T * Hs * Ws
+    n = np.arange(N)
+    t, h, w = n // (Hs * Ws), (n // Ws) % Hs, n % Ws
+    tok = ((np.abs(t[:, None] - t[None, :]) <= win[0]) &
+           (np.abs(h[:, None] - h[None, :]) <= win[1]) &
+           (np.abs(w[:, None] - w[None, :]) <= win[2]))
+    nQb, nKb = -(-N // Bq), -(-N // Bk)
+    blk = np.zeros((nQb, nKb), dtype=bool)
+    for i in range(nQb):
+        for j in range(nKb):
+            blk[i, j] = tok[i * Bq:(i + 1) * Bq, j * Bk:(j + 1) * Bk].any()
+    return blk
+
+
+def csr_to_dense(row_ptr, col_idx, rows, nKb):
+    out = np.zeros((rows, nKb), dtype=bool)
+    for r in range(rows):
+        out[r, col_idx[row_ptr[r]:row_ptr[r + 1]]] = True
+    return out
+
+
+def test_mask_hand_counted():
+    # Grid 2 x 2 x 4, blocks of 4 tokens = one (t,h) row each; block id = 2 t + h.
+    rp, ci = orc.mask_build(2, 2, 4, 4, 4, [(0, 0, 1)])      # same row only
+    assert rp.tolist() == [0, 1, 2, 3, 4] and ci.tolist() == [0, 1, 2, 3]
+    rp, ci = orc.mask_build(2, 2, 4, 4, 4, [(0, 1, 0)])      # both rows of the own frame
+    assert rp.tolist() == [0, 2, 4, 6, 8] and ci.tolist() == [0, 1, 0, 1, 2, 3, 2, 3]
+    rp, ci = orc.mask_build(2, 2, 4, 4, 4, [(1, 0, 0)])      # same row in both frames
+    assert ci.tolist() == [0, 2, 1, 3, 0, 2, 1, 3]
+    # Bq = 8 (one frame per query block), Bk = 4, two mask heads
+    rp, ci = orc.mask_build(2, 2, 4, 8, 4, [(0, 0, 0), (1, 0, 0)])
+    assert rp.tolist() == [0, 2, 4, 8, 12]
+    assert ci.tolist() == [0, 1, 2, 3, 0, 1, 2, 3, 0, 1, 2, 3]
+
+
+@pytest.mark.parametrize("grid,Bq,Bk,win", [
+    ((3, 5, 7), 16, 8, (1, 1, 2)),     # ragged: N = 105
+    ((4, 6, 6), 32, 16, (0, 2, 2)),
+    ((4, 6, 6), 16, 16, (2, 0, 0)),
+    ((2, 9, 11), 64, 32, (1, 3, 4)),   # N = 198
+])
+def test_mask_vs_vectorised_token_mask(grid, Bq, Bk, win):
+    T, Hs, Ws = grid
+    rp, ci = orc.mask_build(T, Hs, Ws, Bq, Bk, [win])
+    ref = window_mask_vectorised(T, Hs, Ws, Bq, Bk, win)
+    got = csr_to_dense(rp, ci, ref.shape[0], ref.shape[1])
+    assert (got == ref).all()
+    for r in range(ref.shape[0]):                             # ascending, unique
+        row = ci[rp[r]:rp[r + 1]]
+        assert (np.diff(row) > 0).all()
+
+
+def test_mask_invariants_tiny_config():
+    wl = wlmod.C1
+    T, Hs, Ws = wl.grid
+    rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    nQb, nKb = wl.nQb, wl.nKb
+    dense = csr_to_dense(rp, ci, 2 * nQb, nKb)
+    assert dense.sum() == 2 * nQb * 4                         # exactly 25 % kept per row
+    for i in range(nQb):
+        frame = i // 4
+        assert dense[i].nonzero()[0].tolist() == [4 * frame + c for c in range(4)]
+        assert dense[nQb + i].nonzero()[0].tolist() == [4 * f + i % 4 for f in range(4)]
+    # window >= grid keeps everything; window 0 keeps exactly the overlapping key blocks
+    rp, ci = orc.mask_build(T, Hs, Ws, 128, 64, [(T, Hs, Ws)])
+    assert len(ci) == (wl.N // 128) * (wl.N // 64)
+    rp, ci = orc.mask_build(T, Hs, Ws, 128, 64, [(0, 0, 0)])
+    assert ci.tolist() == list(range(wl.N // 64))
+
+
+def test_mask_block_counts_wan_shape():
+    # Block counts for the 21 x 30 x 52 grid with 128 x 64 blocks; sparsity targets of the
+    # workload list: ~80 %, ~90 %, ~95 %.
+    total = 256 * 512
+    for win, lo, hi in [((5, 5, 24), 0.79, 0.81), ((2, 5, 24), 0.895, 0.905), ((1, 4, 24), 0.94, 0.955)]:
+        rp, ci = orc.mask_build(21, 30, 52, 128, 64, [win])
+        sp = 1.0 - len(ci) / total
+        assert lo <= sp <= hi, (win, sp)
+        # own blocks always kept
+        for i in (0, 100, 255):
+            row = ci[rp[i]:rp[i + 1]]
+            assert 2 * i in row and min(2 * i + 1, 511) in row
+
+
+# ----------------------------------------------------------------------------- sparse branch
+
+@pytest.mark.parametrize("N,Bq,Bk,d", [(256, 64, 64, 64), (200, 64, 32, 32), (300, 128, 64, 128)])
+def test_sparse_vs_dense_masked_softmax(N, Bq, Bk, d):
+    B, H = 1, 2
+    q, k, v = rand_qkv(B, H, N, d, 11)
+    nQb, nKb = -(-N // Bq), -(-N // Bk)
+    rng = np.random.default_rng(5)
+    rp, cols = [0], []
+    for r in range(H * nQb):
+        row = np.sort(rng.choice(nKb, size=rng.integers(1, nKb + 1), replace=False))
+        cols.append(row); rp.append(rp[-1] + len(row))
+    rp = np.asarray(rp, np.int32); ci = np.concatenate(cols).astype(np.int32)
+    o, lse = orc.sparse_attn(q, k, v, Bq, Bk, rp, ci, H)
+    o = o.reshape(B, H, N, d)
+    for h in range(H):
+        allowed = token_mask_from_csr(N, Bq, Bk, rp, ci, h, nQb)
+        ref = dense_masked_softmax(q[0, h], k[0, h], v[0, h], allowed)
+        np.testing.assert_allclose(o[0, h], ref, rtol=1e-10, atol=1e-12)
+        # library routine as a second witness
+        sd = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q[0, h]).double()[None], torch.from_numpy(k[0, h]).double()[None],
+            torch.from_numpy(v[0, h]).double()[None], attn_mask=torch.from_numpy(allowed)[None])
+        np.testing.assert_allclose(o[0, h], sd[0].numpy(), rtol=1e-9, atol=1e-11)
+        # lse: log of the masked row sums of exp(scores)
+        s = (q[0, h].astype(np.float64) @ k[0, h].astype(np.float64).T) / np.sqrt(d)
+        ref_lse = np.log(np.where(allowed, np.exp(s), 0.0).sum(axis=1))
+        np.testing.assert_allclose(lse.reshape(B, H, N)[0, h], ref_lse, rtol=1e-10)
+
+
+def test_sparse_all_kept_is_full_attention():
+    B, H, N, d = 2, 2, 192, 64
+    q, k, v = rand_qkv(B, H, N, d, 3)
+    rp, ci = wlmod.dense_csr(-(-N // 64), -(-N // 64), 1)
+    o, _ = orc.sparse_attn(q, k, v, 64, 64, rp, ci, 1)
+    o = o.reshape(B, H, N, d)
+    s = np.einsum("bhnd,bhmd->bhnm", q.astype(np.float64), k.astype(np.float64)) / np.sqrt(d)
+    p = np.exp(s - s.max(-1, keepdims=True)); p /= p.sum(-1, keepdims=True)
+    ref = np.einsum("bhnm,bhmd->bhnd", p, v.astype(np.float64))            # Eq. 1
+    np.testing.assert_allclose(o, ref, rtol=1e-10, atol=1e-12)
+
+
+def test_sparse_closed_forms():
+    B, H, N, d, Bq, Bk = 1, 1, 200, 32, 64, 32
+    q, k, v = rand_qkv(B, H, N, d, 9)
+    T = 1
+    rp, ci = orc.mask_build(1, 1, N, Bq, Bk, [(0, 0, 40)])
+    nQb = -(-N // Bq)
+    # K = 0: uniform weights -> O_s is the mean of V over the kept tokens, lse = log(count)
+    o, lse = orc.sparse_attn(q, np.zeros_like(k), v, Bq, Bk, rp, ci, 1)
+    allowed = token_mask_from_csr(N, Bq, Bk, rp, ci, 0, nQb)
+    cnt = allowed.sum(1)
+    ref = (allowed[:, :, None] * v[0, 0][None].astype(np.float64)).sum(1) / cnt[:, None]
+    np.testing.assert_allclose(o, ref, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(lse, np.log(cnt), rtol=1e-12)
+    # V = const: the output is that constant whatever the weights are
+    vc = np.broadcast_to(bf16_round(np.linspace(-1, 1, d)), v.shape).copy()
+    o, _ = orc.sparse_attn(q, k, vc, Bq, Bk, rp, ci, 1)
+    np.testing.assert_allclose(o, np.broadcast_to(vc[0, 0, 0], o.shape), rtol=1e-12, atol=1e-13)
+    # one key with a dominant score: O_s of every row that sees it -> that key's V row
+    kd = k.copy(); qd = np.abs(q)
+    kd[0, 0, 70] = 64.0
+    o, _ = orc.sparse_attn(qd, kd, v, Bq, Bk, rp, ci, 1)
+    sees = allowed[:, 70]
+    np.testing.assert_allclose(o[sees], np.broadcast_to(v[0, 0, 70], o[sees].shape), atol=1e-6)
+    # empty rows: zero output, lse = -inf
+    rp0 = np.zeros(nQb + 1, np.int32)
+    o, lse = orc.sparse_attn(q, k, v, Bq, Bk, rp0, np.zeros(0, np.int32), 1)
+    assert (o == 0).all() and np.isneginf(lse).all()
+
+
+def test_sparse_row_selection_matches_full():
+    B, H, N, d = 2, 3, 130, 32
+    q, k, v = rand_qkv(B, H, N, d, 4)
+    rp, ci = orc.mask_build(1, 10, 13, 32, 16, [(0, 2, 3)] * H)
+    full, lse_full = orc.sparse_attn(q, k, v, 32, 16, rp, ci, H)
+    sel = np.array([0, 5, 129, 130, 777, B * H * N - 1], dtype=np.int64)
+    part, lse = orc.sparse_attn(q, k, v, 32, 16, rp, ci, H, sel=sel)
+    np.testing.assert_array_equal(part, full[sel])
+    np.testing.assert_array_equal(lse, lse_full[sel])
+
+
+# ----------------------------------------------------------------------------- linear branch
+
+def test_linear_vs_explicit_quadratic_form():
+    B, H, N, d = 2, 2, 150, 32
+    q, k, v = rand_qkv(B, H, N, d, 21)
+    o = orc.linear_attn(q, k, v, eps=0.0).reshape(B, H, N, d)
+    fq, fk = np.maximum(q, 0).astype(np.float64), np.maximum(k, 0).astype(np.float64)
+    W = np.einsum("bhnd,bhmd->bhnm", fq, fk)                    # phi(Q) phi(K)^T, N x N
+    ref = (W @ v.astype(np.float64)) / W.sum(-1, keepdims=True)
+    np.testing.assert_allclose(o, ref, rtol=1e-10, atol=1e-12)
+    kv, z = orc.linear_state(k, v)
+    np.testing.assert_allclose(kv, np.einsum("bhna,bhnc->bhac", fk, v.astype(np.float64)), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(z, fk.sum(2), rtol=1e-12)
+    # KV is not symmetric in (key channel, value channel): guard against a transposed state
+    assert not np.allclose(kv, np.swapaxes(kv, -1, -2))
+
+
+def test_linear_closed_forms():
+    B, H, N, d = 1, 2, 97, 16
+    q, k, v = rand_qkv(B, H, N, d, 22)
+    # V = const c -> O_l = c wherever the denominator is positive
+    vc = np.broadcast_to(bf16_round(np.linspace(-2, 2, d)), v.shape).copy()
+    o = orc.linear_attn(q, k, vc, eps=0.0)
+    np.testing.assert_allclose(o, np.broadcast_to(vc[0, 0, 0], o.shape), rtol=1e-12, atol=1e-13)
+    # K = const >= 0 -> uniform weights -> O_l = mean of V
+    kc = np.full_like(k, 0.5)
+    o = orc.linear_attn(q, kc, v, eps=0.0).reshape(B, H, N, d)
+    ref = np.broadcast_to(v.astype(np.float64).mean(2, keepdims=True), o.shape)
+    np.testing.assert_allclose(o, ref, rtol=1e-11, atol=1e-13)
+    # Q <= 0 everywhere -> numerator and denominator vanish -> 0 (eps defines 0/0)
+    o = orc.linear_attn(-np.abs(q), k, v, eps=1e-6)
+    assert (o == 0).all()
+    # homogeneity: phi(a K) = a phi(K) for a > 0 cancels between numerator and denominator
+    o1 = orc.linear_attn(q, k, v, eps=0.0)
+    o2 = orc.linear_attn(q, 4.0 * k, v, eps=0.0)
+    np.testing.assert_allclose(o1, o2, rtol=1e-12, atol=1e-13)
+    # eps enters only the denominator
+    kv, z = orc.linear_state(k, v)
+    fq = np.maximum(q, 0).astype(np.float64)
+    num = np.einsum("bhna,bhac->bhnc", fq, kv); den = np.einsum("bhna,bha->bhn", fq, z)
+    o3 = orc.linear_attn(q, k, v, eps=0.25).reshape(B, H, N, d)
+    np.testing.assert_allclose(o3, num / (den[..., None] + 0.25), rtol=1e-12, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- combination
+
+def test_fused_is_sparse_plus_scaled_linear():
+    wl = wlmod.C1
+    q, k, v = (t.float().numpy() for t in wlmod.make_qkv(wl))
+    T, Hs, Ws = wl.grid
+    rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    lam, s = wlmod.make_scales(wl)
+    o_s, _ = orc.sparse_attn(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm)
+    o_l = orc.linear_attn(q, k, v)
+    fused = orc.salad_fused(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s)
+    c = np.repeat((s.astype(np.float64)[:, None] * lam.astype(np.float64)[None, :]).reshape(-1), wl.N)[:, None]
+    np.testing.assert_allclose(fused, o_s + c * o_l, rtol=1e-13, atol=1e-14)
+    # zero scale (zero-initialised projection / dropped branch) -> exactly the sparse branch
+    z = orc.salad_fused(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, np.zeros_like(lam), s)
+    np.testing.assert_array_equal(z, o_s)
+    # lambda = s = 1 -> plain sum; and the result is linear in the scale
+    one = orc.salad_fused(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, np.ones_like(lam), np.ones_like(s))
+    np.testing.assert_allclose(one, o_s + o_l, rtol=1e-13, atol=1e-14)
+    half = orc.salad_fused(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, 0.5 * np.ones_like(lam), np.ones_like(s))
+    np.testing.assert_allclose(half - o_s, 0.5 * (one - o_s), rtol=1e-9, atol=1e-12)
+    # per-head / per-batch indexing of the scales (B = 2, distinct values)
+    B, H, N, d = 2, 3, 64, 16
+    q2, k2, v2 = rand_qkv(B, H, N, d, 8)
+    rp2, ci2 = wlmod.dense_csr(1, 1, 1)
+    lam2 = np.array([0.1, 0.5, 0.9]); s2 = np.array([0.25, 0.75])
+    f2 = orc.salad_fused(q2, k2, v2, 64, 64, rp2, ci2, 1, lam2, s2).reshape(B, H, N, d)
+    os2 = orc.sparse_attn(q2, k2, v2, 64, 64, rp2, ci2, 1)[0].reshape(B, H, N, d)
+    ol2 = orc.linear_attn(q2, k2, v2).reshape(B, H, N, d)
+    for b in range(B):
+        for h in range(H):
+            np.testing.assert_allclose(f2[b, h], os2[b, h] + s2[b] * lam2[h] * ol2[b, h], rtol=1e-13, atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- input generators
+
+def test_workloads_are_seeded_and_sliceable():
+    wl = wlmod.C1
+    a = wlmod.make_qkv(wl); b = wlmod.make_qkv(wl)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    sub = wlmod.make_qkv(wl, heads=[1])
+    assert torch.equal(sub[0][:, 0], a[0][:, 1])
+    small = wlmod.Workload("s", 1, 2, 32, (3, 10, 12), 128, 64, (), 7, irregular=True)
+    rp, ci = wlmod.irregular_csr(small, 0.3, 0.6)
+    assert rp[-1] == len(ci) and len(rp) == small.H * small.nQb + 1
+    for r in range(len(rp) - 1):
+        row = ci[rp[r]:rp[r + 1]]
+        assert (np.diff(row) > 0).all() and row.min() >= 0 and row.max() < small.nKb
+        i = r % small.nQb
+        assert 2 * i in row
