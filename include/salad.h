@@ -1,0 +1,128 @@
+/*
+ * libsalad -- SALAD sparse-linear attention forward for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the attention core of Algorithm 1 ("SALAD Attention with
+ * Multi-level Scaling"):
+ *
+ *     O_s = SparseAttn(Q, K, V)                 Eq. 2, block-granular mask
+ *     O_l = LinearAttn(Q, K, V)                 Eq. 3, ReLU feature map
+ *     O   = O_s + s_b * lambda_h * O_l          Alg. 1 residual integration, Eq. 5
+ *
+ * Conventions shared by every entry point
+ *   - Q, K, V, O are bf16 tensors [B, H, N, d], contiguous, d fastest, base address 16-byte
+ *     aligned.  Tokens are the row-major flattening of a T x Hs x Ws latent grid, time
+ *     slowest (Appendix A.1).  N need not be a multiple of the block sizes: the last blocks
+ *     are short, keys >= N take no part, queries >= N are never written.
+ *   - The sparsity mask is block granular: query block i covers tokens [i*Bq, (i+1)*Bq),
+ *     key block j covers [j*Bk, (j+1)*Bk).  It is passed as CSR lists: row r = hm*nQb + i
+ *     (nQb = ceil(N/Bq)) owns col_idx[row_ptr[r] .. row_ptr[r+1]), the kept key blocks,
+ *     ascending and unique, each in [0, ceil(N/Bk)).  Hm is 1 (one mask for all heads) or H.
+ *     The mask is shared by all batch items.  An empty row is legal: its O_s is zero.
+ *   - Every pointer is DEVICE memory owned by the caller unless its name starts with h_
+ *     (host).  Nothing is allocated or freed by the library; scratch comes from a caller
+ *     workspace of at least salad_workspace_bytes() bytes, 256-byte aligned, which must
+ *     not be shared by calls that may overlap on the GPU.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is enqueued
+ *     asynchronously on it; only salad_mask_build synchronises (to return nnz).
+ *   - Return value: SALAD_OK or a negative code.  Argument errors are detected on the host
+ *     before anything is launched.  There is no CPU fallback: without a usable CUDA device
+ *     the compute entry points return SALAD_ERR_CUDA.
+ *   - d_status (optional, device int32): set to 0 by a successful launch and to a non-zero
+ *     code by a kernel whose bounded internal wait expired (the kernel then returns early
+ *     instead of hanging; outputs are undefined).  Read it after synchronising the stream.
+ *   - Supported shapes: d in {64, 128}; Bq in {64, 128}; Bk = 64; softmax_scale > 0.
+ */
+#ifndef SALAD_H_
+#define SALAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SALAD_OK 0
+#define SALAD_ERR_INVALID_ARG (-1) /* null pointer, non-positive size, bad Hm, misalignment  */
+#define SALAD_ERR_UNSUPPORTED (-2) /* d, Bq or Bk outside the supported set                  */
+#define SALAD_ERR_WORKSPACE (-3)   /* workspace missing, misaligned or too small             */
+#define SALAD_ERR_CAPACITY (-4)    /* col_idx capacity smaller than nnz (nnz still returned) */
+#define SALAD_ERR_CUDA (-5)        /* a CUDA runtime/driver call or a launch failed          */
+#define SALAD_ERR_TIMEOUT (-6)     /* value written to d_status by a kernel that gave up     */
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* salad_status_string(int status);
+
+/* Bytes of workspace the *_fwd calls need for this problem size (0 if the shape is
+ * unsupported).  Depends only on the arguments, never on the device. */
+size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk);
+
+/*
+ * salad_mask_build -- static spatio-temporal sliding-window block mask (Sec. 3 "static
+ * sparse attention", Appendix A.1), 3-D window form on the un-permuted t,h,w token order.
+ * Key block j is kept for query block i of mask head hm iff some query token (t,h,w) of
+ * block i and some key token (t',h',w') of block j satisfy |t-t'| <= wt, |h-h'| <= wh,
+ * |w-w'| <= ww with (wt,wh,ww) = h_windows[hm].
+ *   T, Hs, Ws      latent grid; N = T*Hs*Ws.
+ *   Bq, Bk         block sizes (any positive values).
+ *   Hm             number of mask heads; h_windows is a HOST array [Hm][3].
+ *   d_row_ptr      device int32 [Hm*nQb + 1], written.
+ *   d_col_idx      device int32 [col_capacity], written ascending per row; may be NULL with
+ *                  col_capacity 0 to obtain only row_ptr and nnz.
+ *   h_nnz          HOST int64, written with the total number of kept blocks (optional).
+ * Synchronises `stream`.  Returns SALAD_ERR_CAPACITY (row_ptr and *h_nnz valid, col_idx
+ * untouched) if col_capacity < nnz and d_col_idx != NULL.
+ */
+int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm, const int32_t* h_windows,
+                     int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
+                     int64_t* h_nnz, void* stream);
+
+/*
+ * salad_sparse_attn_fwd -- block-sparse softmax attention, Eq. 2:
+ *     O_s[n] = sum_m softmax_m(softmax_scale * <Q_n, K_m>) V_m   over keys m of kept blocks.
+ *   o              bf16 [B,H,N,d], written.
+ *   lse            optional fp32 [B,H,N]: log-sum-exp (natural log) of the scaled scores of
+ *                  each row; -inf for rows with an empty list.
+ *   softmax_scale  0 selects 1/sqrt(d).
+ */
+int salad_sparse_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                          int B, int H, int N, int d, int Bq, int Bk,
+                          const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                          float softmax_scale, void* workspace, size_t workspace_bytes,
+                          int32_t* d_status, void* stream);
+
+/*
+ * salad_linear_attn_fwd -- ReLU linear attention, Eq. 3:
+ *     KV = sum_j ReLU(K_j)^T V_j  (d x d),   Z = sum_j ReLU(K_j)  (d),
+ *     O_l[n] = ReLU(Q_n) KV / (ReLU(Q_n) . Z + eps).
+ *   o_l            bf16 [B,H,N,d], written.
+ *   kv_out         optional fp32 [B,H,d,d] (row = key channel, column = value channel).
+ *   z_out          optional fp32 [B,H,d].
+ *   eps            >= 0; only defines the 0/0 case (a row with ReLU(Q_n) = 0 gives 0).
+ */
+int salad_linear_attn_fwd(const void* q, const void* k, const void* v, void* o_l,
+                          float* kv_out, float* z_out, int B, int H, int N, int d, float eps,
+                          void* workspace, size_t workspace_bytes, int32_t* d_status,
+                          void* stream);
+
+/*
+ * salad_fused_fwd -- both branches and the scaled residual sum of Algorithm 1 with a single
+ * bf16 write of O:
+ *     O[b,h,n] = O_s[b,h,n] + d_dyn_scale[b] * d_static_scale[h] * O_l[b,h,n].
+ *   d_static_scale fp32 [H]: the layer-wise static scaling read as one scalar per head
+ *                  (block-diagonal projection; lambda of Eq. 5 multiplied in by the caller).
+ *   d_dyn_scale    fp32 [B]: the input- and timestep-aware factor s of Alg. 1, produced
+ *                  upstream on the device; any finite value is accepted.
+ * A zero product of the scales reproduces salad_sparse_attn_fwd bit for bit.
+ */
+int salad_fused_fwd(const void* q, const void* k, const void* v, void* o,
+                    int B, int H, int N, int d, int Bq, int Bk,
+                    const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                    const float* d_static_scale, const float* d_dyn_scale,
+                    float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                    int32_t* d_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SALAD_H_ */

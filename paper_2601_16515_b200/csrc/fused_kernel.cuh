@@ -1,0 +1,480 @@
+// Block-sparse softmax attention (Eq. 2) fused with the apply step of ReLU linear attention
+// (Eq. 3) and the scaled residual sum of Algorithm 1, for sm_100a.
+//
+// One CTA owns two consecutive query blocks of one (batch, head): two 128-row MMA tiles.
+//   warp 0        TMA producer: Q tiles, linear-state tile, K/V tiles of the kept key blocks
+//   warp 1        tcgen05 MMA issuer (one thread); owns the TMEM allocation
+//   warps 4-7     softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
+//   warps 8-11    the same for tile 1
+// The kept lists of the two query blocks are walked as one sorted merge, so a key block that
+// both keep is fetched once and multiplied against both tiles.  Masked blocks are never
+// loaded.  S = Q K^T lands in TMEM (two 64-column buffers per tile, so the next block's
+// scores are computed while the current block's softmax runs); the softmax warpgroup reads
+// its row, keeps a running max in the log2 domain (rescaling the O accumulator only when the
+// max grows by more than 2^8), writes P = exp2(.) as bf16 over the S columns, and the MMA
+// warp accumulates O += P V with P read from TMEM.  After the last block the warpgroup applies
+// ReLU to its Q rows in shared memory, computes the linear denominator with plain FMAs, the
+// MMA warp multiplies ReLU(Q) with the bf16 linear state, and the epilogue writes
+//     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
+// once, as bf16, through a TMA store.
+//
+// TMEM columns (512 allocated): tile i uses [256 i, 256 i + 128) for the two S/P buffers
+// (reused for the linear numerator) and [256 i + 128, 256 i + 128 + D) for O.
+#pragma once
+#include "ptx.cuh"
+
+namespace salad {
+
+enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
+
+struct FusedParams {
+    int N, H, nQb, nKb, nPairs, Bq, Hm, mode;
+    const int32_t* row_ptr;
+    const int32_t* col_idx;
+    const float* static_scale;   // [H] or null (=1)
+    const float* dyn_scale;      // [B] or null (=1)
+    const float* z;              // [B*H, D] linear normaliser state
+    float* lse;                  // optional [B*H, N]
+    float scale_log2;            // softmax_scale * log2(e)
+    float eps;
+    int32_t* ws_status;          // library status word (never null)
+    int32_t* user_status;        // optional
+};
+
+template <int D>
+struct FusedCfg {
+    static constexpr int BK = 64;
+    static constexpr int CH = D / 64;               // 128-byte chunks per row
+    static constexpr int Q_CHUNK = 128 * 128;       // bytes of one 64-column chunk of a Q tile
+    static constexpr int Q_BYTES = CH * Q_CHUNK;
+    static constexpr int KV_CHUNK = BK * 128;
+    static constexpr int KV_BYTES = CH * KV_CHUNK;  // one K or V tile
+    static constexpr int ST_CHUNK = D * 128;
+    static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]
+    static constexpr int NK = 4, NV = 4;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_ST = 2 * Q_BYTES;
+    static constexpr int OFF_K = OFF_ST + ST_BYTES;
+    static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
+    static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
+    static constexpr int THREADS = 384;
+};
+
+struct FusedBarriers {
+    uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
+    uint64_t s_full[2][2], p_ready[2][2], pv_done[2], lin_ready[2], lin_done[2], out_staged[2], o_final[2];
+};
+
+// Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
+struct MergeWalk {
+    const int32_t* col;
+    int e0, end0, e1, end1;
+    __device__ __forceinline__ bool next(int& c, int& tag) {
+        const int c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff;
+        const int c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff;
+        c = min(c0, c1);
+        if (c == 0x7fffffff) return false;
+        tag = (c0 == c ? 1 : 0) | (c1 == c ? 2 : 0);
+        e0 += (c0 == c); e1 += (c1 == c);
+        return true;
+    }
+};
+
+template <int D>
+__global__ void __launch_bounds__(384, 1)
+salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                   const __grid_constant__ CUtensorMap map_st, const FusedParams p)
+{
+    using C = FusedCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ FusedBarriers bars;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t s_base = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    const int pair = blockIdx.x % p.nPairs, bh = blockIdx.x / p.nPairs;
+    const int h = bh % p.H, b = bh / p.H;
+    const int hm = (p.Hm == 1) ? 0 : h;
+    const bool sparse = (p.mode & MODE_SPARSE) != 0, linear = (p.mode & MODE_LINEAR) != 0;
+
+    // kept lists of the two tiles
+    int qb[2], ls[2], le[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        qb[i] = 2 * pair + i;
+        ls[i] = le[i] = 0;
+        if (sparse && qb[i] < p.nQb) {
+            ls[i] = __ldg(p.row_ptr + hm * p.nQb + qb[i]);
+            le[i] = __ldg(p.row_ptr + hm * p.nQb + qb[i] + 1);
+        }
+    }
+
+    // ------------------------------------------------------------------ set-up
+    if (tid == 0) {
+        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&bars.q_full[i]), 1);
+            mbar_init(smem_u32(&bars.pv_done[i]), 1);
+            mbar_init(smem_u32(&bars.lin_ready[i]), 128);
+            mbar_init(smem_u32(&bars.lin_done[i]), 1);
+            mbar_init(smem_u32(&bars.out_staged[i]), 128);
+            mbar_init(smem_u32(&bars.o_final[i]), 1);
+            for (int j = 0; j < 2; ++j) {
+                mbar_init(smem_u32(&bars.s_full[i][j]), 1);
+                mbar_init(smem_u32(&bars.p_ready[i][j]), 128);
+            }
+        }
+        mbar_init(smem_u32(&bars.st_full), 1);
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        fence_mbar_init();
+    }
+    if (p.Bq < 128) {
+        // rows [Bq, 128) of the Q tiles are never written by TMA: zero them so the unused
+        // half of the MMA tile holds finite numbers
+        for (int i = tid; i < 2 * C::CH * (128 - p.Bq) * 8; i += C::THREADS) {
+            const int chunk = i / ((128 - p.Bq) * 8), rest = i % ((128 - p.Bq) * 8);
+            *reinterpret_cast<uint4*>(smem + C::OFF_Q + chunk * C::Q_CHUNK + p.Bq * 128 + rest * 16) =
+                make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    if (abort_flag == 0) {
+    if (warp == 0) {
+        // ============================================================== TMA producer
+        if (lane == 0) {
+            prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+            for (int i = 0; i < 2; ++i) {
+                if (qb[i] >= p.nQb) continue;
+                const uint32_t bar = smem_u32(&bars.q_full[i]);
+                mbar_arrive_expect_tx(bar, uint32_t(p.Bq) * D * 2);
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_load_3d(s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, &map_q, bar,
+                                ch * 64, qb[i] * p.Bq, bh);
+            }
+            if (linear) {
+                const uint32_t bar = smem_u32(&bars.st_full);
+                mbar_arrive_expect_tx(bar, C::ST_BYTES);
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_load_3d(s_base + C::OFF_ST + ch * C::ST_CHUNK, &map_st, bar, ch * 64, 0, bh);
+            }
+            MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
+            int col, tag, gk = 0, gv = 0, prev_col = -1;
+            bool ok = true;
+            auto load_tile = [&](const CUtensorMap* m, uint32_t off, uint64_t* full, uint64_t* empty,
+                                 int g, int n_stage, int c) -> bool {
+                const int s = g % n_stage;
+                if (!mbar_wait(smem_u32(&empty[s]), ((g / n_stage) & 1) ^ 1, abortp)) return false;
+                const uint32_t bar = smem_u32(&full[s]);
+                mbar_arrive_expect_tx(bar, C::KV_BYTES);
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_load_3d(s_base + off + s * C::KV_BYTES + ch * C::KV_CHUNK, m, bar, ch * 64,
+                                c * C::BK, bh);
+                return true;
+            };
+            // order of need: K(0), K(1), V(0), K(2), V(1), ...
+            while (ok && wk.next(col, tag)) {
+                ok = load_tile(&map_k, C::OFF_K, bars.k_full, bars.k_empty, gk++, C::NK, col);
+                if (ok && prev_col >= 0)
+                    ok = load_tile(&map_v, C::OFF_V, bars.v_full, bars.v_empty, gv++, C::NV, prev_col);
+                prev_col = col;
+            }
+            if (ok && prev_col >= 0)
+                ok = load_tile(&map_v, C::OFF_V, bars.v_full, bars.v_empty, gv++, C::NV, prev_col);
+        }
+    } else if (warp == 1) {
+        // ============================================================== MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
+            const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+            const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
+            bool ok = true;
+            for (int i = 0; i < 2 && ok; ++i)
+                if (qb[i] < p.nQb && (le[i] > ls[i]))
+                    ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
+            tc_fence_after_sync();
+            MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
+            int tq[2] = {0, 0};   // QK issued per tile
+            int tp[2] = {0, 0};   // PV issued per tile
+            int gk = 0, gv = 0;
+            auto issue_qk = [&](int tag) -> bool {
+                const int s = gk % C::NK;
+                if (!mbar_wait(smem_u32(&bars.k_full[s]), (gk / C::NK) & 1, abortp)) return false;
+                tc_fence_after_sync();
+                const uint32_t kb = s_base + C::OFF_K + s * C::KV_BYTES;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    if (!(tag & (1 << i))) continue;
+                    const uint32_t qa = s_base + C::OFF_Q + i * C::Q_BYTES;
+                    const uint32_t dcol = tmem + i * 256 + (tq[i] & 1) * 64;
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t da = make_sdesc_sw128(qa + (k / 4) * C::Q_CHUNK + (k % 4) * 32, 16, 1024);
+                        const uint64_t db = make_sdesc_sw128(kb + (k / 4) * C::KV_CHUNK + (k % 4) * 32, 16, 1024);
+                        mma_ss(dcol, da, db, idesc_qk, k > 0);
+                    }
+                    tc_commit(smem_u32(&bars.s_full[i][tq[i] & 1]));
+                    ++tq[i];
+                }
+                tc_commit(smem_u32(&bars.k_empty[s]));
+                ++gk;
+                return true;
+            };
+            int col, tag, ncol, ntag;
+            bool have = ok && wk.next(col, tag);
+            if (have) ok = issue_qk(tag);
+            while (ok && have) {
+                const bool have_next = wk.next(ncol, ntag);
+                if (have_next) ok = issue_qk(ntag);
+                if (!ok) break;
+                const int s = gv % C::NV;
+                ok = mbar_wait(smem_u32(&bars.v_full[s]), (gv / C::NV) & 1, abortp);
+                if (!ok) break;
+                const uint32_t vb = s_base + C::OFF_V + s * C::KV_BYTES;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    if (!(tag & (1 << i))) continue;
+                    const int t = tp[i];
+                    ok = mbar_wait(smem_u32(&bars.p_ready[i][t & 1]), (t >> 1) & 1, abortp);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t pcol = tmem + i * 256 + (t & 1) * 64;
+                    const uint32_t ocol = tmem + i * 256 + 128;
+#pragma unroll
+                    for (int k = 0; k < C::BK / 16; ++k) {
+                        const uint64_t db = make_sdesc_sw128(vb + k * 2048, C::KV_CHUNK, 1024);
+                        mma_ts(ocol, pcol + k * 8, db, idesc_pv, (t > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&bars.pv_done[i]));
+                    ++tp[i];
+                    if (tp[i] == le[i] - ls[i]) tc_commit(smem_u32(&bars.o_final[i]));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&bars.v_empty[s]));
+                ++gv;
+                have = have_next; col = ncol; tag = ntag;
+            }
+            if (ok && linear) {
+                ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
+                for (int i = 0; i < 2 && ok; ++i) {
+                    if (qb[i] >= p.nQb) continue;
+                    ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t qa = s_base + C::OFF_Q + i * C::Q_BYTES;
+                    const uint32_t sb = s_base + C::OFF_ST;
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t da = make_sdesc_sw128(qa + (k / 4) * C::Q_CHUNK + (k % 4) * 32, 16, 1024);
+                        const uint64_t db = make_sdesc_sw128(sb + (k / 4) * C::ST_CHUNK + (k % 4) * 32, 16, 1024);
+                        mma_ss(tmem + i * 256, da, db, idesc_lin, k > 0);
+                    }
+                    tc_commit(smem_u32(&bars.lin_done[i]));
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // ============================================================== softmax + epilogue
+        const int i = (warp - 4) >> 2;            // tile
+        const int row = tid - 128 - 128 * i;      // query row within the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t t_tile = tmem + i * 256 + lane_addr;
+        const bool tile_valid = qb[i] < p.nQb;
+        const int len = le[i] - ls[i];
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        // every lane of a warp must take the same path around the warp-collective tcgen05
+        // loads/stores, so the outcome of a bounded wait is made warp-uniform
+        auto wait_uniform = [&](uint64_t* bar, uint32_t parity) -> bool {
+            return __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, abortp));
+        };
+
+        for (int t = 0; t < len && ok; ++t) {
+            const int buf = t & 1;
+            ok = wait_uniform(&bars.s_full[i][buf], (t >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t xr[64];
+            tmem_ld32(t_tile + buf * 64, xr);
+            tmem_ld32(t_tile + buf * 64 + 32, xr + 32);
+            tmem_wait_ld();
+            float* x = reinterpret_cast<float*>(xr);
+            const int col = __ldg(p.col_idx + ls[i] + t);
+            const int valid = p.N - col * C::BK;          // keys of this block that exist
+            if (valid < C::BK) {
+#pragma unroll
+                for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
+            }
+            float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
+#pragma unroll
+            for (int c = 4; c < C::BK; c += 4) {
+                mx0 = fmaxf(mx0, x[c]); mx1 = fmaxf(mx1, x[c + 1]);
+                mx2 = fmaxf(mx2, x[c + 2]); mx3 = fmaxf(mx3, x[c + 3]);
+            }
+            const float msc = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+            if (t == 0) {
+                m_run = msc;
+            } else {
+                const bool need = msc > m_run + 8.0f;
+                if (__any_sync(0xffffffffu, need)) {
+                    // bring the accumulator of this warp's rows to the new running max
+                    ok = wait_uniform(&bars.pv_done[i], (t - 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const float m_new = fmaxf(m_run, msc);
+                    const float alpha = ex2_approx(m_run - m_new);
+                    l_run *= alpha;
+                    m_run = m_new;
+#pragma unroll
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t orr[32];
+                        tmem_ld32(t_tile + 128 + cc * 32, orr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                        tmem_st32(t_tile + 128 + cc * 32, orr);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            uint32_t pk[32];
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < C::BK; c += 2) {
+                const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_run));
+                const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_run));
+                s0 += p0; s1 += p1;
+                pk[c >> 1] = pack_bf16x2(p0, p1);
+            }
+            l_run += s0 + s1;
+            tmem_st32(t_tile + buf * 64, pk);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&bars.p_ready[i][buf]));
+        }
+        if (ok && len > 0) {
+            // pv_done cycles once per block and is only safe to test one phase back (as the
+            // rescale does); the end of the last P V product has a barrier of its own
+            ok = wait_uniform(&bars.o_final[i], 0);
+            tc_fence_after_sync();
+        }
+
+        float lin_coef = 0.f;
+        if (ok && tile_valid && linear) {
+            // ReLU of this thread's Q row in place, and the denominator ReLU(Q_n) . Z
+            ok = wait_uniform(&bars.q_full[i], 0);
+            if (ok) {
+                const float* zrow = p.z + size_t(bh) * D;
+                float den = 0.f;
+                uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
+#pragma unroll
+                for (int ch = 0; ch < C::CH; ++ch) {
+#pragma unroll
+                    for (int c16 = 0; c16 < 8; ++c16) {
+                        uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
+                                                              ((c16 ^ (row & 7)) << 4));
+                        uint4 v = *ptr;
+                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
+                            const float2 f = __bfloat1622float2(hv[e]);
+                            const int a = ch * 64 + c16 * 8 + e * 2;
+                            den = fmaf(f.x, __ldg(zrow + a), den);
+                            den = fmaf(f.y, __ldg(zrow + a + 1), den);
+                        }
+                        *ptr = v;
+                    }
+                }
+                float c_scale = 1.f;
+                if (p.static_scale) c_scale *= __ldg(p.static_scale + h);
+                if (p.dyn_scale) c_scale *= __ldg(p.dyn_scale + b);
+                lin_coef = c_scale / (den + p.eps);
+                fence_proxy_async_smem();
+                mbar_arrive(smem_u32(&bars.lin_ready[i]));
+                ok = wait_uniform(&bars.lin_done[i], 0);
+                tc_fence_after_sync();
+            }
+        }
+
+        if (ok && tile_valid) {
+            // O = O_acc / l + lin_coef * num, rounded once to bf16, staged in the Q tile
+            const float inv_l = (len > 0) ? 1.0f / l_run : 0.f;
+            uint8_t* stage = smem + C::OFF_Q + i * C::Q_BYTES;
+#pragma unroll
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t orr[32], nr[32];
+                if (len > 0) tmem_ld32(t_tile + 128 + cc * 32, orr);
+                if (linear) tmem_ld32(t_tile + cc * 32, nr);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int c = c8 * 8 + e * 2;
+                        float o0 = (len > 0) ? __uint_as_float(orr[c]) * inv_l : 0.f;
+                        float o1 = (len > 0) ? __uint_as_float(orr[c + 1]) * inv_l : 0.f;
+                        if (linear) {
+                            o0 = fmaf(lin_coef, __uint_as_float(nr[c]), o0);
+                            o1 = fmaf(lin_coef, __uint_as_float(nr[c + 1]), o1);
+                        }
+                        w[e] = pack_bf16x2(o0, o1);
+                    }
+                    const int col16 = (cc * 32 + c8 * 8) / 8;      // 16-byte chunk index within the row
+                    const int ch = col16 / 8, c16 = col16 % 8;
+                    *reinterpret_cast<uint4*>(stage + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(smem_u32(&bars.out_staged[i]));
+            if (row == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_store_3d(&map_o, s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, ch * 64,
+                                 qb[i] * p.Bq, bh);
+                tma_store_commit();
+                tma_store_wait_all();
+            }
+            if (p.lse != nullptr) {
+                const int n = qb[i] * p.Bq + row;
+                if (row < p.Bq && n < p.N)
+                    p.lse[size_t(bh) * p.N + n] =
+                        (len > 0) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            }
+        }
+    }
+    }  // abort_flag == 0
+
+    // ------------------------------------------------------------------ tear-down
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag != 0) {
+        // a bounded wait expired somewhere: report, give copies in flight time to land, leave
+        if (tid == 0) {
+            atomicExch(p.ws_status, 1);
+            if (p.user_status) atomicExch(p.user_status, -6);
+        }
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace salad

@@ -1,0 +1,220 @@
+// Linear-attention state (Eq. 3):  KV = sum_j ReLU(K_j)^T V_j  (d x d),  Z = sum_j ReLU(K_j).
+//
+// HBM-bound: K and V are read exactly once.  The token axis of every (batch, head) is cut
+// into `chunks` contiguous ranges of key blocks (64 tokens); one CTA streams one range:
+//   warp 0      TMA producer, K and V tiles through a ring of stages
+//   warp 1      tcgen05 MMA issuer; per 16 tokens one MMA  D[d x d] += ReLU(K)^T V with both
+//               operands token-major in shared memory (MN-major descriptors), plus one
+//               N = 16 MMA against an all-ones tile whose columns all equal Z
+//   warps 2-5   apply ReLU to the K tile in place in shared memory (16-byte vectors), and at
+//               the end move the fp32 accumulator from TMEM to this chunk's partial in global
+//               memory
+// A second, tiny kernel adds the partials of a head in a fixed order (deterministic), and
+// emits the fp32 state plus the bf16, transposed copy that the fused attention kernel
+// multiplies with ReLU(Q).
+//
+// For d = 64 the MMA still uses M = 128: the "rows 64..127" of the MN-major A operand are
+// addressed through the leading-byte-offset, which is pointed at the V tile that follows
+// the K tile in the stage; those accumulator rows are ignored.
+#pragma once
+#include "ptx.cuh"
+
+namespace salad {
+
+template <int D>
+struct StateCfg {
+    static constexpr int BK = 64;
+    static constexpr int CH = D / 64;
+    static constexpr int T_CHUNK = BK * 128;           // bytes of one 64-column chunk of a tile
+    static constexpr int T_BYTES = CH * T_CHUNK;       // one K or V tile
+    static constexpr int STAGE_BYTES = 2 * T_BYTES;    // K then V
+    static constexpr int STAGES = (D == 128) ? 3 : 4;
+    static constexpr int OFF_ONES = STAGES * STAGE_BYTES;
+    static constexpr int SMEM_BYTES = OFF_ONES + 2048 + 1024;
+    static constexpr int THREADS = 192;
+    static constexpr int TMEM_COLS = 256;
+};
+
+struct StateParams {
+    int N, nKb, chunks, blocks_per_chunk;
+    float* kv_part;       // [BH][chunks][D][D]
+    float* z_part;        // [BH][chunks][D]
+    int32_t* ws_status;
+    int32_t* user_status;
+};
+
+template <int D>
+__global__ void __launch_bounds__(192)
+salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                          const StateParams p)
+{
+    using C = StateCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full[C::STAGES], relu_done[C::STAGES], empty[C::STAGES], acc_done;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t s_base = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk = blockIdx.x, bh = blockIdx.y;
+    const int kb0 = chunk * p.blocks_per_chunk;
+    const int kb1 = min(p.nKb, kb0 + p.blocks_per_chunk);
+    const int nblk = max(0, kb1 - kb0);
+
+    if (tid == 0) {
+        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&relu_done[s]), 128);
+            mbar_init(smem_u32(&empty[s]), 1);
+        }
+        mbar_init(smem_u32(&acc_done), 1);
+        fence_mbar_init();
+    }
+    // all-ones bf16 tile (0x3F80 = 1.0)
+    for (int i = tid; i < 2048 / 4; i += C::THREADS)
+        reinterpret_cast<uint32_t*>(smem + C::OFF_ONES)[i] = 0x3F803F80u;
+    fence_proxy_async_smem();
+    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    if (abort_flag == 0) {
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+            for (int g = 0; g < nblk; ++g) {
+                const int s = g % C::STAGES;
+                if (!mbar_wait(smem_u32(&empty[s]), ((g / C::STAGES) & 1) ^ 1, abortp)) break;
+                const uint32_t bar = smem_u32(&full[s]);
+                mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                const uint32_t dst = s_base + s * C::STAGE_BYTES;
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    tma_load_3d(dst + ch * C::T_CHUNK, &map_k, bar, ch * 64, (kb0 + g) * C::BK, bh);
+                    tma_load_3d(dst + C::T_BYTES + ch * C::T_CHUNK, &map_v, bar, ch * 64, (kb0 + g) * C::BK, bh);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc_kv = make_idesc_bf16(128, D, 1, 1);
+            const uint32_t idesc_z = make_idesc_bf16(128, 16, 1, 0);
+            const uint64_t ones = make_sdesc_sw128(s_base + C::OFF_ONES, 16, 1024);
+            bool ok = true;
+            for (int g = 0; g < nblk && ok; ++g) {
+                const int s = g % C::STAGES;
+                ok = mbar_wait(smem_u32(&relu_done[s]), (g / C::STAGES) & 1, abortp);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t ka = s_base + s * C::STAGE_BYTES, va = ka + C::T_BYTES;
+#pragma unroll
+                for (int k = 0; k < C::BK / 16; ++k) {
+                    // 16 tokens = 2 groups of 8 rows of 128 B; next 64 channels one chunk further
+                    const uint64_t da = make_sdesc_sw128(ka + k * 2048, C::T_CHUNK, 1024);
+                    const uint64_t db = make_sdesc_sw128(va + k * 2048, C::T_CHUNK, 1024);
+                    const uint32_t acc = (g > 0 || k > 0) ? 1u : 0u;
+                    mma_ss(tmem, da, db, idesc_kv, acc);
+                    mma_ss(tmem + D, da, ones, idesc_z, acc);
+                }
+                tc_commit(smem_u32(&empty[s]));
+            }
+            if (ok) tc_commit(smem_u32(&acc_done));
+        }
+    } else {
+        const int wt = tid - 64;                       // 0..127 within the ReLU/epilogue group
+        bool ok = true;
+        for (int g = 0; g < nblk && ok; ++g) {
+            const int s = g % C::STAGES;
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&full[s]), (g / C::STAGES) & 1, abortp));
+            if (!ok) break;
+            uint4* kt = reinterpret_cast<uint4*>(smem + s * C::STAGE_BYTES);
+            const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
+#pragma unroll
+            for (int i = 0; i < C::T_BYTES / 16 / 128; ++i) {
+                uint4 v = kt[i * 128 + wt];
+                __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+                hv[0] = __hmax2(hv[0], zero); hv[1] = __hmax2(hv[1], zero);
+                hv[2] = __hmax2(hv[2], zero); hv[3] = __hmax2(hv[3], zero);
+                kt[i * 128 + wt] = v;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(smem_u32(&relu_done[s]));
+        }
+        // accumulator -> this chunk's partial.  TMEM lane = key channel a; columns [0,D) = KV
+        // row a, column D = Z[a].
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&acc_done), 0, abortp));
+        if (ok) {
+            tc_fence_after_sync();
+            const int a = (warp & 3) * 32 + lane;       // lanes this warp may access
+            const uint32_t t_row = tmem + (uint32_t((warp & 3) * 32) << 16);
+            float* kv_row = p.kv_part + ((size_t(bh) * p.chunks + chunk) * D + a) * D;
+#pragma unroll
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t r[32];
+                if (nblk > 0) { tmem_ld32(t_row + cc * 32, r); tmem_wait_ld(); }
+                if (a < D) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        float4 o = nblk > 0 ? make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
+                                                          __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+                        *reinterpret_cast<float4*>(kv_row + cc * 32 + c) = o;
+                    }
+                }
+            }
+            uint32_t zr[32];
+            if (nblk > 0) { tmem_ld32(t_row + D, zr); tmem_wait_ld(); }   // reads 32 columns, uses the first
+            if (a < D)
+                p.z_part[(size_t(bh) * p.chunks + chunk) * D + a] = nblk > 0 ? __uint_as_float(zr[0]) : 0.f;
+        }
+    }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag != 0) {
+        if (tid == 0) {
+            atomicExch(p.ws_status, 1);
+            if (p.user_status) atomicExch(p.user_status, -6);
+        }
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+// Sum the partials of each head in chunk order; emit
+//   kv_out  fp32 [BH][D][D]  (optional)      z fp32 [BH][D]  (+ optional user copy)
+//   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
+//           num = ReLU(Q) KV in the fused kernel.
+template <int D>
+__global__ void __launch_bounds__(256)
+salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
+                             float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
+                             __nv_bfloat16* __restrict__ kvt)
+{
+    const int bh = blockIdx.y;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;     // a * D + c
+    if (idx < D * D) {
+        const float* src = kv_part + size_t(bh) * chunks * D * D + idx;
+        float s = 0.f;
+        for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D * D];
+        if (kv_out) kv_out[size_t(bh) * D * D + idx] = s;
+        const int a = idx / D, c = idx % D;
+        kvt[size_t(bh) * D * D + c * D + a] = __float2bfloat16(s);
+    }
+    if (idx < D) {
+        const float* src = z_part + size_t(bh) * chunks * D + idx;
+        float s = 0.f;
+        for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];
+        z_ws[size_t(bh) * D + idx] = s;
+        if (z_out) z_out[size_t(bh) * D + idx] = s;
+    }
+}
+
+}  // namespace salad

@@ -1,0 +1,98 @@
+// Static 3-D sliding-window block mask -> CSR lists of kept key blocks
+// (Sec. 3 static sparse attention; Appendix A.1 token flattening, time slowest).
+//
+// Block pair (i, j) is kept iff some query token of block i and some key token of block j
+// lie within (wt, wh, ww) of each other on the T x Hs x Ws grid.  Instead of enumerating
+// token pairs, each query token's window is intersected with the key block run by run:
+// a key block is a contiguous range [k0, k1) of flat token ids, i.e. a few grid rows
+// (t', h') each contributing one contiguous run of w'; the window of a query token selects,
+// in each such row, the run [w - ww, w + ww].  Two integer interval tests per row decide.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace salad {
+
+struct MaskGeom {
+    int T, Hs, Ws, N, Bq, Bk, nQb, nKb, Hm;
+};
+
+// Window sizes (wt, wh, ww) per mask head, passed by value as a kernel argument so that the
+// builder needs no device scratch.
+struct MaskWindows {
+    int32_t w[3 * 256];
+};
+
+__device__ __forceinline__ bool block_pair_kept(const MaskGeom& g, int i, int j, int wt, int wh, int ww) {
+    const int q0 = i * g.Bq, q1 = min(g.N, q0 + g.Bq);
+    const int k0 = j * g.Bk, k1 = min(g.N, k0 + g.Bk);
+    const int krow0 = k0 / g.Ws, krow1 = (k1 - 1) / g.Ws;   // grid rows (t*Hs + h) the key block touches
+    for (int n = q0; n < q1; ++n) {
+        const int qrow = n / g.Ws, w = n - qrow * g.Ws;
+        const int t = qrow / g.Hs, h = qrow - t * g.Hs;
+        const int wlo = max(0, w - ww), whi = min(g.Ws - 1, w + ww);
+        for (int r = krow0; r <= krow1; ++r) {
+            const int t2 = r / g.Hs, h2 = r - t2 * g.Hs;
+            if (abs(t2 - t) > wt || abs(h2 - h) > wh) continue;
+            const int lo = max(r * g.Ws + wlo, k0), hi = min(r * g.Ws + whi, k1 - 1);
+            if (lo <= hi) return true;
+        }
+    }
+    return false;
+}
+
+// One warp per CSR row.  FILL = false: write the row's count to counts[row + 1].
+// FILL = true: write the kept key-block ids, ascending, at row_ptr[row].
+template <bool FILL>
+__global__ void __launch_bounds__(256) mask_rows_kernel(const MaskGeom g, const __grid_constant__ MaskWindows windows,
+                                                        int32_t* __restrict__ row_ptr,
+                                                        int32_t* __restrict__ col_idx) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int rows = g.Hm * g.nQb;
+    if (warp >= rows) return;
+    const int hm = warp / g.nQb, i = warp - hm * g.nQb;
+    const int wt = windows.w[3 * hm], wh = windows.w[3 * hm + 1], ww = windows.w[3 * hm + 2];
+    int base = FILL ? row_ptr[warp] : 0;
+    int count = 0;
+    for (int j0 = 0; j0 < g.nKb; j0 += 32) {
+        const int j = j0 + lane;
+        const bool keep = (j < g.nKb) && block_pair_kept(g, i, j, wt, wh, ww);
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (FILL && keep) col_idx[base + count + __popc(m & ((1u << lane) - 1u))] = j;
+        count += __popc(m);
+    }
+    if (!FILL && lane == 0) row_ptr[warp + 1] = count;
+}
+
+// In-place exclusive scan of counts stored at row_ptr[1..rows] (row_ptr[0] = 0 afterwards,
+// row_ptr[rows] = nnz).  Single block.  If the total does not fit in int32, row_ptr[rows]
+// is set to -1.
+__global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ row_ptr, int rows) {
+    __shared__ long long part[1024];
+    const int tid = threadIdx.x;
+    const int per = (rows + 1023) / 1024;
+    const int lo = min(rows, tid * per), hi = min(rows, lo + per);
+    long long s = 0;
+    for (int r = lo; r < hi; ++r) s += row_ptr[r + 1];
+    part[tid] = s;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        long long add = (tid >= off) ? part[tid - off] : 0;
+        __syncthreads();
+        part[tid] += add;
+        __syncthreads();
+    }
+    long long run = part[tid] - s;   // exclusive prefix of this thread's segment
+    for (int r = lo; r < hi; ++r) {
+        const int c = row_ptr[r + 1];
+        run += c;
+        row_ptr[r + 1] = (int32_t)run;   // inclusive value belongs at index r + 1
+    }
+    __syncthreads();
+    if (tid == 0) {
+        row_ptr[0] = 0;
+        if (part[1023] > 2147483647ll) row_ptr[rows] = -1;
+    }
+}
+
+}  // namespace salad

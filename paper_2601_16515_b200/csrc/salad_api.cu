@@ -1,0 +1,306 @@
+// C ABI of libsalad (see include/salad.h): argument validation, workspace carving, TMA
+// tensor maps and kernel launches.  No allocation, no global state beyond per-device
+// "attributes already set" flags, no CPU fallback.
+#include "../../include/salad.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+
+#include "fused_kernel.cuh"
+#include "linear_state_kernel.cuh"
+#include "mask_kernels.cuh"
+#include "tmap.cuh"
+
+using namespace salad;
+
+#define SALAD_EXPORT extern "C" __attribute__((visibility("default")))
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kPartialSlots = 512;     // upper bound on (batch*heads) x chunks partial states
+constexpr int kMaxMaskHeads = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Workspace {
+    size_t off_status, off_kvt, off_z, off_kvp, off_zp, total;
+    int slots;
+};
+
+Workspace carve(int B, int H, int d) {
+    Workspace w;
+    const size_t BH = size_t(B) * H;
+    w.slots = int(BH > size_t(kPartialSlots) ? BH : size_t(kPartialSlots));
+    w.off_status = 0;
+    w.off_kvt = kAlign;
+    w.off_z = w.off_kvt + align_up(BH * d * d * 2);
+    w.off_kvp = w.off_z + align_up(BH * d * 4);
+    w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
+    w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
+    return w;
+}
+
+bool shape_supported(int d, int Bq, int Bk) {
+    return (d == 64 || d == 128) && (Bq == 64 || Bq == 128) && Bk == 64;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo { int sms; bool ok; };
+
+// sm_100 check and shared-memory opt-in, once per device.
+int prepare_device(DeviceInfo* info) {
+    static bool attr_set[64] = {};
+    static int sm_count[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return SALAD_ERR_CUDA;
+    if (!attr_set[dev]) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return SALAD_ERR_CUDA;
+        }
+        if (major != 10) return SALAD_ERR_CUDA;   // kernels exist for sm_100a only
+        cudaError_t e = cudaSuccess;
+        e = cudaFuncSetAttribute(salad_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 FusedCfg<128>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     FusedCfg<64>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64>::SMEM_BYTES);
+        if (e != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+        sm_count[dev] = sms;
+        attr_set[dev] = true;
+    }
+    info->sms = sm_count[dev];
+    info->ok = true;
+    return SALAD_OK;
+}
+
+int check_launch() {
+    return cudaGetLastError() == cudaSuccess ? SALAD_OK : SALAD_ERR_CUDA;
+}
+
+struct Problem {
+    const void *q, *k, *v; void* o; float* lse;
+    int B, H, N, d, Bq, Bk, Hm, mode;
+    const int32_t *row_ptr, *col_idx;
+    const float *static_scale, *dyn_scale;
+    float softmax_scale, eps;
+    float *kv_out, *z_out;
+    void* ws; size_t ws_bytes; int32_t* d_status; cudaStream_t stream;
+};
+
+int validate(const Problem& P) {
+    if (!P.q || !P.k || !P.v || !P.o) return SALAD_ERR_INVALID_ARG;
+    if (P.B <= 0 || P.H <= 0 || P.N <= 0 || P.d <= 0 || P.Bq <= 0 || P.Bk <= 0) return SALAD_ERR_INVALID_ARG;
+    if (!shape_supported(P.d, P.Bq, P.Bk)) return SALAD_ERR_UNSUPPORTED;
+    if (!aligned16(P.q) || !aligned16(P.k) || !aligned16(P.v) || !aligned16(P.o)) return SALAD_ERR_INVALID_ARG;
+    if (int64_t(P.B) * P.H > 65535) return SALAD_ERR_UNSUPPORTED;
+    if (P.mode & MODE_SPARSE) {
+        if (!P.row_ptr || !P.col_idx) return SALAD_ERR_INVALID_ARG;
+        if (P.Hm != 1 && P.Hm != P.H) return SALAD_ERR_INVALID_ARG;
+        if (!(P.softmax_scale >= 0.f) || !isfinite(P.softmax_scale)) return SALAD_ERR_INVALID_ARG;
+    }
+    if (P.mode & MODE_LINEAR) {
+        if (!(P.eps >= 0.f) || !isfinite(P.eps)) return SALAD_ERR_INVALID_ARG;
+    }
+    if (P.mode == MODE_FUSED && (!P.static_scale || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
+    const Workspace w = carve(P.B, P.H, P.d);
+    if (!P.ws || (reinterpret_cast<uintptr_t>(P.ws) % kAlign) != 0 || P.ws_bytes < w.total)
+        return SALAD_ERR_WORKSPACE;
+    return SALAD_OK;
+}
+
+template <int D>
+int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
+    const int BH = P.B * P.H;
+    const int nKb = (P.N + 63) / 64;
+    int chunks = (2 * dev.sms) / BH;
+    if (chunks < 1) chunks = 1;
+    if (chunks > nKb) chunks = nKb;
+    if (int64_t(chunks) * BH > w.slots) chunks = w.slots / BH;
+    const int bpc = (nKb + chunks - 1) / chunks;
+    uint8_t* ws = static_cast<uint8_t*>(P.ws);
+    CUtensorMap mk, mv;
+    if (!make_tmap_bf16_3d(&mk, P.k, D, P.N, BH, 64) || !make_tmap_bf16_3d(&mv, P.v, D, P.N, BH, 64))
+        return SALAD_ERR_CUDA;
+    StateParams sp;
+    sp.N = P.N; sp.nKb = nKb; sp.chunks = chunks; sp.blocks_per_chunk = bpc;
+    sp.kv_part = reinterpret_cast<float*>(ws + w.off_kvp);
+    sp.z_part = reinterpret_cast<float*>(ws + w.off_zp);
+    sp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    sp.user_status = P.d_status;
+    salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    salad_linear_finalize_kernel<D><<<dim3((D * D + 255) / 256, BH), 256, 0, P.stream>>>(
+        sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
+        reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt));
+    return check_launch();
+}
+
+template <int D>
+int launch_fused(const Problem& P, const Workspace& w) {
+    const int BH = P.B * P.H;
+    uint8_t* ws = static_cast<uint8_t*>(P.ws);
+    CUtensorMap mq, mk, mv, mo, ms;
+    if (!make_tmap_bf16_3d(&mq, P.q, D, P.N, BH, P.Bq) || !make_tmap_bf16_3d(&mk, P.k, D, P.N, BH, 64) ||
+        !make_tmap_bf16_3d(&mv, P.v, D, P.N, BH, 64) || !make_tmap_bf16_3d(&mo, P.o, D, P.N, BH, P.Bq) ||
+        !make_tmap_bf16_3d(&ms, ws + w.off_kvt, D, D, BH, D))
+        return SALAD_ERR_CUDA;
+    FusedParams fp;
+    fp.N = P.N; fp.H = P.H; fp.Bq = P.Bq; fp.Hm = P.Hm; fp.mode = P.mode;
+    fp.nQb = (P.N + P.Bq - 1) / P.Bq;
+    fp.nKb = (P.N + 63) / 64;
+    fp.nPairs = (fp.nQb + 1) / 2;
+    fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
+    fp.static_scale = P.static_scale; fp.dyn_scale = P.dyn_scale;
+    fp.z = reinterpret_cast<const float*>(ws + w.off_z);
+    fp.lse = P.lse;
+    const float sc = (P.softmax_scale > 0.f) ? P.softmax_scale : 1.0f / sqrtf(float(D));
+    fp.scale_log2 = sc * 1.4426950408889634f;
+    fp.eps = P.eps;
+    fp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    fp.user_status = P.d_status;
+    const int64_t grid = int64_t(fp.nPairs) * BH;
+    if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
+    salad_fused_kernel<D><<<unsigned(grid), FusedCfg<D>::THREADS, FusedCfg<D>::SMEM_BYTES, P.stream>>>(
+        mq, mk, mv, mo, ms, fp);
+    return check_launch();
+}
+
+int run(const Problem& P) {
+    int rc = validate(P);
+    if (rc != SALAD_OK) return rc;
+    DeviceInfo dev{};
+    rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    const Workspace w = carve(P.B, P.H, P.d);
+    uint8_t* ws = static_cast<uint8_t*>(P.ws);
+    if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    if (P.d_status && cudaMemsetAsync(P.d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SALAD_ERR_CUDA;
+    }
+    if (P.mode & MODE_LINEAR) {
+        rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
+        if (rc != SALAD_OK) return rc;
+    }
+    return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
+}
+
+}  // namespace
+
+SALAD_EXPORT const char* salad_status_string(int status) {
+    switch (status) {
+        case SALAD_OK: return "SALAD_OK";
+        case SALAD_ERR_INVALID_ARG: return "SALAD_ERR_INVALID_ARG";
+        case SALAD_ERR_UNSUPPORTED: return "SALAD_ERR_UNSUPPORTED";
+        case SALAD_ERR_WORKSPACE: return "SALAD_ERR_WORKSPACE";
+        case SALAD_ERR_CAPACITY: return "SALAD_ERR_CAPACITY";
+        case SALAD_ERR_CUDA: return "SALAD_ERR_CUDA";
+        case SALAD_ERR_TIMEOUT: return "SALAD_ERR_TIMEOUT";
+        default: return "SALAD_ERR_UNKNOWN";
+    }
+}
+
+SALAD_EXPORT size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk) {
+    if (B <= 0 || H <= 0 || N <= 0 || !shape_supported(d, Bq, Bk)) return 0;
+    return carve(B, H, d).total;
+}
+
+SALAD_EXPORT int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm, const int32_t* h_windows,
+                                  int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
+                                  int64_t* h_nnz, void* stream) {
+    if (T <= 0 || Hs <= 0 || Ws <= 0 || Bq <= 0 || Bk <= 0 || Hm <= 0 || !h_windows || !d_row_ptr)
+        return SALAD_ERR_INVALID_ARG;
+    if (col_capacity < 0 || (d_col_idx == nullptr && col_capacity != 0)) return SALAD_ERR_INVALID_ARG;
+    if (Hm > kMaxMaskHeads) return SALAD_ERR_UNSUPPORTED;
+    const int64_t N64 = int64_t(T) * Hs * Ws;
+    if (N64 > 2147483647ll / 2) return SALAD_ERR_UNSUPPORTED;
+    for (int i = 0; i < 3 * Hm; ++i) if (h_windows[i] < 0) return SALAD_ERR_INVALID_ARG;
+    MaskGeom g;
+    g.T = T; g.Hs = Hs; g.Ws = Ws; g.N = int(N64); g.Bq = Bq; g.Bk = Bk; g.Hm = Hm;
+    g.nQb = (g.N + Bq - 1) / Bq; g.nKb = (g.N + Bk - 1) / Bk;
+    const int64_t rows64 = int64_t(Hm) * g.nQb;
+    if (rows64 > (1 << 24)) return SALAD_ERR_UNSUPPORTED;
+    const int rows = int(rows64);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // The windows travel as a kernel argument; the per-row counts are scanned in place in
+    // row_ptr; row_ptr[rows] doubles as the overflow probe target before it is overwritten.
+    MaskWindows win;
+    for (int i = 0; i < 3 * kMaxMaskHeads; ++i) win.w[i] = (i < 3 * Hm) ? h_windows[i] : 0;
+    const int blocks = (rows * 32 + 255) / 256;
+    mask_rows_kernel<false><<<blocks, 256, 0, st>>>(g, win, d_row_ptr, nullptr);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    mask_scan_kernel<<<1, 1024, 0, st>>>(d_row_ptr, rows);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    int32_t last = 0;
+    if (cudaMemcpyAsync(&last, d_row_ptr + rows, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return SALAD_ERR_CUDA;
+    }
+    if (last < 0) return SALAD_ERR_UNSUPPORTED;     // more than 2^31 - 1 kept blocks
+    if (h_nnz) *h_nnz = last;
+    if (!d_col_idx) return SALAD_OK;
+    if (col_capacity < last) return SALAD_ERR_CAPACITY;
+    mask_rows_kernel<true><<<blocks, 256, 0, st>>>(g, win, d_row_ptr, d_col_idx);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    return SALAD_OK;
+}
+
+SALAD_EXPORT int salad_sparse_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                                       int B, int H, int N, int d, int Bq, int Bk,
+                                       const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                       float softmax_scale, void* workspace, size_t workspace_bytes,
+                                       int32_t* d_status, void* stream) {
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o; P.lse = lse;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_SPARSE;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.softmax_scale = softmax_scale; P.eps = 0.f;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_linear_attn_fwd(const void* q, const void* k, const void* v, void* o_l,
+                                       float* kv_out, float* z_out, int B, int H, int N, int d, float eps,
+                                       void* workspace, size_t workspace_bytes, int32_t* d_status,
+                                       void* stream) {
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o_l;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
+    P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_fused_fwd(const void* q, const void* k, const void* v, void* o,
+                                 int B, int H, int N, int d, int Bq, int Bk,
+                                 const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                 const float* d_static_scale, const float* d_dyn_scale,
+                                 float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                                 int32_t* d_status, void* stream) {
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale;
+    P.softmax_scale = softmax_scale; P.eps = eps;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}

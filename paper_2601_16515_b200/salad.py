@@ -1,0 +1,180 @@
+"""ctypes binding of ``libsalad.so``: the same entry points as ``include/salad.h``.
+
+The functions here only marshal arguments (tensor -> device pointer, sizes, the current
+CUDA stream) and allocate outputs / workspace with torch when the caller does not pass
+them.  Every step of the attention path runs inside the CUDA library; there is no other
+implementation to fall back to: if the library is missing, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsalad.so")
+
+SALAD_OK = 0
+SALAD_ERR_INVALID_ARG = -1
+SALAD_ERR_UNSUPPORTED = -2
+SALAD_ERR_WORKSPACE = -3
+SALAD_ERR_CAPACITY = -4
+SALAD_ERR_CUDA = -5
+SALAD_ERR_TIMEOUT = -6
+
+EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
+           "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd")
+
+
+class SaladError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where} failed: {status_string(code)} ({code})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2601_16515_b200.build` "
+            "(there is no non-CUDA implementation to fall back to)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i32, i64, f32, p, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+    lib.salad_status_string.restype = ctypes.c_char_p
+    lib.salad_status_string.argtypes = [i32]
+    lib.salad_workspace_bytes.restype = sz
+    lib.salad_workspace_bytes.argtypes = [i32] * 6
+    lib.salad_mask_build.restype = i32
+    lib.salad_mask_build.argtypes = [i32] * 6 + [p, p, p, i64, p, p]
+    lib.salad_sparse_attn_fwd.restype = i32
+    lib.salad_sparse_attn_fwd.argtypes = [p, p, p, p, p] + [i32] * 6 + [p, p, i32, f32, p, sz, p, p]
+    lib.salad_linear_attn_fwd.restype = i32
+    lib.salad_linear_attn_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [f32, p, sz, p, p]
+    lib.salad_fused_fwd.restype = i32
+    lib.salad_fused_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, p, sz, p, p]
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(code: int) -> str:
+    return _lib.salad_status_string(int(code)).decode()
+
+
+def _check(rc: int, where: str):
+    if rc != SALAD_OK:
+        raise SaladError(rc, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _bf16_4d(name: str, t: torch.Tensor):
+    if t.dtype != torch.bfloat16 or t.dim() != 4 or not t.is_contiguous() or not t.is_cuda:
+        raise ValueError(f"{name} must be a contiguous CUDA bf16 tensor [B, H, N, d]")
+
+
+def salad_workspace_bytes(B: int, H: int, N: int, d: int, Bq: int = 128, Bk: int = 64) -> int:
+    return int(_lib.salad_workspace_bytes(B, H, N, d, Bq, Bk))
+
+
+def alloc_workspace(B, H, N, d, Bq=128, Bk=64, device="cuda") -> torch.Tensor:
+    n = salad_workspace_bytes(B, H, N, d, Bq, Bk)
+    if n == 0:
+        raise SaladError(SALAD_ERR_UNSUPPORTED, "salad_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def salad_mask_build(T: int, Hs: int, Ws: int, Bq: int, Bk: int,
+                     windows: Sequence[Tuple[int, int, int]], device="cuda",
+                     stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Sliding-window block mask -> (row_ptr int32 [Hm*nQb+1], col_idx int32 [nnz]) on device."""
+    Hm = len(windows)
+    flat = [int(x) for w in windows for x in w]
+    h_win = (ctypes.c_int32 * max(1, len(flat)))(*flat)
+    N = T * Hs * Ws
+    nQb = -(-N // Bq)
+    row_ptr = torch.empty(Hm * nQb + 1, dtype=torch.int32, device=device)
+    nnz = ctypes.c_int64(-1)
+    with torch.cuda.device(row_ptr.device):
+        _check(_lib.salad_mask_build(T, Hs, Ws, Bq, Bk, Hm, h_win, _ptr(row_ptr), None, 0,
+                                     ctypes.byref(nnz), _stream(stream)), "salad_mask_build")
+        col_idx = torch.empty(max(1, nnz.value), dtype=torch.int32, device=device)
+        _check(_lib.salad_mask_build(T, Hs, Ws, Bq, Bk, Hm, h_win, _ptr(row_ptr), _ptr(col_idx),
+                                     col_idx.numel(), ctypes.byref(nnz), _stream(stream)), "salad_mask_build")
+    return row_ptr, col_idx[:nnz.value]
+
+
+def _common(q, k, v, Bq, Bk, workspace):
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _bf16_4d(name, t)
+    if k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("q, k, v must have the same shape")
+    B, H, N, d = q.shape
+    if workspace is None:
+        workspace = alloc_workspace(B, H, N, d, Bq, Bk, q.device)
+    return B, H, N, d, workspace
+
+
+def _i32(name, t):
+    if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA int32 tensor")
+
+
+def salad_sparse_attn_fwd(q, k, v, row_ptr, col_idx, Hm: int, Bq: int = 128, Bk: int = 64,
+                          softmax_scale: float = 0.0, out=None, lse=None, workspace=None,
+                          status=None, stream=None):
+    """Block-sparse softmax attention.  Returns `out` (bf16 [B,H,N,d]); pass `lse` (fp32
+    [B,H,N]) to receive the row log-sum-exp as well."""
+    B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    if out is None:
+        out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_sparse_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, N, d, Bq, Bk,
+                                          _ptr(row_ptr), _ptr(col_idx), Hm, float(softmax_scale),
+                                          _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream)),
+               "salad_sparse_attn_fwd")
+    return out
+
+
+def salad_linear_attn_fwd(q, k, v, eps: float = 1e-6, out=None, kv_out=None, z_out=None,
+                          workspace=None, status=None, stream=None):
+    """ReLU linear attention.  Returns `out` (bf16 [B,H,N,d]); `kv_out` fp32 [B,H,d,d] and
+    `z_out` fp32 [B,H,d] receive the state when given."""
+    B, H, N, d, workspace = _common(q, k, v, 128, 64, workspace)
+    if out is None:
+        out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_linear_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_out), _ptr(z_out),
+                                          B, H, N, d, float(eps), _ptr(workspace), workspace.numel(),
+                                          _ptr(status), _stream(stream)), "salad_linear_attn_fwd")
+    return out
+
+
+def salad_fused_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_scale, Bq: int = 128,
+                    Bk: int = 64, softmax_scale: float = 0.0, eps: float = 1e-6, out=None,
+                    workspace=None, status=None, stream=None):
+    """O = O_sparse + dyn_scale[b] * static_scale[h] * O_linear, one bf16 write."""
+    B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    for name, t, n in (("static_scale", static_scale, H), ("dyn_scale", dyn_scale, B)):
+        if t.dtype != torch.float32 or not t.is_cuda or t.numel() != n or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor with {n} elements")
+    if out is None:
+        out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_fused_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                    _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale),
+                                    float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
+                                    _ptr(status), _stream(stream)), "salad_fused_fwd")
+    return out

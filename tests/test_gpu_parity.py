@@ -1,0 +1,301 @@
+"""GPU parity: every entry point of libsalad, called through the C ABI binding, against the
+CPU oracle on the same seeded inputs.  Mask lists are compared bit for bit; bf16 outputs
+within max-abs 2e-2 and relative-L2 1e-2 (the tolerance of the benchmark spec; the bf16
+rounding of an O(1) output alone is up to 2^-9 relative, and P is rounded to bf16 before the
+P V product)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import salad_oracle as orc
+from paper_2601_16515_b200 import workloads as wlmod
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+REL_L2 = 1e-2
+
+
+@pytest.fixture(scope="module")
+def salad():
+    from paper_2601_16515_b200 import salad as s
+    return s
+
+
+def assert_close(got, ref, what=""):
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    max_abs = np.abs(got - ref).max()
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert max_abs <= MAX_ABS and rel <= REL_L2, f"{what}: max_abs {max_abs:.4g} rel_l2 {rel:.4g}"
+    return max_abs, rel
+
+
+def status_ok(status):
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "kernel reported an expired wait"
+
+
+def bf16(a):
+    return torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16)
+
+
+def rand_qkv(B, H, N, d, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return tuple(bf16(rng.standard_normal((B, H, N, d)) * scale) for _ in range(3))
+
+
+def random_csr(rows, nKb, seed, lo=0, hi=None):
+    rng = np.random.default_rng(seed)
+    hi = nKb if hi is None else hi
+    rp, cols = [0], []
+    for _ in range(rows):
+        row = np.sort(rng.choice(nKb, size=int(rng.integers(lo, hi + 1)), replace=False))
+        cols.append(row); rp.append(rp[-1] + len(row))
+    ci = np.concatenate(cols).astype(np.int32) if rp[-1] else np.zeros(0, np.int32)
+    return np.asarray(rp, np.int32), ci
+
+
+def dev_csr(rp, ci):
+    ci_d = torch.from_numpy(ci if len(ci) else np.zeros(1, np.int32)).cuda()
+    return torch.from_numpy(rp).cuda(), ci_d
+
+
+def f32(t):
+    return t.float().numpy()
+
+
+# ------------------------------------------------------------------------------ mask builder
+
+MASK_CASES = [
+    ((2, 2, 4), 4, 4, [(0, 1, 0)]),
+    ((3, 5, 7), 16, 8, [(1, 1, 2), (0, 0, 0), (3, 5, 7)]),
+    ((4, 6, 6), 32, 16, [(0, 2, 2), (2, 0, 0)]),
+    ((2, 9, 11), 64, 32, [(1, 3, 4)]),
+    ((5, 3, 1), 4, 8, [(1, 1, 0)]),                       # Ws = 1: key blocks span many grid rows
+    (wlmod.C1.grid, 64, 64, list(wlmod.C1.windows)),
+    (wlmod.C1.grid, 64, 64, [(1, 1, 1), (0, 5, 5)]),
+    (wlmod.C2.grid, 128, 64, [(2, 5, 24), (5, 5, 24), (1, 4, 24), (21, 30, 52), (0, 0, 0)]),
+]
+
+
+@pytest.mark.parametrize("grid,Bq,Bk,windows", MASK_CASES)
+def test_mask_bit_exact(salad, grid, Bq, Bk, windows):
+    T, Hs, Ws = grid
+    rp, ci = salad.salad_mask_build(T, Hs, Ws, Bq, Bk, windows)
+    rp_ref, ci_ref = orc.mask_build(T, Hs, Ws, Bq, Bk, windows)
+    assert np.array_equal(rp.cpu().numpy(), rp_ref)
+    assert np.array_equal(ci.cpu().numpy(), ci_ref)
+
+
+def test_mask_bit_exact_wan14b_shape(salad):
+    wl = wlmod.C4
+    T, Hs, Ws = wl.grid
+    rp, ci = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    rp_ref, ci_ref = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    assert np.array_equal(rp.cpu().numpy(), rp_ref) and np.array_equal(ci.cpu().numpy(), ci_ref)
+    sparsity = 1.0 - len(ci_ref) / (wl.nQb * wl.nKb)
+    assert 0.89 < sparsity < 0.91
+
+
+def test_mask_capacity_error(salad):
+    import ctypes
+    T, Hs, Ws = wlmod.C1.grid
+    win = (ctypes.c_int32 * 3)(0, 15, 15)
+    rp = torch.empty(17, dtype=torch.int32, device="cuda")
+    ci = torch.full((8,), -7, dtype=torch.int32, device="cuda")
+    nnz = ctypes.c_int64(0)
+    rc = salad._lib.salad_mask_build(T, Hs, Ws, 64, 64, 1, win, ctypes.c_void_p(rp.data_ptr()),
+                                     ctypes.c_void_p(ci.data_ptr()), 8, ctypes.byref(nnz), None)
+    assert rc == salad.SALAD_ERR_CAPACITY and nnz.value == 64
+    assert (ci.cpu() == -7).all()
+
+
+# ------------------------------------------------------------------------------ sparse branch
+
+SMALL_SHAPES = [
+    # B, H, N, d, Bq, Hm
+    (1, 2, 1024, 64, 64, 2),
+    (1, 2, 1024, 128, 128, 1),
+    (2, 3, 1000, 128, 128, 3),      # ragged: last q block 104 rows, last key block 40 keys
+    (1, 2, 200, 64, 128, 1),        # N < 2 tiles, ragged
+    (1, 1, 712, 64, 64, 1),         # odd number of 64-row query blocks (12), ragged
+    (1, 2, 1100, 128, 64, 2),
+]
+
+
+@pytest.mark.parametrize("B,H,N,d,Bq,Hm", SMALL_SHAPES)
+def test_sparse_random_lists(salad, B, H, N, d, Bq, Hm):
+    q, k, v = rand_qkv(B, H, N, d, 100 + N)
+    nQb, nKb = -(-N // Bq), -(-N // 64)
+    rp, ci = random_csr(Hm * nQb, nKb, 7 + N, lo=0, hi=nKb)       # includes empty and full rows
+    rp_d, ci_d = dev_csr(rp, ci)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device="cuda")
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_sparse_attn_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, Hm, Bq=Bq, lse=lse, status=status)
+    status_ok(status)
+    ref, ref_lse = orc.sparse_attn(f32(q), f32(k), f32(v), Bq, 64, rp, ci, Hm)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "sparse")
+    got_lse = lse.cpu().numpy().reshape(-1)
+    empty = np.isneginf(ref_lse)
+    assert np.array_equal(np.isneginf(got_lse), empty)
+    np.testing.assert_allclose(got_lse[~empty], ref_lse[~empty], atol=2e-3, rtol=1e-4)
+
+
+def test_sparse_all_kept_is_full_attention(salad):
+    B, H, N, d = 1, 2, 1000, 128
+    q, k, v = rand_qkv(B, H, N, d, 5)
+    rp, ci = wlmod.dense_csr(-(-N // 128), -(-N // 64), 1)
+    rp_d, ci_d = dev_csr(rp, ci)
+    out = salad.salad_sparse_attn_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1)
+    ref = torch.nn.functional.scaled_dot_product_attention(q.double(), k.double(), v.double())   # Eq. 1
+    assert_close(f32(out.cpu()), ref.numpy(), "dense")
+
+
+def test_sparse_softmax_scale_and_large_scores(salad):
+    # scores with a wide dynamic range force the running-max rescale of the accumulator
+    B, H, N, d = 1, 1, 1024, 128
+    q, k, _ = rand_qkv(B, H, N, d, 6, scale=3.0)
+    _, _, v = rand_qkv(B, H, N, d, 6, scale=1.0)       # outputs stay O(1): the tolerance is absolute
+    rp, ci = wlmod.dense_csr(N // 128, N // 64, 1)
+    rp_d, ci_d = dev_csr(rp, ci)
+    for scale in (0.25, 1.0 / np.sqrt(d)):
+        out = salad.salad_sparse_attn_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, softmax_scale=scale)
+        ref, _ = orc.sparse_attn(f32(q), f32(k), f32(v), 128, 64, rp, ci, 1, scale=scale)
+        assert_close(f32(out.cpu()).reshape(-1, d), ref, f"scale {scale}")
+
+
+# ------------------------------------------------------------------------------ linear branch
+
+@pytest.mark.parametrize("B,H,N,d", [(1, 2, 1024, 64), (2, 3, 1000, 128), (1, 1, 70, 128), (1, 2, 5000, 64)])
+def test_linear(salad, B, H, N, d):
+    q, k, v = rand_qkv(B, H, N, d, 200 + N)
+    kv = torch.empty((B, H, d, d), dtype=torch.float32, device="cuda")
+    z = torch.empty((B, H, d), dtype=torch.float32, device="cuda")
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_linear_attn_fwd(q.cuda(), k.cuda(), v.cuda(), eps=1e-6, kv_out=kv, z_out=z, status=status)
+    status_ok(status)
+    kv_ref, z_ref = orc.linear_state(f32(k), f32(v))
+    np.testing.assert_allclose(z.cpu().numpy(), z_ref, rtol=1e-4, atol=1e-3)
+    np.testing.assert_allclose(kv.cpu().numpy(), kv_ref, rtol=1e-3, atol=np.abs(kv_ref).max() * 1e-4)
+    ref = orc.linear_attn(f32(q), f32(k), f32(v), eps=1e-6)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "linear")
+
+
+def test_linear_nonpositive_q_gives_zero(salad):
+    B, H, N, d = 1, 1, 256, 64
+    q, k, v = rand_qkv(B, H, N, d, 1)
+    out = salad.salad_linear_attn_fwd((-q.abs()).cuda(), k.cuda(), v.cuda())
+    assert (out == 0).all()
+
+
+# ------------------------------------------------------------------------------ fused
+
+def run_fused(salad, wl, q, k, v, rp, ci, Hm, lam, s, **kw):
+    rp_d, ci_d = dev_csr(rp, ci)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, Hm,
+                                torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda(),
+                                Bq=wl.Bq, Bk=wl.Bk, status=status, **kw)
+    status_ok(status)
+    return out
+
+
+def test_fused_tiny_config_full(salad):
+    wl = wlmod.C1
+    q, k, v = wlmod.make_qkv(wl)
+    T, Hs, Ws = wl.grid
+    rp_d, ci_d = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    assert np.array_equal(rp_d.cpu().numpy(), rp) and np.array_equal(ci_d.cpu().numpy(), ci)
+    lam, s = wlmod.make_scales(wl)
+    out = run_fused(salad, wl, q, k, v, rp, ci, wl.Hm, lam, s)
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s)
+    assert_close(f32(out.cpu()).reshape(-1, wl.d), ref, "fused tiny")
+
+
+@pytest.mark.parametrize("B,H,N,d,Bq,Hm", SMALL_SHAPES)
+def test_fused_small_shapes(salad, B, H, N, d, Bq, Hm):
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), Bq, 64, (), 1)
+    q, k, v = rand_qkv(B, H, N, d, 300 + N)
+    rp, ci = random_csr(Hm * wl.nQb, wl.nKb, 17 + N, lo=0, hi=min(wl.nKb, 9))
+    rng = np.random.default_rng(N)
+    lam = rng.uniform(0, 1, H).astype(np.float32); s = rng.uniform(0, 1, B).astype(np.float32)
+    out = run_fused(salad, wl, q, k, v, rp, ci, Hm, lam, s)
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), Bq, 64, rp, ci, Hm, lam, s)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "fused small")
+
+
+def test_fused_zero_scale_is_sparse_bit_for_bit(salad):
+    wl = wlmod.C1
+    q, k, v = wlmod.make_qkv(wl)
+    T, Hs, Ws = wl.grid
+    rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    lam, s = wlmod.make_scales(wl)
+    fused0 = run_fused(salad, wl, q, k, v, rp, ci, wl.Hm, np.zeros_like(lam), s)
+    rp_d, ci_d = dev_csr(rp, ci)
+    sparse = salad.salad_sparse_attn_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, wl.Hm, Bq=wl.Bq)
+    assert torch.equal(fused0, sparse)
+    # and the fused result equals sparse + scale * linear computed by the standalone calls
+    fused = run_fused(salad, wl, q, k, v, rp, ci, wl.Hm, lam, s)
+    lin = salad.salad_linear_attn_fwd(q.cuda(), k.cuda(), v.cuda())
+    c = torch.from_numpy(s)[:, None] * torch.from_numpy(lam)[None, :]
+    comb = sparse.float().cpu() + c[:, :, None, None] * lin.float().cpu()
+    assert_close(f32(fused.cpu()), comb.numpy(), "fused vs parts")
+
+
+def sampled_fused_check(salad, wl, heads, nrows, windows=None, csr=None):
+    """Full-size run on the GPU, oracle on sampled rows of a subset of heads."""
+    q, k, v = wlmod.make_qkv(wl)
+    T, Hs, Ws = wl.grid
+    lam, s = wlmod.make_scales(wl)
+    if csr is None:
+        windows = wl.windows if windows is None else windows
+        rp_d, ci_d = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, windows)
+        rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, windows)
+        assert np.array_equal(rp_d.cpu().numpy(), rp) and np.array_equal(ci_d.cpu().numpy(), ci)
+        Hm = len(windows)
+    else:
+        rp, ci = csr
+        Hm = wl.H
+    out = run_fused(salad, wl, q, k, v, rp, ci, Hm, lam, s).cpu()
+    assert torch.isfinite(out.float()).all()
+    # oracle on the chosen heads only (identical slices of the same tensors)
+    qs, ks, vs = (f32(t[:, heads].contiguous()) for t in (q, k, v))
+    sub = wlmod.Workload("sub", wl.B, len(heads), wl.d, wl.grid, wl.Bq, wl.Bk, wl.windows, wl.seed)
+    sel = wlmod.sample_rows(sub, nrows)
+    if Hm == 1:
+        rp_s, ci_s, Hm_s = rp, ci, 1
+    else:   # per-head lists: gather the rows of the chosen heads
+        nQb = wl.nQb
+        rows, rp_s = [], [0]
+        for h in heads:
+            for i in range(nQb):
+                r = h * nQb + i
+                rows.append(ci[rp[r]:rp[r + 1]]); rp_s.append(rp_s[-1] + rows[-1].size)
+        rp_s, ci_s, Hm_s = np.asarray(rp_s, np.int32), np.concatenate(rows).astype(np.int32), len(heads)
+    ref = orc.salad_fused(qs, ks, vs, wl.Bq, wl.Bk, rp_s, ci_s, Hm_s, lam[heads], s, sel=sel)
+    got = f32(out[:, heads].contiguous()).reshape(-1, wl.d)[sel]
+    return assert_close(got, ref, wl.name)
+
+
+def test_fused_wan13b_90(salad):
+    sampled_fused_check(salad, wlmod.C2, heads=[0, 5, 11], nrows=1500)
+
+
+def test_fused_wan13b_irregular(salad):
+    wl = wlmod.C3
+    sampled_fused_check(salad, wl, heads=[0, 7], nrows=1000, csr=wlmod.irregular_csr(wl))
+
+
+def test_fused_wan14b_90(salad):
+    sampled_fused_check(salad, wlmod.C4, heads=[0, 39], nrows=600)
+
+
+@pytest.mark.parametrize("wl", [wlmod.C5_80, wlmod.C5_90, wlmod.C5_95])
+def test_fused_cfg_pair_sparsity_sweep(salad, wl):
+    sampled_fused_check(salad, wl, heads=[3], nrows=600)
+
+
+def test_fused_cfg_pair_dense(salad):
+    sampled_fused_check(salad, wlmod.C5_DENSE, heads=[8], nrows=120)
