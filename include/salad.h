@@ -122,6 +122,18 @@ int salad_fused_fwd(const void* q, const void* k, const void* v, void* o,
                     float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
                     int32_t* d_status, void* stream);
 
+/*
+ * salad_set_profile_events -- optional instrumentation for benchmarks (no counterpart in
+ * the paper).  h_events is a HOST array of four cudaEvent_t handles (as void*), or NULL to
+ * switch the instrumentation off.  While set, every *_fwd call made by the calling host
+ * thread records
+ *     h_events[0], h_events[1]   around the linear-state kernels (Eq. 3 reductions), and
+ *     h_events[2], h_events[3]   around the attention kernel (Eq. 2 + apply + combine)
+ * on the call's stream; entries may individually be NULL.  The events stay owned by the
+ * caller.  The setting is per host thread and changes nothing else about the calls.
+ */
+int salad_set_profile_events(void* const* h_events);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,6 +21,12 @@ constexpr size_t kAlign = 256;
 constexpr int kPartialSlots = 512;     // upper bound on (batch*heads) x chunks partial states
 constexpr int kMaxMaskHeads = 256;
 
+thread_local cudaEvent_t g_profile_events[4] = {nullptr, nullptr, nullptr, nullptr};
+
+inline void record_profile(int idx, cudaStream_t st) {
+    if (g_profile_events[idx]) cudaEventRecord(g_profile_events[idx], st);
+}
+
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
@@ -139,11 +145,13 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.z_part = reinterpret_cast<float*>(ws + w.off_zp);
     sp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     sp.user_status = P.d_status;
+    record_profile(0, P.stream);
     salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     salad_linear_finalize_kernel<D><<<dim3((D * D + 255) / 256, BH), 256, 0, P.stream>>>(
         sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
         reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt));
+    record_profile(1, P.stream);
     return check_launch();
 }
 
@@ -172,8 +180,10 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.user_status = P.d_status;
     const int64_t grid = int64_t(fp.nPairs) * BH;
     if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
+    record_profile(2, P.stream);
     salad_fused_kernel<D><<<unsigned(grid), FusedCfg<D>::THREADS, FusedCfg<D>::SMEM_BYTES, P.stream>>>(
         mq, mk, mv, mo, ms, fp);
+    record_profile(3, P.stream);
     return check_launch();
 }
 
@@ -210,6 +220,12 @@ SALAD_EXPORT const char* salad_status_string(int status) {
         case SALAD_ERR_TIMEOUT: return "SALAD_ERR_TIMEOUT";
         default: return "SALAD_ERR_UNKNOWN";
     }
+}
+
+SALAD_EXPORT int salad_set_profile_events(void* const* h_events) {
+    for (int i = 0; i < 4; ++i)
+        g_profile_events[i] = h_events ? static_cast<cudaEvent_t>(h_events[i]) : nullptr;
+    return SALAD_OK;
 }
 
 SALAD_EXPORT size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk) {

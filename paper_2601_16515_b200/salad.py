@@ -25,7 +25,8 @@ SALAD_ERR_CUDA = -5
 SALAD_ERR_TIMEOUT = -6
 
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
-           "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd")
+           "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
+           "salad_set_profile_events")
 
 
 class SaladError(RuntimeError):
@@ -53,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_linear_attn_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [f32, p, sz, p, p]
     lib.salad_fused_fwd.restype = i32
     lib.salad_fused_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, p, sz, p, p]
+    lib.salad_set_profile_events.restype = i32
+    lib.salad_set_profile_events.argtypes = [p]
     return lib
 
 
@@ -112,6 +115,17 @@ def salad_mask_build(T: int, Hs: int, Ws: int, Bq: int, Bk: int,
         _check(_lib.salad_mask_build(T, Hs, Ws, Bq, Bk, Hm, h_win, _ptr(row_ptr), _ptr(col_idx),
                                      col_idx.numel(), ctypes.byref(nnz), _stream(stream)), "salad_mask_build")
     return row_ptr, col_idx[:nnz.value]
+
+
+def salad_set_profile_events(events=None):
+    """events: None, or four torch.cuda.Event(enable_timing=True) / None entries:
+    (state start, state stop, attention start, attention stop).  The events must have been
+    recorded once (or otherwise materialised) so that they own a CUDA handle."""
+    if events is None:
+        _check(_lib.salad_set_profile_events(None), "salad_set_profile_events")
+        return
+    arr = (ctypes.c_void_p * 4)(*[None if e is None else e.cuda_event for e in events])
+    _check(_lib.salad_set_profile_events(arr), "salad_set_profile_events")
 
 
 def _common(q, k, v, Bq, Bk, workspace):
