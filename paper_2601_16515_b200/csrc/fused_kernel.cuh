@@ -125,7 +125,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_init(smem_u32(&bars.o_final[i]), 1);
             for (int j = 0; j < 2; ++j) {
                 mbar_init(smem_u32(&bars.s_full[i][j]), 1);
-                mbar_init(smem_u32(&bars.p_ready[i][j]), 128);
+                mbar_init(smem_u32(&bars.p_ready[i][j]), 4);
             }
         }
         mbar_init(smem_u32(&bars.st_full), 1);
@@ -212,21 +212,25 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             int tq[2] = {0, 0};   // QK issued per tile
             int tp[2] = {0, 0};   // PV issued per tile
             int gk = 0, gv = 0;
+            // descriptor halves: the high word is one constant for every operand here
+            constexpr uint32_t HI = sdesc_hi_sw128(1024);
+            const uint32_t q_lo[2] = {sdesc_lo(s_base + C::OFF_Q, 16), sdesc_lo(s_base + C::OFF_Q + C::Q_BYTES, 16)};
+            const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
+            const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
             auto issue_qk = [&](int tag) -> bool {
                 const int s = gk % C::NK;
                 if (!mbar_wait(smem_u32(&bars.k_full[s]), (gk / C::NK) & 1, abortp)) return false;
                 tc_fence_after_sync();
-                const uint32_t kb = s_base + C::OFF_K + s * C::KV_BYTES;
+                const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     if (!(tag & (1 << i))) continue;
-                    const uint32_t qa = s_base + C::OFF_Q + i * C::Q_BYTES;
                     const uint32_t dcol = tmem + i * 256 + (tq[i] & 1) * 64;
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
-                        const uint64_t da = make_sdesc_sw128(qa + (k / 4) * C::Q_CHUNK + (k % 4) * 32, 16, 1024);
-                        const uint64_t db = make_sdesc_sw128(kb + (k / 4) * C::KV_CHUNK + (k % 4) * 32, 16, 1024);
-                        mma_ss(dcol, da, db, idesc_qk, k > 0);
+                        // k-th 16-channel slice: chunk k/4, 32 bytes per slice inside the 128-byte row
+                        mma_ss_lohi(dcol, q_lo[i] + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
                     }
                     tc_commit(smem_u32(&bars.s_full[i][tq[i] & 1]));
                     ++tq[i];
@@ -245,7 +249,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const int s = gv % C::NV;
                 ok = mbar_wait(smem_u32(&bars.v_full[s]), (gv / C::NV) & 1, abortp);
                 if (!ok) break;
-                const uint32_t vb = s_base + C::OFF_V + s * C::KV_BYTES;
+                const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     if (!(tag & (1 << i))) continue;
@@ -256,10 +260,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const uint32_t pcol = tmem + i * 256 + (t & 1) * 64;
                     const uint32_t ocol = tmem + i * 256 + 128;
 #pragma unroll
-                    for (int k = 0; k < C::BK / 16; ++k) {
-                        const uint64_t db = make_sdesc_sw128(vb + k * 2048, C::KV_CHUNK, 1024);
-                        mma_ts(ocol, pcol + k * 8, db, idesc_pv, (t > 0 || k > 0) ? 1u : 0u);
-                    }
+                    for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
+                        mma_ts_lohi(ocol, pcol + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
+                                    (t > 0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&bars.pv_done[i]));
                     ++tp[i];
                     if (tp[i] == le[i] - ls[i]) tc_commit(smem_u32(&bars.o_final[i]));
@@ -276,14 +279,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t qa = s_base + C::OFF_Q + i * C::Q_BYTES;
-                    const uint32_t sb = s_base + C::OFF_ST;
+                    const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST, 16);
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint64_t da = make_sdesc_sw128(qa + (k / 4) * C::Q_CHUNK + (k % 4) * 32, 16, 1024);
-                        const uint64_t db = make_sdesc_sw128(sb + (k / 4) * C::ST_CHUNK + (k % 4) * 32, 16, 1024);
-                        mma_ss(tmem + i * 256, da, db, idesc_lin, k > 0);
-                    }
+                    for (int k = 0; k < D / 16; ++k)
+                        mma_ss_lohi(tmem + i * 256, q_lo[i] + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                    st_lo + (((k / 4) * C::ST_CHUNK + (k % 4) * 32) >> 4), HI, idesc_lin, k > 0);
                     tc_commit(smem_u32(&bars.lin_done[i]));
                 }
             }
@@ -365,7 +365,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_st32(t_tile + buf * 64, pk);
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(smem_u32(&bars.p_ready[i][buf]));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i][buf]));   // one arrival per warp
         }
         if (ok && len > 0) {
             // pv_done cycles once per block and is only safe to test one phase back (as the

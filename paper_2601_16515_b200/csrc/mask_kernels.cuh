@@ -2,11 +2,11 @@
 // (Sec. 3 static sparse attention; Appendix A.1 token flattening, time slowest).
 //
 // Block pair (i, j) is kept iff some query token of block i and some key token of block j
-// lie within (wt, wh, ww) of each other on the T x Hs x Ws grid.  Instead of enumerating
-// token pairs, each query token's window is intersected with the key block run by run:
-// a key block is a contiguous range [k0, k1) of flat token ids, i.e. a few grid rows
-// (t', h') each contributing one contiguous run of w'; the window of a query token selects,
-// in each such row, the run [w - ww, w + ww].  Two integer interval tests per row decide.
+// lie within (wt, wh, ww) of each other on the T x Hs x Ws grid.  Token pairs are not
+// enumerated: a block is a contiguous range of flat token ids, i.e. a few grid rows (t, h)
+// each contributing one contiguous run of w.  For every (query row, key row) pair whose t and
+// h differ by at most wt and wh, two w-runs [wa, wb] and [ka, kb] hold a pair within ww iff
+// ka - wb <= ww and wa - kb <= ww.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -24,18 +24,20 @@ struct MaskWindows {
 };
 
 __device__ __forceinline__ bool block_pair_kept(const MaskGeom& g, int i, int j, int wt, int wh, int ww) {
-    const int q0 = i * g.Bq, q1 = min(g.N, q0 + g.Bq);
-    const int k0 = j * g.Bk, k1 = min(g.N, k0 + g.Bk);
-    const int krow0 = k0 / g.Ws, krow1 = (k1 - 1) / g.Ws;   // grid rows (t*Hs + h) the key block touches
-    for (int n = q0; n < q1; ++n) {
-        const int qrow = n / g.Ws, w = n - qrow * g.Ws;
-        const int t = qrow / g.Hs, h = qrow - t * g.Hs;
-        const int wlo = max(0, w - ww), whi = min(g.Ws - 1, w + ww);
-        for (int r = krow0; r <= krow1; ++r) {
-            const int t2 = r / g.Hs, h2 = r - t2 * g.Hs;
+    const int q0 = i * g.Bq, q1 = min(g.N, q0 + g.Bq) - 1;    // inclusive token ranges
+    const int k0 = j * g.Bk, k1 = min(g.N, k0 + g.Bk) - 1;
+    const int qrow0 = q0 / g.Ws, qrow1 = q1 / g.Ws;            // grid rows (t*Hs + h) touched
+    const int krow0 = k0 / g.Ws, krow1 = k1 / g.Ws;
+    for (int r = qrow0; r <= qrow1; ++r) {
+        const int t = r / g.Hs, h = r - t * g.Hs;
+        const int wa = (r == qrow0) ? q0 - r * g.Ws : 0;
+        const int wb = (r == qrow1) ? q1 - r * g.Ws : g.Ws - 1;
+        for (int r2 = krow0; r2 <= krow1; ++r2) {
+            const int t2 = r2 / g.Hs, h2 = r2 - t2 * g.Hs;
             if (abs(t2 - t) > wt || abs(h2 - h) > wh) continue;
-            const int lo = max(r * g.Ws + wlo, k0), hi = min(r * g.Ws + whi, k1 - 1);
-            if (lo <= hi) return true;
+            const int ka = (r2 == krow0) ? k0 - r2 * g.Ws : 0;
+            const int kb = (r2 == krow1) ? k1 - r2 * g.Ws : g.Ws - 1;
+            if (ka - wb <= ww && wa - kb <= ww) return true;
         }
     }
     return false;
