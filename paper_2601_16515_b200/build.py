@@ -25,6 +25,9 @@ def nvcc_command(out: str, verbose: bool = False):
            "-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
+    extra = os.environ.get("SALAD_NVCC_FLAGS")       # e.g. -DSALAD_TRACE for the cycle trace points
+    if extra:
+        cmd[1:1] = extra.split()
     return cmd
 
 

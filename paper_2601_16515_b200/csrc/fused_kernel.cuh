@@ -3,27 +3,39 @@
 //
 // One CTA owns two consecutive query blocks of one (batch, head): two 128-row MMA tiles.
 //   warp 0        TMA producer: Q tiles, linear-state tile, K/V tiles of the kept key blocks
-//   warp 1        tcgen05 MMA issuer (one thread); owns the TMEM allocation
+//   warp 1, 2     tcgen05 MMA issuers of tile 0 and tile 1 (one thread each); warp 1 owns TMEM
 //   warps 4-7     softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
 //   warps 8-11    the same for tile 1
 // The kept lists of the two query blocks are walked as one sorted merge, so a key block that
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
-// loaded.  S = Q K^T lands in TMEM (two 64-column buffers per tile, so the next block's
-// scores are computed while the current block's softmax runs); the softmax warpgroup reads
-// its row, keeps a running max in the log2 domain (rescaling the O accumulator only when the
-// max grows by more than 2^8), writes P = exp2(.) as bf16 over the S columns, and the MMA
-// warp accumulates O += P V with P read from TMEM.  After the last block the warpgroup applies
-// ReLU to its Q rows in shared memory, computes the linear denominator with plain FMAs, the
-// MMA warp multiplies ReLU(Q) with the bf16 linear state, and the epilogue writes
+// loaded.
+//
+// Both products read their A operand from tensor memory: a tcgen05.mma whose A comes from
+// shared memory costs ~110 cycles per 128xNx16 instruction on this part whatever N <= 128 is,
+// against ~60 with A in TMEM, so the Q tile is copied into TMEM once and S = Q K^T uses it
+// there; P = exp2(.) is written as bf16 over the S columns and O += P V reads it from TMEM.
+// Per tile the chain  S = Q K^T -> softmax -> O += P V  is serial (one S buffer); the two
+// tiles have their own issuing threads and run out of phase, so the tensor pipe works for
+// one tile while the other tile's warpgroup is in its softmax.
+// The softmax keeps a running max in the log2 domain and rescales the O accumulator only
+// when the max grows by more than 2^8.  After the last block the warpgroup applies ReLU to
+// its Q rows in shared memory, computes the linear denominator with plain FMAs, the issuing
+// thread multiplies ReLU(Q) with the bf16 linear state, and the epilogue writes
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
 //
-// TMEM columns (512 allocated): tile i uses [256 i, 256 i + 128) for the two S/P buffers
-// (reused for the linear numerator) and [256 i + 128, 256 i + 128 + D) for O.
+// TMEM columns (512 allocated), tile i at 256 i:  [0,64) S, first 32 reused for P;
+// [64,64+D/2) Q as bf16 pairs;  [128,128+D) O.  The linear numerator reuses [0,D).
 #pragma once
 #include "ptx.cuh"
 
 namespace salad {
+
+#ifdef SALAD_TRACE
+#define TRACE(role, step, k) do { if (blockIdx.x == 700 && (step) < 64) reinterpret_cast<long long*>(p.lse)[((role) * 64 + (step)) * 8 + (k)] = clock64(); } while (0)
+#else
+#define TRACE(role, step, k) do {} while (0)
+#endif
 
 enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
 
@@ -58,11 +70,13 @@ struct FusedCfg {
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
     static constexpr int THREADS = 384;
+    // TMEM columns within a tile's 256
+    static constexpr uint32_t COL_S = 0, COL_Q = 64, COL_O = 128;
 };
 
 struct FusedBarriers {
     uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2][2], p_ready[2][2], pv_done[2], lin_ready[2], lin_done[2], out_staged[2], o_final[2];
+    uint64_t q_tmem[2], s_full[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
 };
 
 // Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
@@ -118,22 +132,20 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.pv_done[i]), 1);
+            mbar_init(smem_u32(&bars.q_tmem[i]), 4);
+            mbar_init(smem_u32(&bars.s_full[i]), 1);
+            mbar_init(smem_u32(&bars.p_ready[i]), 4);
+            mbar_init(smem_u32(&bars.o_final[i]), 1);
             mbar_init(smem_u32(&bars.lin_ready[i]), 128);
             mbar_init(smem_u32(&bars.lin_done[i]), 1);
             mbar_init(smem_u32(&bars.out_staged[i]), 128);
-            mbar_init(smem_u32(&bars.o_final[i]), 1);
-            for (int j = 0; j < 2; ++j) {
-                mbar_init(smem_u32(&bars.s_full[i][j]), 1);
-                mbar_init(smem_u32(&bars.p_ready[i][j]), 4);
-            }
         }
         mbar_init(smem_u32(&bars.st_full), 1);
         for (int s = 0; s < 4; ++s) {
             mbar_init(smem_u32(&bars.k_full[s]), 1);
-            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 2);     // released by both issuing threads
             mbar_init(smem_u32(&bars.v_full[s]), 1);
-            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 2);
         }
         fence_mbar_init();
     }
@@ -197,92 +209,79 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (ok && prev_col >= 0)
                 ok = load_tile(&map_v, C::OFF_V, bars.v_full, bars.v_empty, gv++, C::NV, prev_col);
         }
-    } else if (warp == 1) {
-        // ============================================================== MMA issuer
+    } else if (warp == 1 || warp == 2) {
+        // ============================================================== MMA issuer of tile i
+        // Walks every entry of the merged list in order: entries of its own tile are multiplied,
+        // the others are only released (each K/V stage needs both issuers' release), always
+        // after waiting for the stage to be full so that a release can never run a phase ahead.
         if (lane == 0) {
+            const int i = warp - 1;
             const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
             const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
             const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
-            bool ok = true;
-            for (int i = 0; i < 2 && ok; ++i)
-                if (qb[i] < p.nQb && (le[i] > ls[i]))
-                    ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
-            tc_fence_after_sync();
-            MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
-            int tq[2] = {0, 0};   // QK issued per tile
-            int tp[2] = {0, 0};   // PV issued per tile
-            int gk = 0, gv = 0;
-            // descriptor halves: the high word is one constant for every operand here
-            constexpr uint32_t HI = sdesc_hi_sw128(1024);
-            const uint32_t q_lo[2] = {sdesc_lo(s_base + C::OFF_Q, 16), sdesc_lo(s_base + C::OFF_Q + C::Q_BYTES, 16)};
+            constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
             const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
             const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
-            auto issue_qk = [&](int tag) -> bool {
-                const int s = gk % C::NK;
-                if (!mbar_wait(smem_u32(&bars.k_full[s]), (gk / C::NK) & 1, abortp)) return false;
+            const uint32_t t_tile = tmem + i * 256;
+            const int len = le[i] - ls[i];
+            bool ok = true;
+            if (len > 0) {
+                ok = mbar_wait(smem_u32(&bars.q_tmem[i]), 0, abortp);
                 tc_fence_after_sync();
-                const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    if (!(tag & (1 << i))) continue;
-                    const uint32_t dcol = tmem + i * 256 + (tq[i] & 1) * 64;
-#pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        // k-th 16-channel slice: chunk k/4, 32 bytes per slice inside the 128-byte row
-                        mma_ss_lohi(dcol, q_lo[i] + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
-                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                    }
-                    tc_commit(smem_u32(&bars.s_full[i][tq[i] & 1]));
-                    ++tq[i];
-                }
-                tc_commit(smem_u32(&bars.k_empty[s]));
-                ++gk;
-                return true;
-            };
-            int col, tag, ncol, ntag;
-            bool have = ok && wk.next(col, tag);
-            if (have) ok = issue_qk(tag);
-            while (ok && have) {
-                const bool have_next = wk.next(ncol, ntag);
-                if (have_next) ok = issue_qk(ntag);
+            }
+            MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
+            int col, tag, g = 0, t = 0;
+            while (ok && wk.next(col, tag)) {
+                const bool mine = (tag >> i) & 1;
+                const int sk = g % C::NK, sv = g % C::NV;
+                const uint32_t par = (g / C::NK) & 1;      // NK == NV
+                TRACE(2 + i, g, 0);
+                ok = mbar_wait(smem_u32(&bars.k_full[sk]), par, abortp);
                 if (!ok) break;
-                const int s = gv % C::NV;
-                ok = mbar_wait(smem_u32(&bars.v_full[s]), (gv / C::NV) & 1, abortp);
-                if (!ok) break;
-                const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    if (!(tag & (1 << i))) continue;
-                    const int t = tp[i];
-                    ok = mbar_wait(smem_u32(&bars.p_ready[i][t & 1]), (t >> 1) & 1, abortp);
-                    if (!ok) break;
+                if (mine) {
                     tc_fence_after_sync();
-                    const uint32_t pcol = tmem + i * 256 + (t & 1) * 64;
-                    const uint32_t ocol = tmem + i * 256 + 128;
+                    const uint32_t kb_lo = k_lo0 + sk * (C::KV_BYTES >> 4);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k)   // 16 channels: 8 TMEM columns of Q, 32 bytes of each K row
+                        mma_ts_lohi(t_tile + C::COL_S, t_tile + C::COL_Q + k * 8,
+                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
+                    tc_commit(smem_u32(&bars.s_full[i]));
+                    tc_commit(smem_u32(&bars.k_empty[sk]));
+                } else {
+                    mbar_arrive(smem_u32(&bars.k_empty[sk]));
+                }
+                TRACE(2 + i, g, 1);
+                ok = mbar_wait(smem_u32(&bars.v_full[sv]), par, abortp);
+                if (!ok) break;
+                if (mine) {
+                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), t & 1, abortp);
+                    if (!ok) break;
+                    TRACE(2 + i, g, 2);
+                    tc_fence_after_sync();
+                    const uint32_t vb_lo = v_lo0 + sv * (C::KV_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
-                        mma_ts_lohi(ocol, pcol + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
-                                    (t > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&bars.pv_done[i]));
-                    ++tp[i];
-                    if (tp[i] == le[i] - ls[i]) tc_commit(smem_u32(&bars.o_final[i]));
+                        mma_ts_lohi(t_tile + C::COL_O, t_tile + C::COL_S + k * 8, vb_lo + ((k * 2048) >> 4), HI,
+                                    idesc_pv, (t > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&bars.v_empty[sv]));
+                    ++t;
+                    if (t == len) tc_commit(smem_u32(&bars.o_final[i]));
+                    TRACE(2 + i, g, 3);
+                } else {
+                    mbar_arrive(smem_u32(&bars.v_empty[sv]));
                 }
-                if (!ok) break;
-                tc_commit(smem_u32(&bars.v_empty[s]));
-                ++gv;
-                have = have_next; col = ncol; tag = ntag;
+                ++g;
             }
-            if (ok && linear) {
+            if (ok && linear && qb[i] < p.nQb) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
-                for (int i = 0; i < 2 && ok; ++i) {
-                    if (qb[i] >= p.nQb) continue;
-                    ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
-                    if (!ok) break;
+                if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
+                if (ok) {
                     tc_fence_after_sync();
+                    const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
                     const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST, 16);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k)
-                        mma_ss_lohi(tmem + i * 256, q_lo[i] + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                        mma_ss_lohi(t_tile, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
                                     st_lo + (((k / 4) * C::ST_CHUNK + (k % 4) * 32) >> 4), HI, idesc_lin, k > 0);
                     tc_commit(smem_u32(&bars.lin_done[i]));
                 }
@@ -296,6 +295,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t t_tile = tmem + i * 256 + lane_addr;
         const bool tile_valid = qb[i] < p.nQb;
         const int len = le[i] - ls[i];
+        uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
         // every lane of a warp must take the same path around the warp-collective tcgen05
@@ -304,15 +304,39 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             return __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, abortp));
         };
 
+        if (len > 0) {
+            // this thread's Q row: shared memory (128-byte swizzle) -> TMEM, bf16 pairs
+            ok = wait_uniform(&bars.q_full[i], 0);
+            if (ok) {
+#pragma unroll
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int c16 = 0; c16 < 8; ++c16) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
+                                                                        ((c16 ^ (row & 7)) << 4));
+                        w[c16 * 4 + 0] = v.x; w[c16 * 4 + 1] = v.y; w[c16 * 4 + 2] = v.z; w[c16 * 4 + 3] = v.w;
+                    }
+                    tmem_st32(t_tile + C::COL_Q + ch * 32, w);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.q_tmem[i]));
+            }
+        }
+
         for (int t = 0; t < len && ok; ++t) {
-            const int buf = t & 1;
-            ok = wait_uniform(&bars.s_full[i][buf], (t >> 1) & 1);
+            if (row == 0) TRACE(i, t, 0);
+            ok = wait_uniform(&bars.s_full[i], t & 1);
             if (!ok) break;
+            if (row == 0) TRACE(i, t, 1);
             tc_fence_after_sync();
             uint32_t xr[64];
-            tmem_ld32(t_tile + buf * 64, xr);
-            tmem_ld32(t_tile + buf * 64 + 32, xr + 32);
+            tmem_ld32(t_tile + C::COL_S, xr);
+            tmem_ld32(t_tile + C::COL_S + 32, xr + 32);
             tmem_wait_ld();
+            if (row == 0) TRACE(i, t, 2);
             float* x = reinterpret_cast<float*>(xr);
             const int col = __ldg(p.col_idx + ls[i] + t);
             const int valid = p.N - col * C::BK;          // keys of this block that exist
@@ -320,22 +344,24 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
             }
-            float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
+            float mx[8];
 #pragma unroll
-            for (int c = 4; c < C::BK; c += 4) {
-                mx0 = fmaxf(mx0, x[c]); mx1 = fmaxf(mx1, x[c + 1]);
-                mx2 = fmaxf(mx2, x[c + 2]); mx3 = fmaxf(mx3, x[c + 3]);
+            for (int c = 0; c < 8; ++c) mx[c] = x[c];
+#pragma unroll
+            for (int c = 8; c < C::BK; c += 8) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
             }
-            const float msc = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+            const float msc = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                    fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
             if (t == 0) {
                 m_run = msc;
             } else {
                 const bool need = msc > m_run + 8.0f;
                 if (__any_sync(0xffffffffu, need)) {
-                    // bring the accumulator of this warp's rows to the new running max
-                    ok = wait_uniform(&bars.pv_done[i], (t - 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
+                    // bring the accumulator of this warp's rows to the new running max.  The
+                    // previous P V product is complete: it was issued before this block's Q K^T
+                    // by the same thread, and that product's completion was just observed.
                     const float m_new = fmaxf(m_run, msc);
                     const float alpha = ex2_approx(m_run - m_new);
                     l_run *= alpha;
@@ -343,15 +369,16 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                     for (int cc = 0; cc < D / 32; ++cc) {
                         uint32_t orr[32];
-                        tmem_ld32(t_tile + 128 + cc * 32, orr);
+                        tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
                         tmem_wait_ld();
 #pragma unroll
                         for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        tmem_st32(t_tile + 128 + cc * 32, orr);
+                        tmem_st32(t_tile + C::COL_O + cc * 32, orr);
                     }
                     tmem_wait_st();
                 }
             }
+            if (row == 0) TRACE(i, t, 3);
             uint32_t pk[32];
             float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -362,15 +389,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 pk[c >> 1] = pack_bf16x2(p0, p1);
             }
             l_run += s0 + s1;
-            tmem_st32(t_tile + buf * 64, pk);
+            if (row == 0) TRACE(i, t, 4);
+            tmem_st32(t_tile + C::COL_S, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i][buf]));   // one arrival per warp
+            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i]));   // one arrival per warp
+            if (row == 0) TRACE(i, t, 5);
         }
         if (ok && len > 0) {
-            // pv_done cycles once per block and is only safe to test one phase back (as the
-            // rescale does); the end of the last P V product has a barrier of its own
             ok = wait_uniform(&bars.o_final[i], 0);
             tc_fence_after_sync();
         }
@@ -382,7 +409,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (ok) {
                 const float* zrow = p.z + size_t(bh) * D;
                 float den = 0.f;
-                uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
 #pragma unroll
                 for (int ch = 0; ch < C::CH; ++ch) {
 #pragma unroll
@@ -416,11 +442,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (ok && tile_valid) {
             // O = O_acc / l + lin_coef * num, rounded once to bf16, staged in the Q tile
             const float inv_l = (len > 0) ? 1.0f / l_run : 0.f;
-            uint8_t* stage = smem + C::OFF_Q + i * C::Q_BYTES;
 #pragma unroll
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t orr[32], nr[32];
-                if (len > 0) tmem_ld32(t_tile + 128 + cc * 32, orr);
+                if (len > 0) tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
                 if (linear) tmem_ld32(t_tile + cc * 32, nr);
                 tmem_wait_ld();
 #pragma unroll
@@ -439,7 +464,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                     const int col16 = (cc * 32 + c8 * 8) / 8;      // 16-byte chunk index within the row
                     const int ch = col16 / 8, c16 = col16 % 8;
-                    *reinterpret_cast<uint4*>(stage + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
+                    *reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
@@ -452,12 +477,14 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tma_store_commit();
                 tma_store_wait_all();
             }
+#ifndef SALAD_TRACE
             if (p.lse != nullptr) {
                 const int n = qb[i] * p.Bq + row;
                 if (row < p.Bq && n < p.N)
                     p.lse[size_t(bh) * p.N + n] =
                         (len > 0) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
             }
+#endif
         }
     }
     }  // abort_flag == 0
