@@ -230,8 +230,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tc_fence_after_sync();
             }
             MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
-            int col, tag, g = 0, t = 0;
-            while (ok && wk.next(col, tag)) {
+            int col, tag, ncol = 0, ntag = 0, g = 0, t = 0;
+            bool have = ok && wk.next(col, tag);
+            while (ok && have) {
                 const bool mine = (tag >> i) & 1;
                 const int sk = g % C::NK, sv = g % C::NV;
                 const uint32_t par = (g / C::NK) & 1;      // NK == NV
@@ -251,6 +252,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     mbar_arrive(smem_u32(&bars.k_empty[sk]));
                 }
                 TRACE(2 + i, g, 1);
+                const bool have_next = wk.next(ncol, ntag);     // list reads overlap the waits below
                 ok = mbar_wait(smem_u32(&bars.v_full[sv]), par, abortp);
                 if (!ok) break;
                 if (mine) {
@@ -271,6 +273,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     mbar_arrive(smem_u32(&bars.v_empty[sv]));
                 }
                 ++g;
+                have = have_next; col = ncol; tag = ntag;
             }
             if (ok && linear && qb[i] < p.nQb) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
@@ -326,8 +329,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
         }
 
+        const bool ragged_keys = (p.N % C::BK) != 0;
         for (int t = 0; t < len && ok; ++t) {
             if (row == 0) TRACE(i, t, 0);
+            // only the last key block can be short; its id is needed only then
+            const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
             ok = wait_uniform(&bars.s_full[i], t & 1);
             if (!ok) break;
             if (row == 0) TRACE(i, t, 1);
@@ -338,27 +344,45 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_wait_ld();
             if (row == 0) TRACE(i, t, 2);
             float* x = reinterpret_cast<float*>(xr);
-            const int col = __ldg(p.col_idx + ls[i] + t);
             const int valid = p.N - col * C::BK;          // keys of this block that exist
-            if (valid < C::BK) {
+            if (ragged_keys && valid < C::BK) {
 #pragma unroll
                 for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
             }
-            float mx[8];
+            auto row_max_scaled = [&]() -> float {
+                float mx[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) mx[c] = x[c];
+                for (int c = 0; c < 8; ++c) mx[c] = x[c];
 #pragma unroll
-            for (int c = 8; c < C::BK; c += 8) {
+                for (int c = 8; c < C::BK; c += 8) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
-            }
-            const float msc = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                    fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+                    for (int e = 0; e < 8; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
+                }
+                return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                             fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+            };
+            uint32_t pk[32];
+            auto exp_row = [&](float m_ref) -> float {    // P = exp2(x * scale - m_ref), packed bf16; returns the row sum
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int c = 0; c < C::BK; c += 2) {
+                    const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
+                    const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
+                    s0 += p0; s1 += p1;
+                    pk[c >> 1] = pack_bf16x2(p0, p1);
+                }
+                return s0 + s1;
+            };
+            float row_sum;
             if (t == 0) {
-                m_run = msc;
+                m_run = row_max_scaled();
+                row_sum = exp_row(m_run);
             } else {
-                const bool need = msc > m_run + 8.0f;
-                if (__any_sync(0xffffffffu, need)) {
+                // exponentials against the running max of the earlier blocks start at once; the
+                // max of this block is found alongside and only matters if it is 2^8 larger
+                row_sum = exp_row(m_run);
+                const float msc = row_max_scaled();
+                if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
                     // bring the accumulator of this warp's rows to the new running max.  The
                     // previous P V product is complete: it was issued before this block's Q K^T
                     // by the same thread, and that product's completion was just observed.
@@ -376,19 +400,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         tmem_st32(t_tile + C::COL_O + cc * 32, orr);
                     }
                     tmem_wait_st();
+                    row_sum = exp_row(m_run);
                 }
             }
-            if (row == 0) TRACE(i, t, 3);
-            uint32_t pk[32];
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int c = 0; c < C::BK; c += 2) {
-                const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_run));
-                const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_run));
-                s0 += p0; s1 += p1;
-                pk[c >> 1] = pack_bf16x2(p0, p1);
-            }
-            l_run += s0 + s1;
+            l_run += row_sum;
             if (row == 0) TRACE(i, t, 4);
             tmem_st32(t_tile + C::COL_S, pk);
             tmem_wait_st();
