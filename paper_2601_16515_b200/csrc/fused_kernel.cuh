@@ -4,8 +4,10 @@
 // One CTA owns two consecutive query blocks of one (batch, head): two 128-row MMA tiles.
 //   warp 0        TMA producer: Q tiles, linear-state tile, K/V tiles of the kept key blocks
 //   warp 1, 2     tcgen05 MMA issuers of tile 0 and tile 1 (one thread each); warp 1 owns TMEM
-//   warps 4-7     softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
-//   warps 8-11    the same for tile 1
+//   warps 4-11    softmax + epilogue of tile 0: two warpgroups, thread = (query row, half of the
+//                 64 key columns); the two threads of a row exchange their block max through
+//                 shared memory and a two-warp mbarrier
+//   warps 12-19   the same for tile 1
 // The kept lists of the two query blocks are walked as one sorted merge, so a key block that
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
 // loaded.
@@ -63,13 +65,15 @@ struct FusedCfg {
     static constexpr int KV_BYTES = CH * KV_CHUNK;  // one K or V tile
     static constexpr int ST_CHUNK = D * 128;
     static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]
-    static constexpr int NK = 4, NV = 4;
+    static constexpr int NK = 4, NV = 3;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_ST = 2 * Q_BYTES;
     static constexpr int OFF_K = OFF_ST + ST_BYTES;
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
-    static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
-    static constexpr int THREADS = 384;
+    static constexpr int OFF_X = OFF_V + NV * KV_BYTES;               // row exchange between column halves
+    static constexpr int X_BYTES = 2 * 2 * 4 * 128 * 4;              // [tile][half][slot][row] floats
+    static constexpr int SMEM_BYTES = OFF_X + X_BYTES + 1024;         // + alignment slack
+    static constexpr int THREADS = 640;
     // TMEM columns within a tile's 256
     static constexpr uint32_t COL_S = 0, COL_Q = 64, COL_O = 128;
 };
@@ -77,6 +81,7 @@ struct FusedCfg {
 struct FusedBarriers {
     uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
     uint64_t q_tmem[2], s_full[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
+    uint64_t pair[2][4];   // the two warps that share a 32-row TMEM lane quarter of a tile
 };
 
 // Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
@@ -95,7 +100,7 @@ struct MergeWalk {
 };
 
 template <int D>
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(640, 1)
 salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                    const __grid_constant__ CUtensorMap map_st, const FusedParams p)
@@ -132,13 +137,14 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.q_tmem[i]), 4);
+            mbar_init(smem_u32(&bars.q_tmem[i]), 8);        // one arrival per softmax warp
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.p_ready[i]), 4);
+            mbar_init(smem_u32(&bars.p_ready[i]), 8);
             mbar_init(smem_u32(&bars.o_final[i]), 1);
-            mbar_init(smem_u32(&bars.lin_ready[i]), 128);
+            mbar_init(smem_u32(&bars.lin_ready[i]), 8);
             mbar_init(smem_u32(&bars.lin_done[i]), 1);
-            mbar_init(smem_u32(&bars.out_staged[i]), 128);
+            mbar_init(smem_u32(&bars.out_staged[i]), 8);
+            for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&bars.pair[i][qd]), 2);
         }
         mbar_init(smem_u32(&bars.st_full), 1);
         for (int s = 0; s < 4; ++s) {
@@ -235,7 +241,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             while (ok && have) {
                 const bool mine = (tag >> i) & 1;
                 const int sk = g % C::NK, sv = g % C::NV;
-                const uint32_t par = (g / C::NK) & 1;      // NK == NV
+                const uint32_t par = (g / C::NK) & 1, par_v = (g / C::NV) & 1;
                 TRACE(2 + i, g, 0);
                 ok = mbar_wait(smem_u32(&bars.k_full[sk]), par, abortp);
                 if (!ok) break;
@@ -253,7 +259,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 TRACE(2 + i, g, 1);
                 const bool have_next = wk.next(ncol, ntag);     // list reads overlap the waits below
-                ok = mbar_wait(smem_u32(&bars.v_full[sv]), par, abortp);
+                ok = mbar_wait(smem_u32(&bars.v_full[sv]), par_v, abortp);
                 if (!ok) break;
                 if (mine) {
                     ok = mbar_wait(smem_u32(&bars.p_ready[i]), t & 1, abortp);
@@ -292,80 +298,91 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp >= 4) {
         // ============================================================== softmax + epilogue
-        const int i = (warp - 4) >> 2;            // tile
-        const int row = tid - 128 - 128 * i;      // query row within the tile = TMEM lane
-        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t t_tile = tmem + i * 256 + lane_addr;
+        const int sw = warp - 4;
+        const int i = sw >> 3;                    // tile
+        const int hf = (sw >> 2) & 1;             // which half of the key columns / output channels
+        const int quarter = warp & 3;             // TMEM lane quarter this warp may access
+        const int row = quarter * 32 + lane;      // query row within the tile = TMEM lane
+        const uint32_t t_tile = tmem + i * 256 + (uint32_t(quarter * 32) << 16);
         const bool tile_valid = qb[i] < p.nQb;
         const int len = le[i] - ls[i];
         uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
-        float m_run = -INFINITY, l_run = 0.f;
+        float* xch = reinterpret_cast<float*>(smem + C::OFF_X);        // [tile][half][slot][row]
+        float* x_mine = xch + ((i * 2 + hf) * 4) * 128 + row;
+        float* x_other = xch + ((i * 2 + (hf ^ 1)) * 4) * 128 + row;
+        uint64_t* pair_bar = &bars.pair[i][quarter];
+        constexpr int HD = D / 2;                 // output channels per thread
+        float m_run = -INFINITY, l_part = 0.f;
         bool ok = true;
         // every lane of a warp must take the same path around the warp-collective tcgen05
         // loads/stores, so the outcome of a bounded wait is made warp-uniform
         auto wait_uniform = [&](uint64_t* bar, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, abortp));
         };
+        auto warp_arrive = [&](uint64_t* bar) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(bar));
+        };
 
         if (len > 0) {
-            // this thread's Q row: shared memory (128-byte swizzle) -> TMEM, bf16 pairs
+            // this thread's half of its Q row: shared memory (128-byte swizzle) -> TMEM, bf16 pairs
             ok = wait_uniform(&bars.q_full[i], 0);
             if (ok) {
 #pragma unroll
-                for (int ch = 0; ch < C::CH; ++ch) {
-                    uint32_t w[32];
+                for (int part = 0; part < HD / 32; ++part) {      // 16 TMEM columns = 32 channels at a time
+                    uint32_t w[16];
 #pragma unroll
-                    for (int c16 = 0; c16 < 8; ++c16) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
-                                                                        ((c16 ^ (row & 7)) << 4));
-                        w[c16 * 4 + 0] = v.x; w[c16 * 4 + 1] = v.y; w[c16 * 4 + 2] = v.z; w[c16 * 4 + 3] = v.w;
+                    for (int j = 0; j < 4; ++j) {
+                        const int c16g = hf * (HD / 8) + part * 4 + j;    // 16-byte chunk index within the row
+                        const uint4 v = *reinterpret_cast<const uint4*>(qtile + (c16g / 8) * C::Q_CHUNK + row * 128 +
+                                                                        (((c16g % 8) ^ (row & 7)) << 4));
+                        w[j * 4 + 0] = v.x; w[j * 4 + 1] = v.y; w[j * 4 + 2] = v.z; w[j * 4 + 3] = v.w;
                     }
-                    tmem_st32(t_tile + C::COL_Q + ch * 32, w);
+                    tmem_st16(t_tile + C::COL_Q + hf * (HD / 2) + part * 16, w);
                 }
                 tmem_wait_st();
                 tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.q_tmem[i]));
+                warp_arrive(&bars.q_tmem[i]);
             }
         }
 
         const bool ragged_keys = (p.N % C::BK) != 0;
         for (int t = 0; t < len && ok; ++t) {
-            if (row == 0) TRACE(i, t, 0);
+            if (row == 0 && hf == 0) TRACE(i, t, 0);
             // only the last key block can be short; its id is needed only then
             const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
             ok = wait_uniform(&bars.s_full[i], t & 1);
             if (!ok) break;
-            if (row == 0) TRACE(i, t, 1);
+            if (row == 0 && hf == 0) TRACE(i, t, 1);
             tc_fence_after_sync();
-            uint32_t xr[64];
-            tmem_ld32(t_tile + C::COL_S, xr);
-            tmem_ld32(t_tile + C::COL_S + 32, xr + 32);
+            uint32_t xr[32];
+            tmem_ld32(t_tile + C::COL_S + hf * 32, xr);
             tmem_wait_ld();
-            if (row == 0) TRACE(i, t, 2);
+            if (row == 0 && hf == 0) TRACE(i, t, 2);
             float* x = reinterpret_cast<float*>(xr);
-            const int valid = p.N - col * C::BK;          // keys of this block that exist
-            if (ragged_keys && valid < C::BK) {
+            const int valid = p.N - col * C::BK - hf * 32;     // keys of this half that exist
+            if (ragged_keys && valid < 32) {
 #pragma unroll
-                for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
+                for (int c = 0; c < 32; ++c) if (c >= valid) x[c] = -INFINITY;
             }
-            auto row_max_scaled = [&]() -> float {
-                float mx[8];
+            // max of this half of the row; published to the other half's thread
+            float mx[4];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) mx[c] = x[c];
+            for (int c = 0; c < 4; ++c) mx[c] = x[c];
 #pragma unroll
-                for (int c = 8; c < C::BK; c += 8) {
+            for (int c = 4; c < 32; c += 4) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
-                }
-                return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                             fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
-            };
-            uint32_t pk[32];
-            auto exp_row = [&](float m_ref) -> float {    // P = exp2(x * scale - m_ref), packed bf16; returns the row sum
+                for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
+            }
+            const float lm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            x_mine[(t & 1) * 128] = lm;
+            warp_arrive(pair_bar);          // also tells the partner that this warp has read its S columns
+
+            uint32_t pk[16];
+            auto exp_half = [&](float m_ref) -> float {   // P = exp2(x * scale - m_ref) as bf16 pairs; returns the sum
                 float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                for (int c = 0; c < C::BK; c += 2) {
+                for (int c = 0; c < 32; c += 2) {
                     const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
                     const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
                     s0 += p0; s1 += p1;
@@ -373,98 +390,112 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 return s0 + s1;
             };
-            float row_sum;
+            float row_sum = 0.f;
+            // exponentials against the running max of the earlier blocks start at once; the max
+            // of this block only matters if it is more than 2^8 larger
+            if (row == 0 && hf == 0) TRACE(i, t, 3);
+            if (t > 0) row_sum = exp_half(m_run);
+            if (row == 0 && hf == 0) TRACE(i, t, 6);
+            ok = wait_uniform(pair_bar, t & 1);
+            if (!ok) break;
+            if (row == 0 && hf == 0) TRACE(i, t, 7);
+            const float msc = fmaxf(lm, x_other[(t & 1) * 128]) * p.scale_log2;   // same value in both halves
             if (t == 0) {
-                m_run = row_max_scaled();
-                row_sum = exp_row(m_run);
-            } else {
-                // exponentials against the running max of the earlier blocks start at once; the
-                // max of this block is found alongside and only matters if it is 2^8 larger
-                row_sum = exp_row(m_run);
-                const float msc = row_max_scaled();
-                if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
-                    // bring the accumulator of this warp's rows to the new running max.  The
-                    // previous P V product is complete: it was issued before this block's Q K^T
-                    // by the same thread, and that product's completion was just observed.
-                    const float m_new = fmaxf(m_run, msc);
-                    const float alpha = ex2_approx(m_run - m_new);
-                    l_run *= alpha;
-                    m_run = m_new;
+                m_run = msc;
+                row_sum = exp_half(m_run);
+            } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
+                // bring this thread's half of the accumulator to the new running max.  The previous
+                // P V product is complete: it was issued before this block's Q K^T by the same
+                // thread, and that product's completion was just observed.
+                const float m_new = fmaxf(m_run, msc);
+                const float alpha = ex2_approx(m_run - m_new);
+                l_part *= alpha;
+                m_run = m_new;
 #pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t orr[32];
-                        tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
-                        tmem_wait_ld();
+                for (int cc = 0; cc < HD / 16; ++cc) {
+                    uint32_t orr[16];
+                    tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        tmem_st32(t_tile + C::COL_O + cc * 32, orr);
-                    }
-                    tmem_wait_st();
-                    row_sum = exp_row(m_run);
+                    for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                    tmem_st16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
                 }
+                tmem_wait_st();
+                row_sum = exp_half(m_run);
             }
-            l_run += row_sum;
-            if (row == 0) TRACE(i, t, 4);
-            tmem_st32(t_tile + C::COL_S, pk);
+            l_part += row_sum;
+            if (row == 0 && hf == 0) TRACE(i, t, 4);
+            // P over the S columns (the partner has read its S values: it arrived on pair_bar)
+            tmem_st16(t_tile + C::COL_S + hf * 16, pk);
             tmem_wait_st();
             tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i]));   // one arrival per warp
-            if (row == 0) TRACE(i, t, 5);
+            warp_arrive(&bars.p_ready[i]);
+            if (row == 0 && hf == 0) TRACE(i, t, 5);
         }
         if (ok && len > 0) {
             ok = wait_uniform(&bars.o_final[i], 0);
             tc_fence_after_sync();
         }
 
-        float lin_coef = 0.f;
+        // row sum and linear denominator: add the two halves
+        float den_part = 0.f;
         if (ok && tile_valid && linear) {
-            // ReLU of this thread's Q row in place, and the denominator ReLU(Q_n) . Z
+            // ReLU of this thread's half of its Q row, in place, and its share of ReLU(Q_n) . Z
             ok = wait_uniform(&bars.q_full[i], 0);
             if (ok) {
                 const float* zrow = p.z + size_t(bh) * D;
-                float den = 0.f;
 #pragma unroll
-                for (int ch = 0; ch < C::CH; ++ch) {
+                for (int j = 0; j < HD / 8; ++j) {
+                    const int c16g = hf * (HD / 8) + j;
+                    uint4* ptr = reinterpret_cast<uint4*>(qtile + (c16g / 8) * C::Q_CHUNK + row * 128 +
+                                                          (((c16g % 8) ^ (row & 7)) << 4));
+                    uint4 v = *ptr;
+                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
 #pragma unroll
-                    for (int c16 = 0; c16 < 8; ++c16) {
-                        uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
-                                                              ((c16 ^ (row & 7)) << 4));
-                        uint4 v = *ptr;
-                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
-                            const float2 f = __bfloat1622float2(hv[e]);
-                            const int a = ch * 64 + c16 * 8 + e * 2;
-                            den = fmaf(f.x, __ldg(zrow + a), den);
-                            den = fmaf(f.y, __ldg(zrow + a + 1), den);
-                        }
-                        *ptr = v;
+                    for (int e = 0; e < 4; ++e) {
+                        hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
+                        const float2 f = __bfloat1622float2(hv[e]);
+                        const int a = c16g * 8 + e * 2;
+                        den_part = fmaf(f.x, __ldg(zrow + a), den_part);
+                        den_part = fmaf(f.y, __ldg(zrow + a + 1), den_part);
                     }
+                    *ptr = v;
                 }
-                float c_scale = 1.f;
-                if (p.static_scale) c_scale *= __ldg(p.static_scale + h);
-                if (p.dyn_scale) c_scale *= __ldg(p.dyn_scale + b);
-                lin_coef = c_scale / (den + p.eps);
                 fence_proxy_async_smem();
-                mbar_arrive(smem_u32(&bars.lin_ready[i]));
-                ok = wait_uniform(&bars.lin_done[i], 0);
-                tc_fence_after_sync();
             }
+        }
+        float l_run = l_part, den = den_part;
+        if (ok && tile_valid) {
+            x_mine[2 * 128] = l_part;
+            x_mine[3 * 128] = den_part;
+            warp_arrive(pair_bar);
+            ok = wait_uniform(pair_bar, len & 1);
+            if (ok) { l_run += x_other[2 * 128]; den += x_other[3 * 128]; }
+        }
+
+        float lin_coef = 0.f;
+        if (ok && tile_valid && linear) {
+            float c_scale = 1.f;
+            if (p.static_scale) c_scale *= __ldg(p.static_scale + h);
+            if (p.dyn_scale) c_scale *= __ldg(p.dyn_scale + b);
+            lin_coef = c_scale / (den + p.eps);
+            warp_arrive(&bars.lin_ready[i]);       // ReLU(Q) is in shared memory (fenced above)
+            ok = wait_uniform(&bars.lin_done[i], 0);
+            tc_fence_after_sync();
         }
 
         if (ok && tile_valid) {
-            // O = O_acc / l + lin_coef * num, rounded once to bf16, staged in the Q tile
+            // O = O_acc / l + lin_coef * num for this thread's channels, rounded once to bf16,
+            // staged in the Q tile (128-byte swizzle) for the TMA store
             const float inv_l = (len > 0) ? 1.0f / l_run : 0.f;
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
-                uint32_t orr[32], nr[32];
-                if (len > 0) tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
-                if (linear) tmem_ld32(t_tile + cc * 32, nr);
+            for (int cc = 0; cc < HD / 16; ++cc) {
+                uint32_t orr[16], nr[16];
+                if (len > 0) tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                if (linear) tmem_ld16(t_tile + hf * HD + cc * 16, nr);
                 tmem_wait_ld();
 #pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
+                for (int c8 = 0; c8 < 2; ++c8) {
                     uint32_t w[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -477,15 +508,14 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                         w[e] = pack_bf16x2(o0, o1);
                     }
-                    const int col16 = (cc * 32 + c8 * 8) / 8;      // 16-byte chunk index within the row
-                    const int ch = col16 / 8, c16 = col16 % 8;
-                    *reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
-                        make_uint4(w[0], w[1], w[2], w[3]);
+                    const int c16g = (hf * HD + cc * 16 + c8 * 8) / 8;      // 16-byte chunk index within the row
+                    *reinterpret_cast<uint4*>(qtile + (c16g / 8) * C::Q_CHUNK + row * 128 +
+                                              (((c16g % 8) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
             fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&bars.out_staged[i]));
-            if (row == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
+            warp_arrive(&bars.out_staged[i]);
+            if (row == 0 && hf == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
                 for (int ch = 0; ch < C::CH; ++ch)
                     tma_store_3d(&map_o, s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, ch * 64,
                                  qb[i] * p.Bq, bh);
@@ -493,7 +523,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tma_store_wait_all();
             }
 #ifndef SALAD_TRACE
-            if (p.lse != nullptr) {
+            if (p.lse != nullptr && hf == 0) {
                 const int n = qb[i] * p.Bq + row;
                 if (row < p.Bq && n < p.N)
                     p.lse[size_t(bh) * p.N + n] =
