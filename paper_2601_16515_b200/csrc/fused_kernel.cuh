@@ -35,8 +35,10 @@ namespace salad {
 
 #ifdef SALAD_TRACE
 #define TRACE(role, step, k) do { if (blockIdx.x == 700 && (step) < 64) reinterpret_cast<long long*>(p.lse)[((role) * 64 + (step)) * 8 + (k)] = clock64(); } while (0)
+#define TRACE_CTA(k) do { reinterpret_cast<long long*>(p.lse)[4096 + blockIdx.x * 8 + (k)] = (long long)global_timer_ns(); } while (0)
 #else
 #define TRACE(role, step, k) do {} while (0)
+#define TRACE_CTA(k) do {} while (0)
 #endif
 
 enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
@@ -65,10 +67,17 @@ struct FusedCfg {
     static constexpr int KV_BYTES = CH * KV_CHUNK;  // one K or V tile
     static constexpr int ST_CHUNK = D * 128;
     static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]
+#ifdef SALAD_EXPERIMENT_RINGS   /* sparse-only experiment: no room for the state tile */
+    static constexpr int NK = 5, NV = 4;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_ST = 2 * Q_BYTES;
+    static constexpr int OFF_K = OFF_ST;
+#else
     static constexpr int NK = 4, NV = 3;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_ST = 2 * Q_BYTES;
     static constexpr int OFF_K = OFF_ST + ST_BYTES;
+#endif
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int OFF_X = OFF_V + NV * KV_BYTES;               // row exchange between column halves
     static constexpr int X_BYTES = 2 * 2 * 4 * 128 * 4;              // [tile][half][slot][row] floats
@@ -79,8 +88,8 @@ struct FusedCfg {
 };
 
 struct FusedBarriers {
-    uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t q_tmem[2], s_full[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
+    uint64_t q_full[2], st_full, k_full[8], k_empty[8], v_full[8], v_empty[8];
+    uint64_t q_tmem[2], s_full[2], s_free[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
     uint64_t pair[2][4];   // the two warps that share a 32-row TMEM lane quarter of a tile
 };
 
@@ -134,11 +143,16 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     // ------------------------------------------------------------------ set-up
     if (tid == 0) {
+        TRACE_CTA(0);
+#ifdef SALAD_TRACE
+        { uint32_t smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); reinterpret_cast<long long*>(p.lse)[4096 + blockIdx.x * 8 + 7] = smid; }
+#endif
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
             mbar_init(smem_u32(&bars.q_tmem[i]), 8);        // one arrival per softmax warp
             mbar_init(smem_u32(&bars.s_full[i]), 1);
+            mbar_init(smem_u32(&bars.s_free[i]), 8);
             mbar_init(smem_u32(&bars.p_ready[i]), 8);
             mbar_init(smem_u32(&bars.o_final[i]), 1);
             mbar_init(smem_u32(&bars.lin_ready[i]), 8);
@@ -147,7 +161,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&bars.pair[i][qd]), 2);
         }
         mbar_init(smem_u32(&bars.st_full), 1);
-        for (int s = 0; s < 4; ++s) {
+        for (int s = 0; s < 8; ++s) {
             mbar_init(smem_u32(&bars.k_full[s]), 1);
             mbar_init(smem_u32(&bars.k_empty[s]), 2);     // released by both issuing threads
             mbar_init(smem_u32(&bars.v_full[s]), 1);
@@ -171,6 +185,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    if (tid == 0) TRACE_CTA(1);
 
     if (abort_flag == 0) {
     if (warp == 0) {
@@ -236,15 +251,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tc_fence_after_sync();
             }
             MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
-            int col, tag, ncol = 0, ntag = 0, g = 0, t = 0;
-            bool have = ok && wk.next(col, tag);
-            while (ok && have) {
-                const bool mine = (tag >> i) & 1;
-                const int sk = g % C::NK, sv = g % C::NV;
-                const uint32_t par = (g / C::NK) & 1, par_v = (g / C::NV) & 1;
-                TRACE(2 + i, g, 0);
-                ok = mbar_wait(smem_u32(&bars.k_full[sk]), par, abortp);
-                if (!ok) break;
+            int col, tag, ncol = 0, ntag = 0, g = 0, t = 0, steps = 0, pairs = 0;
+            // K part of entry g: S = Q K^T for an own entry, release only for a foreign one
+            auto k_part = [&](int ge, bool mine) -> bool {
+                const int sk = ge % C::NK;
+                if (!mbar_wait(smem_u32(&bars.k_full[sk]), (ge / C::NK) & 1, abortp)) return false;
                 if (mine) {
                     tc_fence_after_sync();
                     const uint32_t kb_lo = k_lo0 + sk * (C::KV_BYTES >> 4);
@@ -257,28 +268,60 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 } else {
                     mbar_arrive(smem_u32(&bars.k_empty[sk]));
                 }
-                TRACE(2 + i, g, 1);
-                const bool have_next = wk.next(ncol, ntag);     // list reads overlap the waits below
-                ok = mbar_wait(smem_u32(&bars.v_full[sv]), par_v, abortp);
-                if (!ok) break;
+                return true;
+            };
+            // V part of entry g: O += P V with P at TMEM column p_col for an own entry
+            auto v_part = [&](int ge, bool mine, uint32_t p_col, bool first) -> bool {
+                const int sv = ge % C::NV;
+                if (!mbar_wait(smem_u32(&bars.v_full[sv]), (ge / C::NV) & 1, abortp)) return false;
                 if (mine) {
-                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), t & 1, abortp);
-                    if (!ok) break;
-                    TRACE(2 + i, g, 2);
                     tc_fence_after_sync();
                     const uint32_t vb_lo = v_lo0 + sv * (C::KV_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
-                        mma_ts_lohi(t_tile + C::COL_O, t_tile + C::COL_S + k * 8, vb_lo + ((k * 2048) >> 4), HI,
-                                    idesc_pv, (t > 0 || k > 0) ? 1u : 0u);
+                        mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
+                                    (!first || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&bars.v_empty[sv]));
-                    ++t;
-                    if (t == len) tc_commit(smem_u32(&bars.o_final[i]));
-                    TRACE(2 + i, g, 3);
                 } else {
                     mbar_arrive(smem_u32(&bars.v_empty[sv]));
                 }
-                ++g;
+                return true;
+            };
+            bool have = ok && wk.next(col, tag);
+            while (ok && have) {
+                const bool mine = (tag >> i) & 1;
+                TRACE(2 + i, g, 0);
+                ok = k_part(g, mine);
+                if (!ok) break;
+                TRACE(2 + i, g, 1);
+                bool have_next = wk.next(ncol, ntag);     // list reads overlap the waits below
+                if (!mine) {
+                    ok = v_part(g, false, 0, false);
+                    ++g;
+                } else if (have_next && ((ntag >> i) & 1)) {
+                    // the next entry is this tile's too: its scores are computed as soon as the
+                    // softmax warps have read the first block's, and both blocks share one P hand-over
+                    ok = mbar_wait(smem_u32(&bars.s_free[i]), pairs & 1, abortp);
+                    if (!ok) break;
+                    ok = k_part(g + 1, true);
+                    if (!ok) break;
+                    have_next = wk.next(ncol, ntag);
+                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), steps & 1, abortp);
+                    if (!ok) break;
+                    TRACE(2 + i, g, 2);
+                    ok = v_part(g, true, t_tile + C::COL_S, t == 0) && v_part(g + 1, true, t_tile + C::COL_S + 32, false);
+                    TRACE(2 + i, g, 3);
+                    g += 2; t += 2; ++steps; ++pairs;
+                    if (ok && t == len) tc_commit(smem_u32(&bars.o_final[i]));
+                } else {
+                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), steps & 1, abortp);
+                    if (!ok) break;
+                    TRACE(2 + i, g, 2);
+                    ok = v_part(g, true, t_tile + C::COL_S, t == 0);
+                    TRACE(2 + i, g, 3);
+                    ++g; ++t; ++steps;
+                    if (ok && t == len) tc_commit(smem_u32(&bars.o_final[i]));
+                }
                 have = have_next; col = ncol; tag = ntag;
             }
             if (ok && linear && qb[i] < p.nQb) {
@@ -347,95 +390,135 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
 
         const bool ragged_keys = (p.N % C::BK) != 0;
-        for (int t = 0; t < len && ok; ++t) {
-            if (row == 0 && hf == 0) TRACE(i, t, 0);
-            // only the last key block can be short; its id is needed only then
-            const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
-            ok = wait_uniform(&bars.s_full[i], t & 1);
-            if (!ok) break;
-            if (row == 0 && hf == 0) TRACE(i, t, 1);
-            tc_fence_after_sync();
-            uint32_t xr[32];
-            tmem_ld32(t_tile + C::COL_S + hf * 32, xr);
-            tmem_wait_ld();
-            if (row == 0 && hf == 0) TRACE(i, t, 2);
-            float* x = reinterpret_cast<float*>(xr);
-            const int valid = p.N - col * C::BK - hf * 32;     // keys of this half that exist
-            if (ragged_keys && valid < 32) {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) if (c >= valid) x[c] = -INFINITY;
+        // Blocks are taken one or two per hand-over of P.  Two when the tile's next kept block is
+        // also the next entry of the merged list (no block of the other tile in between), the
+        // same rule the issuing thread applies.
+        const int32_t* own = p.col_idx + ls[i];
+        const int32_t* oth = p.col_idx + ls[i ^ 1];
+        const int oth_len = le[i ^ 1] - ls[i ^ 1];
+        int eo = 0;                               // cursor into the other tile's list
+        int bar_phase = 0;                        // phases of pair_bar used so far
+        int steps = 0;
+        uint32_t pk[2][16];
+        for (int t = 0; t < len && ok; ) {
+            const int col_a = __ldg(own + t);
+            bool paired = false;
+            if (t + 1 < len) {
+                const int col_b = __ldg(own + t + 1);
+                while (eo < oth_len && __ldg(oth + eo) <= col_a) ++eo;
+                paired = (eo == oth_len) || (__ldg(oth + eo) >= col_b);
             }
-            // max of this half of the row; published to the other half's thread
-            float mx[4];
+            const int nb = paired ? 2 : 1;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) mx[c] = x[c];
+            for (int j = 0; j < 2; ++j) {
+                if (j >= nb) break;
+                const int tt = t + j;
+                const int col = j == 0 ? col_a : __ldg(own + tt);
+                if (row == 0 && hf == 0) TRACE(i, tt, 0);
+                ok = wait_uniform(&bars.s_full[i], tt & 1);
+                if (!ok) break;
+                if (row == 0 && hf == 0) TRACE(i, tt, 1);
+                tc_fence_after_sync();
+                uint32_t xr[32];
+                tmem_ld32(t_tile + C::COL_S + hf * 32, xr);
+                tmem_wait_ld();
+                if (row == 0 && hf == 0) TRACE(i, tt, 2);
+                if (j == 0 && paired) {
+                    // the S columns are in registers: the second block's scores may overwrite them
+                    tc_fence_before_sync();
+                    warp_arrive(&bars.s_free[i]);
+                }
+                float* x = reinterpret_cast<float*>(xr);
+                const int valid = p.N - col * C::BK - hf * 32;     // keys of this half that exist
+                if (ragged_keys && valid < 32) {
 #pragma unroll
-            for (int c = 4; c < 32; c += 4) {
+                    for (int c = 0; c < 32; ++c) if (c >= valid) x[c] = -INFINITY;
+                }
+                // max of this half of the row; published to the other half's thread
+                float mx[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
-            }
-            const float lm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            x_mine[(t & 1) * 128] = lm;
-            warp_arrive(pair_bar);          // also tells the partner that this warp has read its S columns
+                for (int c = 0; c < 4; ++c) mx[c] = x[c];
+#pragma unroll
+                for (int c = 4; c < 32; c += 4) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
+                }
+                const float lm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                x_mine[(bar_phase & 1) * 128] = lm;
+                warp_arrive(pair_bar);      // also tells the partner that this warp has read its S columns
 
-            uint32_t pk[16];
-            auto exp_half = [&](float m_ref) -> float {   // P = exp2(x * scale - m_ref) as bf16 pairs; returns the sum
-                float s0 = 0.f, s1 = 0.f;
+                auto exp_half = [&](float m_ref) -> float {   // P = exp2(x * scale - m_ref) as bf16 pairs; returns the sum
+                    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
-                    const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
-                    s0 += p0; s1 += p1;
-                    pk[c >> 1] = pack_bf16x2(p0, p1);
+                    for (int c = 0; c < 32; c += 2) {
+                        const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
+                        const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
+                        s0 += p0; s1 += p1;
+                        pk[j][c >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    return s0 + s1;
+                };
+                float row_sum = 0.f;
+                // exponentials against the running max of the earlier blocks start at once; the
+                // max of this block only matters if it is more than 2^8 larger
+                if (tt > 0) row_sum = exp_half(m_run);
+                if (row == 0 && hf == 0) TRACE(i, tt, 6);
+                ok = wait_uniform(pair_bar, bar_phase & 1);
+                if (!ok) break;
+                if (row == 0 && hf == 0) TRACE(i, tt, 7);
+                const float msc = fmaxf(lm, x_other[(bar_phase & 1) * 128]) * p.scale_log2;   // same in both halves
+                ++bar_phase;
+                if (tt == 0) {
+                    m_run = msc;
+                    row_sum = exp_half(m_run);
+                } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
+                    // bring this thread's half of the accumulator to the new running max.  Every
+                    // earlier P V product is complete: it was issued before this block's Q K^T by
+                    // the same thread, and that product's completion was just observed.  A first
+                    // block of this hand-over is rescaled in its packed form.
+                    const float m_new = fmaxf(m_run, msc);
+                    const float alpha = ex2_approx(m_run - m_new);
+                    l_part *= alpha;
+                    m_run = m_new;
+#pragma unroll
+                    for (int cc = 0; cc < HD / 16; ++cc) {
+                        uint32_t orr[16];
+                        tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                        tmem_st16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                    }
+                    tmem_wait_st();
+                    if (j == 1) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const float lo = __uint_as_float(pk[0][c] << 16) * alpha;
+                            const float hi = __uint_as_float(pk[0][c] & 0xffff0000u) * alpha;
+                            pk[0][c] = pack_bf16x2(lo, hi);
+                        }
+                    }
+                    row_sum = exp_half(m_run);
                 }
-                return s0 + s1;
-            };
-            float row_sum = 0.f;
-            // exponentials against the running max of the earlier blocks start at once; the max
-            // of this block only matters if it is more than 2^8 larger
-            if (row == 0 && hf == 0) TRACE(i, t, 3);
-            if (t > 0) row_sum = exp_half(m_run);
-            if (row == 0 && hf == 0) TRACE(i, t, 6);
-            ok = wait_uniform(pair_bar, t & 1);
-            if (!ok) break;
-            if (row == 0 && hf == 0) TRACE(i, t, 7);
-            const float msc = fmaxf(lm, x_other[(t & 1) * 128]) * p.scale_log2;   // same value in both halves
-            if (t == 0) {
-                m_run = msc;
-                row_sum = exp_half(m_run);
-            } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
-                // bring this thread's half of the accumulator to the new running max.  The previous
-                // P V product is complete: it was issued before this block's Q K^T by the same
-                // thread, and that product's completion was just observed.
-                const float m_new = fmaxf(m_run, msc);
-                const float alpha = ex2_approx(m_run - m_new);
-                l_part *= alpha;
-                m_run = m_new;
-#pragma unroll
-                for (int cc = 0; cc < HD / 16; ++cc) {
-                    uint32_t orr[16];
-                    tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                    tmem_st16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
-                }
-                tmem_wait_st();
-                row_sum = exp_half(m_run);
+                l_part += row_sum;
+                if (row == 0 && hf == 0) TRACE(i, tt, 4);
             }
-            l_part += row_sum;
-            if (row == 0 && hf == 0) TRACE(i, t, 4);
-            // P over the S columns (the partner has read its S values: it arrived on pair_bar)
-            tmem_st16(t_tile + C::COL_S + hf * 16, pk);
+            if (!ok) break;
+            // P over the S columns.  The partner has read its S values of the last block: it
+            // arrived on pair_bar after loading them.
+            tmem_st16(t_tile + C::COL_S + hf * 16, pk[0]);
+            if (paired) tmem_st16(t_tile + C::COL_S + 32 + hf * 16, pk[1]);
             tmem_wait_st();
             tc_fence_before_sync();
             warp_arrive(&bars.p_ready[i]);
             if (row == 0 && hf == 0) TRACE(i, t, 5);
+            t += nb; ++steps;
         }
         if (ok && len > 0) {
             ok = wait_uniform(&bars.o_final[i], 0);
             tc_fence_after_sync();
         }
+        if (row == 0 && hf == 0) TRACE_CTA(2 + i);
 
         // row sum and linear denominator: add the two halves
         float den_part = 0.f;
@@ -469,7 +552,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             x_mine[2 * 128] = l_part;
             x_mine[3 * 128] = den_part;
             warp_arrive(pair_bar);
-            ok = wait_uniform(pair_bar, len & 1);
+            ok = wait_uniform(pair_bar, bar_phase & 1);
             if (ok) { l_run += x_other[2 * 128]; den += x_other[3 * 128]; }
         }
 
@@ -537,6 +620,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     // ------------------------------------------------------------------ tear-down
     tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) TRACE_CTA(4);
     if (abort_flag != 0) {
         // a bounded wait expired somewhere: report, give copies in flight time to land, leave
         if (tid == 0) {
