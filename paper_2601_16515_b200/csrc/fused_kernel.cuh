@@ -12,22 +12,25 @@
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
 // loaded.
 //
-// Both products read their A operand from tensor memory: a tcgen05.mma whose A comes from
-// shared memory costs ~110 cycles per 128xNx16 instruction on this part whatever N <= 128 is,
-// against ~60 with A in TMEM, so the Q tile is copied into TMEM once and S = Q K^T uses it
-// there; P = exp2(.) is written as bf16 over the S columns and O += P V reads it from TMEM.
-// Per tile the chain  S = Q K^T -> softmax -> O += P V  is serial (one S buffer); the two
-// tiles have their own issuing threads and run out of phase, so the tensor pipe works for
-// one tile while the other tile's warpgroup is in its softmax.
-// The softmax keeps a running max in the log2 domain and rescales the O accumulator only
-// when the max grows by more than 2^8.  After the last block the warpgroup applies ReLU to
-// its Q rows in shared memory, computes the linear denominator with plain FMAs, the issuing
-// thread multiplies ReLU(Q) with the bf16 linear state, and the epilogue writes
+// A single thread can issue a tcgen05.mma only every ~60 cycles, whatever its size, so the
+// work per instruction is kept large: whenever a tile's next kept block is also the next entry
+// of the merged list the two blocks form one step, S = Q [K_a; K_b]^T is one 128x128x16 MMA
+// series (the K ring is laid out chunk-major so that consecutive stages are contiguous rows),
+// and the softmax warps, the P hand-over and O += P V (with P read from TMEM, bf16, over the
+// S columns) all work on 128 keys at a time.  Per tile the chain S -> softmax -> O += P V is
+// serial; the two tiles have their own issuing threads and run out of phase, so the tensor
+// pipe works for one tile while the other tile's warps are in their softmax.
+// In a two-block step the two warpgroups of a tile take one block each (64 columns of every
+// row); in a one-block step the second warpgroup idles.  The running max lives in the log2
+// domain; exponentials start against the max of the earlier steps and the O accumulator is
+// rescaled only when the max grows by more than 2^8.  After the last block the warps apply
+// ReLU to their Q rows in shared memory, compute the linear denominator with plain FMAs, the
+// issuing thread multiplies ReLU(Q) with the bf16 linear state, and the epilogue writes
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
 //
-// TMEM columns (512 allocated), tile i at 256 i:  [0,64) S, first 32 reused for P;
-// [64,64+D/2) Q as bf16 pairs;  [128,128+D) O.  The linear numerator reuses [0,D).
+// TMEM columns (512 allocated), tile i at 256 i:  [0,128) S of up to two blocks, the first 32
+// columns of each 64 reused for P;  [128,128+D) O.  The linear numerator reuses [0,D).
 #pragma once
 #include "ptx.cuh"
 
@@ -67,13 +70,15 @@ struct FusedCfg {
     static constexpr int KV_BYTES = CH * KV_CHUNK;  // one K or V tile
     static constexpr int ST_CHUNK = D * 128;
     static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]
-#ifdef SALAD_EXPERIMENT_RINGS   /* sparse-only experiment: no room for the state tile */
-    static constexpr int NK = 5, NV = 4;
+#ifdef SALAD_EXPERIMENT_RINGS   /* sparse-only experiment: the state tile's space goes to the V ring */
+    static constexpr int NK = 4, NV = 5;
+    static constexpr int K_CH_STRIDE = NK * KV_CHUNK;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_ST = 2 * Q_BYTES;
     static constexpr int OFF_K = OFF_ST;
 #else
     static constexpr int NK = 4, NV = 3;
+    static constexpr int K_CH_STRIDE = NK * KV_CHUNK;   // K ring is [chunk][stage][64 rows x 128 B]
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_ST = 2 * Q_BYTES;
     static constexpr int OFF_K = OFF_ST + ST_BYTES;
@@ -84,12 +89,12 @@ struct FusedCfg {
     static constexpr int SMEM_BYTES = OFF_X + X_BYTES + 1024;         // + alignment slack
     static constexpr int THREADS = 640;
     // TMEM columns within a tile's 256
-    static constexpr uint32_t COL_S = 0, COL_Q = 64, COL_O = 128;
+    static constexpr uint32_t COL_S = 0, COL_O = 128;
 };
 
 struct FusedBarriers {
     uint64_t q_full[2], st_full, k_full[8], k_empty[8], v_full[8], v_empty[8];
-    uint64_t q_tmem[2], s_full[2], s_free[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
+    uint64_t s_full[2], p_ready[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
     uint64_t pair[2][4];   // the two warps that share a 32-row TMEM lane quarter of a tile
 };
 
@@ -119,6 +124,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __shared__ FusedBarriers bars;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int mma_turn;     // taken by the issuing thread whose MMA series owns the tensor pipe
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t s_base = smem_u32(smem);
@@ -148,12 +154,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         { uint32_t smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); reinterpret_cast<long long*>(p.lse)[4096 + blockIdx.x * 8 + 7] = smid; }
 #endif
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+        mma_turn = 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.q_tmem[i]), 8);        // one arrival per softmax warp
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_free[i]), 8);
-            mbar_init(smem_u32(&bars.p_ready[i]), 8);
+            mbar_init(smem_u32(&bars.p_ready[i]), 8);        // one arrival per softmax warp
             mbar_init(smem_u32(&bars.o_final[i]), 1);
             mbar_init(smem_u32(&bars.lin_ready[i]), 8);
             mbar_init(smem_u32(&bars.lin_done[i]), 1);
@@ -209,26 +214,30 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
             int col, tag, gk = 0, gv = 0, prev_col = -1;
             bool ok = true;
-            auto load_tile = [&](const CUtensorMap* m, uint32_t off, uint64_t* full, uint64_t* empty,
-                                 int g, int n_stage, int c) -> bool {
+            auto load_tile = [&](bool is_k, int g, int c) -> bool {
+                const int n_stage = is_k ? C::NK : C::NV;
+                uint64_t* full = is_k ? bars.k_full : bars.v_full;
+                uint64_t* empty = is_k ? bars.k_empty : bars.v_empty;
                 const int s = g % n_stage;
                 if (!mbar_wait(smem_u32(&empty[s]), ((g / n_stage) & 1) ^ 1, abortp)) return false;
                 const uint32_t bar = smem_u32(&full[s]);
                 mbar_arrive_expect_tx(bar, C::KV_BYTES);
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(s_base + off + s * C::KV_BYTES + ch * C::KV_CHUNK, m, bar, ch * 64,
-                                c * C::BK, bh);
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    const uint32_t dst = is_k ? s_base + C::OFF_K + ch * C::K_CH_STRIDE + s * C::KV_CHUNK
+                                              : s_base + C::OFF_V + s * C::KV_BYTES + ch * C::KV_CHUNK;
+                    tma_load_3d(dst, is_k ? &map_k : &map_v, bar, ch * 64, c * C::BK, bh);
+                }
                 return true;
             };
             // order of need: K(0), K(1), V(0), K(2), V(1), ...
             while (ok && wk.next(col, tag)) {
-                ok = load_tile(&map_k, C::OFF_K, bars.k_full, bars.k_empty, gk++, C::NK, col);
+                ok = load_tile(true, gk++, col);
                 if (ok && prev_col >= 0)
-                    ok = load_tile(&map_v, C::OFF_V, bars.v_full, bars.v_empty, gv++, C::NV, prev_col);
+                    ok = load_tile(false, gv++, prev_col);
                 prev_col = col;
             }
             if (ok && prev_col >= 0)
-                ok = load_tile(&map_v, C::OFF_V, bars.v_full, bars.v_empty, gv++, C::NV, prev_col);
+                ok = load_tile(false, gv++, prev_col);
         }
     } else if (warp == 1 || warp == 2) {
         // ============================================================== MMA issuer of tile i
@@ -237,99 +246,124 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // after waiting for the stage to be full so that a release can never run a phase ahead.
         if (lane == 0) {
             const int i = warp - 1;
-            const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
+            const uint32_t idesc_qk64 = make_idesc_bf16(128, 64, 0, 0);
+            const uint32_t idesc_qk128 = make_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
             const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
             constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
+            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
             const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
             const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
             const uint32_t t_tile = tmem + i * 256;
             const int len = le[i] - ls[i];
             bool ok = true;
             if (len > 0) {
-                ok = mbar_wait(smem_u32(&bars.q_tmem[i]), 0, abortp);
+                ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
                 tc_fence_after_sync();
             }
             MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
-            int col, tag, ncol = 0, ntag = 0, g = 0, t = 0, steps = 0, pairs = 0;
-            // K part of entry g: S = Q K^T for an own entry, release only for a foreign one
-            auto k_part = [&](int ge, bool mine) -> bool {
-                const int sk = ge % C::NK;
-                if (!mbar_wait(smem_u32(&bars.k_full[sk]), (ge / C::NK) & 1, abortp)) return false;
-                if (mine) {
-                    tc_fence_after_sync();
-                    const uint32_t kb_lo = k_lo0 + sk * (C::KV_BYTES >> 4);
+            int col, tag, ncol = 0, ntag = 0, g = 0, t = 0, steps = 0;
+            // S[:, d_col .. d_col + N) = Q K^T for N/64 consecutive K stages starting at sk
+            auto qk = [&](int sk, uint32_t d_col, uint32_t idesc) {
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k)   // 16 channels: 8 TMEM columns of Q, 32 bytes of each K row
-                        mma_ts_lohi(t_tile + C::COL_S, t_tile + C::COL_Q + k * 8,
-                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                    tc_commit(smem_u32(&bars.s_full[i]));
-                    tc_commit(smem_u32(&bars.k_empty[sk]));
-                } else {
-                    mbar_arrive(smem_u32(&bars.k_empty[sk]));
+                for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
+                    mma_ss_lohi(d_col, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                k_lo0 + (((k / 4) * C::K_CH_STRIDE + sk * C::KV_CHUNK + (k % 4) * 32) >> 4), HI,
+                                idesc, k > 0);
+            };
+            // O += P V for one block: P (bf16 pairs) at TMEM column p_col, V in stage sv
+            auto pv = [&](int sv, uint32_t p_col, bool first) {
+                const uint32_t vb_lo = v_lo0 + sv * (C::KV_BYTES >> 4);
+#pragma unroll
+                for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
+                    mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
+                                (!first || k > 0) ? 1u : 0u);
+            };
+            // The two tiles' MMA series must not interleave in the tensor pipe: interleaved, both
+            // tiles finish their products together, run their softmax together and the tensor
+            // and exponential units are never busy at the same time.  An issuing thread holds
+            // `mma_turn` for the duration of one series (never across a wait on a barrier), which
+            // keeps the tiles out of phase.
+            bool holding = false;
+            auto take_turn = [&]() -> bool {
+                if (holding) return true;
+                const uint64_t t0 = global_timer_ns();
+                while (atomicCAS(&mma_turn, 0, 1) != 0) {
+                    if (*abortp != 0) return false;
+                    if (global_timer_ns() - t0 > 1000000000ull) { *abortp = 1; return false; }
                 }
+                holding = true;
                 return true;
             };
-            // V part of entry g: O += P V with P at TMEM column p_col for an own entry
-            auto v_part = [&](int ge, bool mine, uint32_t p_col, bool first) -> bool {
-                const int sv = ge % C::NV;
-                if (!mbar_wait(smem_u32(&bars.v_full[sv]), (ge / C::NV) & 1, abortp)) return false;
-                if (mine) {
-                    tc_fence_after_sync();
-                    const uint32_t vb_lo = v_lo0 + sv * (C::KV_BYTES >> 4);
-#pragma unroll
-                    for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
-                        mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
-                                    (!first || k > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&bars.v_empty[sv]));
-                } else {
-                    mbar_arrive(smem_u32(&bars.v_empty[sv]));
-                }
-                return true;
+            auto give_turn = [&]() {
+                if (holding) { atomicExch(&mma_turn, 0); holding = false; }
             };
+            // the current and the next entry of the merged list are always known here
             bool have = ok && wk.next(col, tag);
+            bool have_n = have && wk.next(ncol, ntag);
             while (ok && have) {
                 const bool mine = (tag >> i) & 1;
+                const int sk = g % C::NK, sv = g % C::NV;
                 TRACE(2 + i, g, 0);
-                ok = k_part(g, mine);
-                if (!ok) break;
-                TRACE(2 + i, g, 1);
-                bool have_next = wk.next(ncol, ntag);     // list reads overlap the waits below
                 if (!mine) {
-                    ok = v_part(g, false, 0, false);
+                    // a block of the other tile only: release its stages, after they were filled
+                    ok = mbar_wait(smem_u32(&bars.k_full[sk]), (g / C::NK) & 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive(smem_u32(&bars.k_empty[sk]));
+                    have = have_n; col = ncol; tag = ntag;
+                    have_n = have && wk.next(ncol, ntag);
+                    ok = mbar_wait(smem_u32(&bars.v_full[sv]), (g / C::NV) & 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive(smem_u32(&bars.v_empty[sv]));
                     ++g;
-                } else if (have_next && ((ntag >> i) & 1)) {
-                    // the next entry is this tile's too: its scores are computed as soon as the
-                    // softmax warps have read the first block's, and both blocks share one P hand-over
-                    ok = mbar_wait(smem_u32(&bars.s_free[i]), pairs & 1, abortp);
-                    if (!ok) break;
-                    ok = k_part(g + 1, true);
-                    if (!ok) break;
-                    have_next = wk.next(ncol, ntag);
-                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), steps & 1, abortp);
-                    if (!ok) break;
-                    TRACE(2 + i, g, 2);
-                    ok = v_part(g, true, t_tile + C::COL_S, t == 0) && v_part(g + 1, true, t_tile + C::COL_S + 32, false);
-                    TRACE(2 + i, g, 3);
-                    g += 2; t += 2; ++steps; ++pairs;
-                    if (ok && t == len) tc_commit(smem_u32(&bars.o_final[i]));
-                } else {
-                    ok = mbar_wait(smem_u32(&bars.p_ready[i]), steps & 1, abortp);
-                    if (!ok) break;
-                    TRACE(2 + i, g, 2);
-                    ok = v_part(g, true, t_tile + C::COL_S, t == 0);
-                    TRACE(2 + i, g, 3);
-                    ++g; ++t; ++steps;
-                    if (ok && t == len) tc_commit(smem_u32(&bars.o_final[i]));
+                    continue;
                 }
-                have = have_next; col = ncol; tag = ntag;
+                const bool paired = have_n && ((ntag >> i) & 1);
+                const int sk2 = (g + 1) % C::NK, sv2 = (g + 1) % C::NV;
+                ok = mbar_wait(smem_u32(&bars.k_full[sk]), (g / C::NK) & 1, abortp);
+                if (ok && paired) ok = mbar_wait(smem_u32(&bars.k_full[sk2]), ((g + 1) / C::NK) & 1, abortp);
+                if (ok) ok = take_turn();
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (paired && sk2 == sk + 1) {
+                    qk(sk, t_tile + C::COL_S, idesc_qk128);            // both blocks in one series
+                } else {
+                    qk(sk, t_tile + C::COL_S, idesc_qk64);
+                    if (paired) qk(sk2, t_tile + C::COL_S + 64, idesc_qk64);   // ring wrapped between them
+                }
+                tc_commit(smem_u32(&bars.s_full[i]));
+                tc_commit(smem_u32(&bars.k_empty[sk]));
+                if (paired) tc_commit(smem_u32(&bars.k_empty[sk2]));
+                give_turn();
+                TRACE(2 + i, g, 1);
+                // advance the list while the softmax runs
+                if (paired) { have = wk.next(col, tag); have_n = have && wk.next(ncol, ntag); }
+                else { have = have_n; col = ncol; tag = ntag; have_n = have && wk.next(ncol, ntag); }
+                ok = mbar_wait(smem_u32(&bars.p_ready[i]), steps & 1, abortp);
+                if (ok) ok = mbar_wait(smem_u32(&bars.v_full[sv]), (g / C::NV) & 1, abortp);
+                if (ok && paired) ok = mbar_wait(smem_u32(&bars.v_full[sv2]), ((g + 1) / C::NV) & 1, abortp);
+                if (ok) ok = take_turn();
+                if (!ok) break;
+                TRACE(2 + i, g, 2);
+                tc_fence_after_sync();
+                pv(sv, t_tile + C::COL_S, t == 0);
+                tc_commit(smem_u32(&bars.v_empty[sv]));
+                if (paired) {
+                    pv(sv2, t_tile + C::COL_S + 64, false);
+                    tc_commit(smem_u32(&bars.v_empty[sv2]));
+                }
+                give_turn();
+                TRACE(2 + i, g, 3);
+                const int nb = paired ? 2 : 1;
+                g += nb; t += nb; ++steps;
+                if (t == len) tc_commit(smem_u32(&bars.o_final[i]));
             }
+            give_turn();
             if (ok && linear && qb[i] < p.nQb) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
                 if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
                 if (ok) {
                     tc_fence_after_sync();
-                    const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
                     const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST, 16);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k)
@@ -367,153 +401,124 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (lane == 0) mbar_arrive(smem_u32(bar));
         };
 
-        if (len > 0) {
-            // this thread's half of its Q row: shared memory (128-byte swizzle) -> TMEM, bf16 pairs
-            ok = wait_uniform(&bars.q_full[i], 0);
-            if (ok) {
-#pragma unroll
-                for (int part = 0; part < HD / 32; ++part) {      // 16 TMEM columns = 32 channels at a time
-                    uint32_t w[16];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int c16g = hf * (HD / 8) + part * 4 + j;    // 16-byte chunk index within the row
-                        const uint4 v = *reinterpret_cast<const uint4*>(qtile + (c16g / 8) * C::Q_CHUNK + row * 128 +
-                                                                        (((c16g % 8) ^ (row & 7)) << 4));
-                        w[j * 4 + 0] = v.x; w[j * 4 + 1] = v.y; w[j * 4 + 2] = v.z; w[j * 4 + 3] = v.w;
-                    }
-                    tmem_st16(t_tile + C::COL_Q + hf * (HD / 2) + part * 16, w);
-                }
-                tmem_wait_st();
-                tc_fence_before_sync();
-                warp_arrive(&bars.q_tmem[i]);
-            }
-        }
-
         const bool ragged_keys = (p.N % C::BK) != 0;
-        // Blocks are taken one or two per hand-over of P.  Two when the tile's next kept block is
-        // also the next entry of the merged list (no block of the other tile in between), the
-        // same rule the issuing thread applies.
+        // Steps take one or two blocks.  Two when the tile's next kept block is also the next
+        // entry of the merged list (no block of the other tile in between), the same rule the
+        // issuing thread applies.
         const int32_t* own = p.col_idx + ls[i];
         const int32_t* oth = p.col_idx + ls[i ^ 1];
         const int oth_len = le[i ^ 1] - ls[i ^ 1];
         int eo = 0;                               // cursor into the other tile's list
-        int bar_phase = 0;                        // phases of pair_bar used so far
-        int steps = 0;
-        uint32_t pk[2][16];
+        int steps = 0;                            // also the phase count of pair_bar
         for (int t = 0; t < len && ok; ) {
             const int col_a = __ldg(own + t);
+            int col_b = col_a;
             bool paired = false;
             if (t + 1 < len) {
-                const int col_b = __ldg(own + t + 1);
+                col_b = __ldg(own + t + 1);
                 while (eo < oth_len && __ldg(oth + eo) <= col_a) ++eo;
                 paired = (eo == oth_len) || (__ldg(oth + eo) >= col_b);
             }
-            const int nb = paired ? 2 : 1;
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                if (j >= nb) break;
-                const int tt = t + j;
-                const int col = j == 0 ? col_a : __ldg(own + tt);
-                if (row == 0 && hf == 0) TRACE(i, tt, 0);
-                ok = wait_uniform(&bars.s_full[i], tt & 1);
-                if (!ok) break;
-                if (row == 0 && hf == 0) TRACE(i, tt, 1);
-                tc_fence_after_sync();
-                uint32_t xr[32];
-                tmem_ld32(t_tile + C::COL_S + hf * 32, xr);
-                tmem_wait_ld();
-                if (row == 0 && hf == 0) TRACE(i, tt, 2);
-                if (j == 0 && paired) {
-                    // the S columns are in registers: the second block's scores may overwrite them
-                    tc_fence_before_sync();
-                    warp_arrive(&bars.s_free[i]);
-                }
-                float* x = reinterpret_cast<float*>(xr);
-                const int valid = p.N - col * C::BK - hf * 32;     // keys of this half that exist
-                if (ragged_keys && valid < 32) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) if (c >= valid) x[c] = -INFINITY;
-                }
-                // max of this half of the row; published to the other half's thread
-                float mx[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) mx[c] = x[c];
-#pragma unroll
-                for (int c = 4; c < 32; c += 4) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
-                }
-                const float lm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                x_mine[(bar_phase & 1) * 128] = lm;
-                warp_arrive(pair_bar);      // also tells the partner that this warp has read its S columns
+            const bool active = (hf == 0) || paired;          // warpgroup hf takes block hf of the step
+            const int valid = p.N - (hf == 0 ? col_a : col_b) * C::BK;   // keys of this block that exist
+            const uint32_t t_blk = t_tile + C::COL_S + hf * 64;
+            if (row == 0 && hf == 0) TRACE(i, steps, 0);
+            ok = wait_uniform(&bars.s_full[i], steps & 1);
+            if (!ok) break;
+            if (row == 0 && hf == 0) TRACE(i, steps, 1);
+            tc_fence_after_sync();
 
-                auto exp_half = [&](float m_ref) -> float {   // P = exp2(x * scale - m_ref) as bf16 pairs; returns the sum
-                    float s0 = 0.f, s1 = 0.f;
+            uint32_t pk[32];
+            float lm = -INFINITY, row_sum = 0.f;
+            // one pass over this thread's 64 scores, 32 at a time: block max, and (optionally)
+            // P = exp2(x * scale - m_ref) as bf16 pairs with its row sum
+            auto pass = [&](float m_ref, bool do_exp) {
+                lm = -INFINITY; row_sum = 0.f;
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                float sm[2] = {0.f, 0.f};
+                uint32_t xa[16], xb[16];
+                // 16 columns at a time; the next 16 are in flight while these are processed
+                auto chunk = [&](uint32_t* xr, int cc) {
+                    float* x = reinterpret_cast<float*>(xr);
+                    if (ragged_keys && valid - cc * 16 < 16) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
-                        const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
-                        s0 += p0; s1 += p1;
-                        pk[j][c >> 1] = pack_bf16x2(p0, p1);
+                        for (int c = 0; c < 16; ++c) if (c >= valid - cc * 16) x[c] = -INFINITY;
                     }
-                    return s0 + s1;
-                };
-                float row_sum = 0.f;
-                // exponentials against the running max of the earlier blocks start at once; the
-                // max of this block only matters if it is more than 2^8 larger
-                if (tt > 0) row_sum = exp_half(m_run);
-                if (row == 0 && hf == 0) TRACE(i, tt, 6);
-                ok = wait_uniform(pair_bar, bar_phase & 1);
-                if (!ok) break;
-                if (row == 0 && hf == 0) TRACE(i, tt, 7);
-                const float msc = fmaxf(lm, x_other[(bar_phase & 1) * 128]) * p.scale_log2;   // same in both halves
-                ++bar_phase;
-                if (tt == 0) {
-                    m_run = msc;
-                    row_sum = exp_half(m_run);
-                } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
-                    // bring this thread's half of the accumulator to the new running max.  Every
-                    // earlier P V product is complete: it was issued before this block's Q K^T by
-                    // the same thread, and that product's completion was just observed.  A first
-                    // block of this hand-over is rescaled in its packed form.
-                    const float m_new = fmaxf(m_run, msc);
-                    const float alpha = ex2_approx(m_run - m_new);
-                    l_part *= alpha;
-                    m_run = m_new;
 #pragma unroll
-                    for (int cc = 0; cc < HD / 16; ++cc) {
-                        uint32_t orr[16];
-                        tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
-                        tmem_wait_ld();
+                    for (int c = 0; c < 16; c += 4) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        tmem_st16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                        for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
                     }
-                    tmem_wait_st();
-                    if (j == 1) {
+                    if (do_exp) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const float lo = __uint_as_float(pk[0][c] << 16) * alpha;
-                            const float hi = __uint_as_float(pk[0][c] & 0xffff0000u) * alpha;
-                            pk[0][c] = pack_bf16x2(lo, hi);
+                        for (int c = 0; c < 16; c += 2) {
+                            const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
+                            const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
+                            sm[0] += p0; sm[1] += p1;
+                            pk[cc * 8 + (c >> 1)] = pack_bf16x2(p0, p1);
                         }
                     }
-                    row_sum = exp_half(m_run);
-                }
-                l_part += row_sum;
-                if (row == 0 && hf == 0) TRACE(i, tt, 4);
-            }
+                };
+                tmem_ld16(t_blk, xa);
+                tmem_wait_ld();
+                tmem_ld16(t_blk + 16, xb);
+                chunk(xa, 0);
+                tmem_wait_ld();
+                tmem_ld16(t_blk + 32, xa);
+                chunk(xb, 1);
+                tmem_wait_ld();
+                tmem_ld16(t_blk + 48, xb);
+                chunk(xa, 2);
+                tmem_wait_ld();
+                chunk(xb, 3);
+                lm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                row_sum = sm[0] + sm[1];
+            };
+            // exponentials against the running max of the earlier steps start at once; the max
+            // of this step only matters if it is more than 2^8 larger.  The first step has no
+            // earlier max and reduces first.
+            if (active) pass(m_run, steps > 0);
+            if (row == 0 && hf == 0) TRACE(i, steps, 2);
+            x_mine[(steps & 1) * 128] = lm;
+            warp_arrive(pair_bar);
+            ok = wait_uniform(pair_bar, steps & 1);
             if (!ok) break;
-            // P over the S columns.  The partner has read its S values of the last block: it
-            // arrived on pair_bar after loading them.
-            tmem_st16(t_tile + C::COL_S + hf * 16, pk[0]);
-            if (paired) tmem_st16(t_tile + C::COL_S + 32 + hf * 16, pk[1]);
-            tmem_wait_st();
+            const float msc = fmaxf(lm, x_other[(steps & 1) * 128]) * p.scale_log2;   // same in both halves
+            if (steps == 0) {
+                m_run = msc;
+                if (active) pass(m_run, true);
+            } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
+                // bring this thread's half of the accumulator to the new running max.  Every
+                // earlier P V product is complete: it was issued before this step's Q K^T by the
+                // same thread, and that product's completion was just observed.  The scores are
+                // still in TMEM (P has not been stored yet) and are read again.
+                const float m_new = fmaxf(m_run, msc);
+                const float alpha = ex2_approx(m_run - m_new);
+                l_part *= alpha;
+                m_run = m_new;
+#pragma unroll
+                for (int cc = 0; cc < HD / 16; ++cc) {
+                    uint32_t orr[16];
+                    tmem_ld16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                    tmem_st16(t_tile + C::COL_O + hf * HD + cc * 16, orr);
+                }
+                tmem_wait_st();
+                if (active) pass(m_run, true);
+            }
+            l_part += row_sum;
+            if (row == 0 && hf == 0) TRACE(i, steps, 4);
+            // P over the first 32 of this block's 64 S columns (read by this thread only)
+            if (active) { tmem_st32(t_blk, pk); tmem_wait_st(); }
             tc_fence_before_sync();
             warp_arrive(&bars.p_ready[i]);
-            if (row == 0 && hf == 0) TRACE(i, t, 5);
-            t += nb; ++steps;
+            if (row == 0 && hf == 0) TRACE(i, steps, 5);
+            t += paired ? 2 : 1;
+            ++steps;
         }
+        const int bar_phase = steps;
         if (ok && len > 0) {
             ok = wait_uniform(&bars.o_final[i], 0);
             tc_fence_after_sync();
