@@ -84,16 +84,24 @@ struct FusedBarriers {
 };
 
 // Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
+// The heads of both lists are loaded one call ahead, so that the global-load latency of an
+// entry is spent while the caller works on the previous one (the kernel leaves almost no L1).
 struct MergeWalk {
     const int32_t* col;
     int e0, end0, e1, end1;
+    int c0, c1;
+    __device__ __forceinline__ MergeWalk(const int32_t* c, int s0, int n0, int s1, int n1)
+        : col(c), e0(s0), end0(n0), e1(s1), end1(n1) {
+        c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff;
+        c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff;
+    }
     __device__ __forceinline__ bool next(int& c, int& tag) {
-        const int c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff;
-        const int c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff;
         c = min(c0, c1);
         if (c == 0x7fffffff) return false;
-        tag = (c0 == c ? 1 : 0) | (c1 == c ? 2 : 0);
-        e0 += (c0 == c); e1 += (c1 == c);
+        const bool a0 = (c0 == c), a1 = (c1 == c);
+        tag = (a0 ? 1 : 0) | (a1 ? 2 : 0);
+        if (a0) { ++e0; c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff; }
+        if (a1) { ++e1; c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff; }
         return true;
     }
 };
@@ -203,7 +211,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             uint64_t* empty = is_k ? bars.k_empty : bars.v_empty;
             const uint32_t ring = s_base + (is_k ? C::OFF_K : C::OFF_V);
             constexpr int NS = 4;                          // NK == NV
-            MergeWalk wk{p.col_idx, ls[0], le[0], ls[1], le[1]};
+            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
             int col, tag, g = 0;
             while (wk.next(col, tag)) {
                 const int s = g % NS;
@@ -239,15 +247,22 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // one side cannot keep it from serving the other side (which the other tile may be
             // waiting for through the shared K/V rings).
             struct Side { MergeWalk wk; int g, col, tag; bool have; };
-            Side ks{{p.col_idx, ls[0], le[0], ls[1], le[1]}, 0, 0, 0, false};
+            Side ks{MergeWalk(p.col_idx, ls[0], le[0], ls[1], le[1]), 0, 0, 0, false};
             Side vs = ks;
             ks.have = ok && ks.wk.next(ks.col, ks.tag);
             vs.have = ok && vs.wk.next(vs.col, vs.tag);
             int tk = 0, tv = 0;
+#ifdef SALAD_TRACE
+            long long cnt[6] = {0, 0, 0, 0, 0, 0};   // loops, p not ready, v not ready, k not ready, tk limit, progress
+#define CNT(j) (++cnt[j])
+#else
+#define CNT(j) do {} while (0)
+#endif
             uint32_t idle = 0;
             uint64_t idle_t0 = 0;
             while (ok && (ks.have || vs.have)) {
                 bool progress = false;
+                CNT(0);
                 if (vs.have) {
                     const int s = vs.g % C::NV;
                     const uint32_t par = (vs.g / C::NV) & 1;
@@ -256,8 +271,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             mbar_arrive(smem_u32(&bars.v_empty[s]));      // a block of the other tile only
                             progress = true;
                         }
-                    } else if (mbar_test(smem_u32(&bars.p_ready[i][tv & 1]), (tv >> 1) & 1) &&
-                               mbar_test(smem_u32(&bars.v_full[s]), par)) {
+                    } else if (!mbar_test(smem_u32(&bars.p_ready[i][tv & 1]), (tv >> 1) & 1)) {
+                        CNT(1);
+                    } else if (!mbar_test(smem_u32(&bars.v_full[s]), par)) {
+                        CNT(2);
+                    } else {
                         TRACE(2 + i, tv, 1);
                         tc_fence_after_sync();
                         const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
@@ -284,7 +302,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             mbar_arrive(smem_u32(&bars.k_empty[s]));
                             done = true;
                         }
-                    } else if (tk < tv + 2 && mbar_test(smem_u32(&bars.k_full[s]), par)) {
+                    } else if (tk >= tv + 2) {
+                        CNT(4);
+                    } else if (!mbar_test(smem_u32(&bars.k_full[s]), par)) {
+                        CNT(3);
+                    } else {
                         // S buffer tk & 1 is free: O += P V of block tk - 2 has been issued
                         TRACE(2 + i, tk, 0);
                         tc_fence_after_sync();
@@ -303,13 +325,16 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (done) { ++ks.g; ks.have = ks.wk.next(ks.col, ks.tag); progress = true; }
                 }
                 if (progress) {
-                    idle = 0;
+                    idle = 0; CNT(5);
                 } else if ((++idle & 255u) == 0u) {
                     if (idle == 256u) idle_t0 = global_timer_ns();
                     if (*abortp != 0) ok = false;
                     else if (global_timer_ns() - idle_t0 > 1000000000ull) { *abortp = 1; ok = false; }
                 }
             }
+#ifdef SALAD_TRACE
+            if (blockIdx.x == 700) for (int j = 0; j < 6; ++j) reinterpret_cast<long long*>(p.lse)[3000 + i * 8 + j] = cnt[j];
+#endif
             if (ok && linear && qb[i] < p.nQb) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
                 if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
