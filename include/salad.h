@@ -123,6 +123,34 @@ int salad_fused_fwd(const void* q, const void* k, const void* v, void* o,
                     int32_t* d_status, void* stream);
 
 /*
+ * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide
+ * scratch memory (the paper has no counterpart; this is a deployment convenience).
+ * Some hosts of this library may not call cudaMalloc at the point where attention runs: a
+ * plugin inside an inference server whose memory pool is fixed at start-up, code running
+ * while a CUDA graph is being captured or replayed, a real-time loop that must not touch the
+ * driver's allocator.  For them this entry point takes no workspace: its scratch (status
+ * word, partial and final linear states) lives in a fixed array inside the library image,
+ * SALAD_NOALLOC_SCRATCH_BYTES bytes of device memory that every GPU which loads the library
+ * holds until the process exits.
+ *   Arguments as salad_linear_attn_fwd, without workspace / workspace_bytes.
+ *   Limits: B*H <= SALAD_NOALLOC_MAX_HEADS and d in {64, 128}; anything larger returns
+ *   SALAD_ERR_UNSUPPORTED before any launch (use salad_linear_attn_fwd with a workspace).
+ *   The first call on each device looks up the device address of the array (one runtime
+ *   query, no allocation, with that device current); make that first call outside of any
+ *   stream capture.  Later calls only enqueue work.
+ *   All calls on a device share the one array: calls that may overlap on the GPU (different
+ *   streams, different host threads) race on it and must be serialised by the caller.  The
+ *   array keeps the previous call's contents; the call itself re-initialises everything it
+ *   reads (the status word is cleared, every partial it sums is rewritten first).
+ *   No cudaMalloc, cudaFree or other allocating routine is called.
+ */
+#define SALAD_NOALLOC_MAX_HEADS 16
+#define SALAD_NOALLOC_SCRATCH_BYTES 4759808
+int salad_linear_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o_l,
+                                  float* kv_out, float* z_out, int B, int H, int N, int d,
+                                  float eps, int32_t* d_status, void* stream);
+
+/*
  * salad_set_profile_events -- optional instrumentation for benchmarks (no counterpart in
  * the paper).  h_events is a HOST array of four cudaEvent_t handles (as void*), or NULL to
  * switch the instrumentation off.  While set, every *_fwd call made by the calling host

@@ -207,6 +207,55 @@ int run(const Problem& P) {
     return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }
 
+// ---------------------------------------------------------------------------------------
+// Scratch for salad_linear_attn_fwd_noalloc: a fixed array in the library image instead of a
+// caller workspace.  In host code the symbol below is only a handle; the device address is
+// obtained once per device with cudaGetSymbolAddress and cached.
+constexpr int kNoAllocSlots = 64;      // partial-state slots (batch*heads x chunks)
+
+constexpr size_t noalloc_align(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+constexpr size_t kNoAllocBytes =
+    kAlign +                                                              // status word
+    noalloc_align(size_t(SALAD_NOALLOC_MAX_HEADS) * 128 * 128 * 2) +      // bf16 transposed state
+    noalloc_align(size_t(SALAD_NOALLOC_MAX_HEADS) * 128 * 4) +            // Z
+    noalloc_align(size_t(kNoAllocSlots) * 128 * 128 * 4) +                // partial KV
+    noalloc_align(size_t(kNoAllocSlots) * 128 * 4);                       // partial Z
+static_assert(kNoAllocBytes == SALAD_NOALLOC_SCRATCH_BYTES, "header constant out of date");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+// Layout of the fixed scratch for this (B, H, d): the same regions as a caller workspace,
+// with fewer partial slots.
+Workspace carve_noalloc(int B, int H, int d) {
+    Workspace w;
+    const size_t BH = size_t(B) * H;
+    w.slots = kNoAllocSlots;
+    w.off_status = 0;
+    w.off_kvt = kAlign;
+    w.off_z = w.off_kvt + align_up(BH * d * d * 2);
+    w.off_kvp = w.off_z + align_up(BH * d * 4);
+    w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
+    w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
+    return w;
+}
+
+// Device address of g_noalloc_scratch on the current device (looked up on first use).
+int noalloc_scratch_ptr(void** out) {
+    static void* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return SALAD_ERR_CUDA;
+        }
+        cached[dev] = ptr;
+    }
+    *out = cached[dev];
+    return SALAD_OK;
+}
+
 }  // namespace
 
 SALAD_EXPORT const char* salad_status_string(int status) {
@@ -319,4 +368,40 @@ SALAD_EXPORT int salad_fused_fwd(const void* q, const void* k, const void* v, vo
     P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
     P.stream = static_cast<cudaStream_t>(stream);
     return run(P);
+}
+
+SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o_l,
+                                               float* kv_out, float* z_out, int B, int H, int N, int d,
+                                               float eps, int32_t* d_status, void* stream) {
+    if (!q || !k || !v || !o_l) return SALAD_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || N <= 0 || d <= 0) return SALAD_ERR_INVALID_ARG;
+    if (!(eps >= 0.f) || !isfinite(eps)) return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o_l)) return SALAD_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return SALAD_ERR_UNSUPPORTED;
+    if (int64_t(B) * H > SALAD_NOALLOC_MAX_HEADS) return SALAD_ERR_UNSUPPORTED;   // beyond the fixed scratch
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    void* scratch = nullptr;
+    rc = noalloc_scratch_ptr(&scratch);
+    if (rc != SALAD_OK) return rc;
+    const Workspace w = carve_noalloc(B, H, d);
+    if (w.total > kNoAllocBytes) return SALAD_ERR_UNSUPPORTED;
+
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o_l;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
+    P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;
+    P.ws = scratch; P.ws_bytes = kNoAllocBytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    // the array keeps the last call's contents: the status word must start at zero
+    uint8_t* ws = static_cast<uint8_t*>(scratch);
+    if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    if (d_status && cudaMemsetAsync(d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SALAD_ERR_CUDA;
+    }
+    rc = (d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
+    if (rc != SALAD_OK) return rc;
+    return (d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }

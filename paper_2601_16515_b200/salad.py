@@ -26,7 +26,7 @@ SALAD_ERR_TIMEOUT = -6
 
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
-           "salad_set_profile_events")
+           "salad_set_profile_events", "salad_linear_attn_fwd_noalloc")
 
 
 class SaladError(RuntimeError):
@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_linear_attn_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [f32, p, sz, p, p]
     lib.salad_fused_fwd.restype = i32
     lib.salad_fused_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, p, sz, p, p]
+    lib.salad_linear_attn_fwd_noalloc.restype = i32
+    lib.salad_linear_attn_fwd_noalloc.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [f32, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -172,6 +174,30 @@ def salad_linear_attn_fwd(q, k, v, eps: float = 1e-6, out=None, kv_out=None, z_o
         _check(_lib.salad_linear_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_out), _ptr(z_out),
                                           B, H, N, d, float(eps), _ptr(workspace), workspace.numel(),
                                           _ptr(status), _stream(stream)), "salad_linear_attn_fwd")
+    return out
+
+
+NOALLOC_MAX_HEADS = 16
+
+
+def salad_linear_attn_fwd_noalloc(q, k, v, eps: float = 1e-6, out=None, kv_out=None, z_out=None,
+                                  status=None, stream=None):
+    """ReLU linear attention without a workspace, for hosts that must not allocate device
+    memory when attention runs (fixed memory pools, capture/replay, real-time loops).  The
+    scratch is a fixed array inside the library (B*H <= 16, d in {64, 128}); calls on one
+    device share it and must not overlap on the GPU.  Pass `out` to avoid the one output
+    allocation this Python wrapper would otherwise make; the C entry point allocates nothing."""
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _bf16_4d(name, t)
+    if k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("q, k, v must have the same shape")
+    B, H, N, d = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_linear_attn_fwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_out), _ptr(z_out),
+                                                  B, H, N, d, float(eps), _ptr(status), _stream(stream)),
+               "salad_linear_attn_fwd_noalloc")
     return out
 
 
