@@ -48,6 +48,8 @@ struct FusedParams {
     int N, H, nQb, nKb, nPairs, Bq, Hm, mode;
     const int32_t* row_ptr;
     const int32_t* col_idx;
+    const int32_t* order;        // [Hm][nPairs] launch order of the query-block pairs, or null (identity)
+    int BH;                      // batch * heads
     const float* static_scale;   // [H] or null (=1)
     const float* dyn_scale;      // [B] or null (=1)
     const float* z;              // [B*H, D] linear normaliser state
@@ -122,9 +124,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    const int pair = blockIdx.x % p.nPairs, bh = blockIdx.x / p.nPairs;
+    // work item: head by head (K/V of one head stay hot in L2), within a head the pairs of query
+    // blocks from the most to the least expensive, so that the kernel ends on short items
+    const int rank = blockIdx.x % p.nPairs, bh = blockIdx.x / p.nPairs;
     const int h = bh % p.H, b = bh / p.H;
     const int hm = (p.Hm == 1) ? 0 : h;
+    const int pair = p.order ? __ldg(p.order + size_t(hm) * p.nPairs + rank) : rank;
     const bool sparse = (p.mode & MODE_SPARSE) != 0, linear = (p.mode & MODE_LINEAR) != 0;
 
     // kept lists of the two tiles

@@ -97,4 +97,32 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
     }
 }
 
+// Launch order of the attention kernel's work items: for every mask head, the pairs of query
+// blocks sorted by decreasing cost (the longer of the two kept lists), so that the long items
+// start first and the short ones fill the tail.  Counting sort in shared memory; one CTA per
+// mask head.  The order among equal costs is arbitrary (it only affects scheduling).
+__global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
+                                                          int nPairs, int32_t* __restrict__ order) {
+    constexpr int BINS = 2048;
+    __shared__ int hist[BINS];
+    const int hm = blockIdx.x, tid = threadIdx.x;
+    const int32_t* rp = row_ptr + size_t(hm) * nQb;
+    auto cost_of = [&](int pr) {
+        const int a = rp[2 * pr + 1] - rp[2 * pr];
+        const int b = (2 * pr + 1 < nQb) ? rp[2 * pr + 2] - rp[2 * pr + 1] : 0;
+        return min(BINS - 1, max(a, b));
+    };
+    for (int i = tid; i < BINS; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (int pr = tid; pr < nPairs; pr += blockDim.x) atomicAdd(&hist[cost_of(pr)], 1);
+    __syncthreads();
+    if (tid == 0) {                       // start position of every cost, largest cost first
+        int run = 0;
+        for (int c = BINS - 1; c >= 0; --c) { const int n = hist[c]; hist[c] = run; run += n; }
+    }
+    __syncthreads();
+    for (int pr = tid; pr < nPairs; pr += blockDim.x)
+        order[size_t(hm) * nPairs + atomicAdd(&hist[cost_of(pr)], 1)] = pr;
+}
+
 }  // namespace salad

@@ -30,20 +30,22 @@ inline void record_profile(int idx, cudaStream_t st) {
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
-    size_t off_status, off_kvt, off_z, off_kvp, off_zp, total;
+    size_t off_status, off_kvt, off_z, off_kvp, off_zp, off_order, total;
     int slots;
 };
 
-Workspace carve(int B, int H, int d) {
+Workspace carve(int B, int H, int N, int d, int Bq) {
     Workspace w;
     const size_t BH = size_t(B) * H;
+    const size_t nPairs = (size_t(N + Bq - 1) / Bq + 1) / 2;
     w.slots = int(BH > size_t(kPartialSlots) ? BH : size_t(kPartialSlots));
     w.off_status = 0;
     w.off_kvt = kAlign;
     w.off_z = w.off_kvt + align_up(BH * d * d * 2);
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
-    w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
+    w.off_order = w.off_zp + align_up(size_t(w.slots) * d * 4);
+    w.total = w.off_order + align_up(size_t(H) * nPairs * 4);       // launch order, per mask head
     return w;
 }
 
@@ -120,7 +122,7 @@ int validate(const Problem& P) {
         if (!(P.eps >= 0.f) || !isfinite(P.eps)) return SALAD_ERR_INVALID_ARG;
     }
     if (P.mode == MODE_FUSED && (!P.static_scale || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
-    const Workspace w = carve(P.B, P.H, P.d);
+    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
     if (!P.ws || (reinterpret_cast<uintptr_t>(P.ws) % kAlign) != 0 || P.ws_bytes < w.total)
         return SALAD_ERR_WORKSPACE;
     return SALAD_OK;
@@ -170,6 +172,15 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.nKb = (P.N + 63) / 64;
     fp.nPairs = (fp.nQb + 1) / 2;
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
+    fp.BH = BH;
+    fp.order = nullptr;
+    if (P.mode & MODE_SPARSE) {
+        // longest work items first (the mask is an input of every call, so is its order)
+        int32_t* order = reinterpret_cast<int32_t*>(ws + w.off_order);
+        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, fp.nQb, fp.nPairs, order);
+        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+        fp.order = order;
+    }
     fp.static_scale = P.static_scale; fp.dyn_scale = P.dyn_scale;
     fp.z = reinterpret_cast<const float*>(ws + w.off_z);
     fp.lse = P.lse;
@@ -193,7 +204,7 @@ int run(const Problem& P) {
     DeviceInfo dev{};
     rc = prepare_device(&dev);
     if (rc != SALAD_OK) return rc;
-    const Workspace w = carve(P.B, P.H, P.d);
+    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
     if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
     if (P.d_status && cudaMemsetAsync(P.d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
@@ -235,6 +246,7 @@ Workspace carve_noalloc(int B, int H, int d) {
     w.off_z = w.off_kvt + align_up(BH * d * d * 2);
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
+    w.off_order = 0;                                  // linear attention has no kept lists to order
     w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
     return w;
 }
@@ -279,7 +291,7 @@ SALAD_EXPORT int salad_set_profile_events(void* const* h_events) {
 
 SALAD_EXPORT size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk) {
     if (B <= 0 || H <= 0 || N <= 0 || !shape_supported(d, Bq, Bk)) return 0;
-    return carve(B, H, d).total;
+    return carve(B, H, N, d, Bq).total;
 }
 
 SALAD_EXPORT int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm, const int32_t* h_windows,
