@@ -12,11 +12,11 @@
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
 // loaded.
 //
-// Per tile, S = Q K^T (128x64xd, operands in shared memory) has two TMEM buffers: the issuing
-// thread computes the scores of block t+2 as soon as O += P V of block t has been issued, so
-// the softmax warps find the next block's scores waiting and the tensor pipe works while they
-// compute.  P = exp2(.) is written as bf16 over the S columns and O += P V reads it from
-// TMEM.  The running max lives in the log2 domain; exponentials start against the max of the
+// Per tile, S = Q K^T (128x64xd, operands in shared memory) lands in one TMEM buffer that the
+// softmax warps copy to registers at once and hand back, so the scores of block t+1 are
+// computed while the softmax of block t runs.  P = exp2(.) goes, as bf16, to one of two P
+// buffers in TMEM (so O += P V of block t, which reads P from TMEM, overlaps the softmax of
+// block t+1).  The running max lives in the log2 domain; exponentials start against the max of the
 // earlier blocks and the O accumulator is rescaled only when the max grows by more than 2^8.
 // Each issuing thread walks the merged list twice, once for the Q K^T side (two own blocks
 // ahead) and once for the P V side; blocks of the other tile are only released, always after
@@ -27,8 +27,8 @@
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
 //
-// TMEM columns (512 allocated), tile i at 256 i:  [0,64) and [64,128) the two S buffers, the
-// first 32 columns of each reused for P;  [128,128+D) O.  The linear numerator reuses [0,D).
+// TMEM columns (512 allocated), tile i at 256 i:  [0,64) S;  [64,96) and [96,128) the two P
+// buffers;  [128,128+D) O.  The linear numerator reuses [0,D).
 #pragma once
 #include "ptx.cuh"
 
@@ -77,12 +77,12 @@ struct FusedCfg {
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
     static constexpr int THREADS = 384;
-    static constexpr uint32_t COL_S = 0, COL_O = 128;                 // TMEM columns within a tile's 256
+    static constexpr uint32_t COL_S = 0, COL_P = 64, COL_O = 128;     // TMEM columns within a tile's 256
 };
 
 struct FusedBarriers {
     uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2][2], p_ready[2][2], pv_done[2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
+    uint64_t s_full[2], s_free[2], p_ready[2][2], pv_done[2][2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
 };
 
 // Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
@@ -150,14 +150,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.pv_done[i]), 1);
+            mbar_init(smem_u32(&bars.s_full[i]), 1);
+            mbar_init(smem_u32(&bars.s_free[i]), 4);              // one arrival per softmax warp
             mbar_init(smem_u32(&bars.o_final[i]), 1);
             mbar_init(smem_u32(&bars.lin_ready[i]), 128);
             mbar_init(smem_u32(&bars.lin_done[i]), 1);
             mbar_init(smem_u32(&bars.out_staged[i]), 128);
             for (int j = 0; j < 2; ++j) {
-                mbar_init(smem_u32(&bars.s_full[i][j]), 1);
-                mbar_init(smem_u32(&bars.p_ready[i][j]), 4);      // one arrival per softmax warp
+                mbar_init(smem_u32(&bars.p_ready[i][j]), 4);
+                mbar_init(smem_u32(&bars.pv_done[i][j]), 1);
             }
         }
         mbar_init(smem_u32(&bars.st_full), 1);
@@ -246,8 +247,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
                 tc_fence_after_sync();
             }
-            // Two walks of the merged list: the Q K^T side runs up to two own blocks ahead of the
-            // P V side.  The thread never blocks on a single barrier here: it polls what each side
+            // Two walks of the merged list: the Q K^T side runs ahead of the P V side (by the block
+            // whose scores are being computed while the previous block's softmax runs).  The thread never blocks on a single barrier here: it polls what each side
             // needs next and does whatever is ready, so a long run of the other tile's blocks on
             // one side cannot keep it from serving the other side (which the other tile may be
             // waiting for through the shared K/V rings).
@@ -284,13 +285,13 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         TRACE(2 + i, tv, 1);
                         tc_fence_after_sync();
                         const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
-                        const uint32_t p_col = t_tile + C::COL_S + (tv & 1) * 64;
+                        const uint32_t p_col = t_tile + C::COL_P + (tv & 1) * 32;
 #pragma unroll
                         for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
                             mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
                                         (tv > 0 || k > 0) ? 1u : 0u);
                         tc_commit(smem_u32(&bars.v_empty[s]));
-                        tc_commit(smem_u32(&bars.pv_done[i]));
+                        tc_commit(smem_u32(&bars.pv_done[i][tv & 1]));
                         ++tv;
                         if (tv == len) tc_commit(smem_u32(&bars.o_final[i]));
                         TRACE(2 + i, tv - 1, 2);
@@ -316,12 +317,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         TRACE(2 + i, tk, 0);
                         tc_fence_after_sync();
                         const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
-                        const uint32_t d_col = t_tile + C::COL_S + (tk & 1) * 64;
+                        const uint32_t d_col = t_tile + C::COL_S;
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
                             mma_ss_lohi(d_col, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
                                         kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                        tc_commit(smem_u32(&bars.s_full[i][tk & 1]));
+                        tc_commit(smem_u32(&bars.s_full[i]));
                         tc_commit(smem_u32(&bars.k_empty[s]));
                         ++tk;
                         TRACE(2 + i, tk - 1, 3);
@@ -376,15 +377,18 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (row == 0) TRACE(i, t, 0);
             // only the last key block can be short; its id is needed only then
             const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
-            const uint32_t t_buf = t_tile + C::COL_S + (t & 1) * 64;     // S buffer of this block
-            ok = wait_uniform(&bars.s_full[i][t & 1], (t >> 1) & 1);
+            ok = wait_uniform(&bars.s_full[i], t & 1);
             if (!ok) break;
             if (row == 0) TRACE(i, t, 1);
             tc_fence_after_sync();
             uint32_t xr[64];
-            tmem_ld32(t_buf, xr);
-            tmem_ld32(t_buf + 32, xr + 32);
+            tmem_ld32(t_tile + C::COL_S, xr);
+            tmem_ld32(t_tile + C::COL_S + 32, xr + 32);
             tmem_wait_ld();
+            // the scores are in registers: the S buffer may take the next block's
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[i]));
             if (row == 0) TRACE(i, t, 2);
             float* x = reinterpret_cast<float*>(xr);
             const int valid = p.N - col * C::BK;          // keys of this block that exist
@@ -427,10 +431,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const float msc = row_max_scaled();
                 if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
                     // bring the accumulator of this warp's rows to the new running max, once the
-                    // previous P V product has landed in it.  pv_done cycles once per block and
-                    // is at most one phase behind here (the product of block t cannot be issued
-                    // before this thread hands over P of block t), so the parity test is exact.
-                    ok = wait_uniform(&bars.pv_done[i], (t - 1) & 1);
+                    // previous P V product has landed in it.  pv_done[b] completes a phase for
+                    // every second block; the product of block t cannot be issued before this
+                    // thread hands over P of block t, so the barrier is at most one phase past
+                    // the one tested here and the parity test is exact.
+                    ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const float m_new = fmaxf(m_run, msc);
@@ -452,7 +457,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             l_run += row_sum;
             if (row == 0) TRACE(i, t, 4);
-            tmem_st32(t_buf, pk);                 // P over the first 32 columns of the block's S buffer
+            if (t >= 2) {
+                // P buffer t & 1 was read by the P V product of block t - 2
+                ok = wait_uniform(&bars.pv_done[i][t & 1], ((t >> 1) - 1) & 1);
+                if (!ok) break;
+            }
+            tmem_st32(t_tile + C::COL_P + (t & 1) * 32, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
