@@ -3,11 +3,13 @@
 //
 // One CTA owns two consecutive query blocks of one (batch, head): two 128-row MMA tiles.
 //   warp 0        TMA producer of the Q tiles, the linear-state tile and the K ring
-//   warp 3        TMA producer of the V ring (independent of the K ring, so neither ring can
+//   warp 1        TMA producer of the V ring (independent of the K ring, so neither ring can
 //                 stall the other)
-//   warp 1, 2     tcgen05 MMA issuers of tile 0 and tile 1 (one thread each); warp 1 owns TMEM
-//   warps 4-7     softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
-//   warps 8-11    the same for tile 1
+//   warps 2, 3    tcgen05 issuers of S = Q K^T for tile 0 and tile 1 (one thread each); warp 2
+//                 owns the TMEM allocation
+//   warps 4, 5    tcgen05 issuers of O += P V (and of the linear numerator) for tile 0 and 1
+//   warps 8-11    softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
+//   warps 12-15   the same for tile 1
 // The kept lists of the two query blocks are walked as one sorted merge, so a key block that
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
 // loaded.
@@ -18,9 +20,10 @@
 // buffers in TMEM (so O += P V of block t, which reads P from TMEM, overlaps the softmax of
 // block t+1).  The running max lives in the log2 domain; exponentials start against the max of the
 // earlier blocks and the O accumulator is rescaled only when the max grows by more than 2^8.
-// Each issuing thread walks the merged list twice, once for the Q K^T side (two own blocks
-// ahead) and once for the P V side; blocks of the other tile are only released, always after
-// waiting for the stage to be full so that a release can never run a phase ahead.
+// The two products of a tile have their own issuing threads: each walks the merged list,
+// waits only for what its next MMA series needs (so it reacts as soon as that arrives), and
+// releases the ring stages of the other tile's blocks, always after waiting for the stage to
+// be full so that a release can never run a phase ahead.
 // After the last block the warpgroup applies ReLU to its Q rows in shared memory, computes
 // the linear denominator with plain FMAs, the issuing thread multiplies ReLU(Q) with the bf16
 // linear state, and the epilogue writes
@@ -76,7 +79,7 @@ struct FusedCfg {
     static constexpr int OFF_K = OFF_ST + ST_BYTES;
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
-    static constexpr int THREADS = 384;
+    static constexpr int THREADS = 512;
     static constexpr uint32_t COL_S = 0, COL_P = 64, COL_O = 128;     // TMEM columns within a tile's 256
 };
 
@@ -109,7 +112,7 @@ struct MergeWalk {
 };
 
 template <int D>
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(512, 1)
 salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                    const __grid_constant__ CUtensorMap map_st, const FusedParams p)
@@ -180,7 +183,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         fence_proxy_async_smem();
     }
-    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
+    if (warp == 2) { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -189,7 +192,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (tid == 0) TRACE_CTA(1);
 
     if (abort_flag == 0) {
-    if (warp == 0 || warp == 3) {
+    if (warp == 0 || warp == 1) {
         // ============================================================== TMA producers
         if (lane == 0) {
             const bool is_k = (warp == 0);
@@ -229,17 +232,14 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ++g;
             }
         }
-    } else if (warp == 1 || warp == 2) {
-        // ============================================================== MMA issuer of tile i
+    } else if (warp == 2 || warp == 3) {
+        // ============================================================== issuer of S = Q K^T, tile i
         if (lane == 0) {
-            const int i = warp - 1;
+            const int i = warp - 2;
             const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
-            const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
-            const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
             constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
             const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
             const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
-            const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
             const uint32_t t_tile = tmem + i * 256;
             const int len = le[i] - ls[i];
             bool ok = true;
@@ -247,100 +247,72 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
                 tc_fence_after_sync();
             }
-            // Two walks of the merged list: the Q K^T side runs ahead of the P V side (by the block
-            // whose scores are being computed while the previous block's softmax runs).  The thread never blocks on a single barrier here: it polls what each side
-            // needs next and does whatever is ready, so a long run of the other tile's blocks on
-            // one side cannot keep it from serving the other side (which the other tile may be
-            // waiting for through the shared K/V rings).
-            struct Side { MergeWalk wk; int g, col, tag; bool have; };
-            Side ks{MergeWalk(p.col_idx, ls[0], le[0], ls[1], le[1]), 0, 0, 0, false};
-            Side vs = ks;
-            ks.have = ok && ks.wk.next(ks.col, ks.tag);
-            vs.have = ok && vs.wk.next(vs.col, vs.tag);
-            int tk = 0, tv = 0;
-#ifdef SALAD_TRACE
-            long long cnt[6] = {0, 0, 0, 0, 0, 0};   // loops, p not ready, v not ready, k not ready, tk limit, progress
-#define CNT(j) (++cnt[j])
-#else
-#define CNT(j) do {} while (0)
-#endif
-            uint32_t idle = 0;
-            uint64_t idle_t0 = 0;
-            while (ok && (ks.have || vs.have)) {
-                bool progress = false;
-                CNT(0);
-                if (vs.have) {
-                    const int s = vs.g % C::NV;
-                    const uint32_t par = (vs.g / C::NV) & 1;
-                    if (!((vs.tag >> i) & 1)) {
-                        if (mbar_test(smem_u32(&bars.v_full[s]), par)) {
-                            mbar_arrive(smem_u32(&bars.v_empty[s]));      // a block of the other tile only
-                            progress = true;
-                        }
-                    } else if (!mbar_test(smem_u32(&bars.p_ready[i][tv & 1]), (tv >> 1) & 1)) {
-                        CNT(1);
-                    } else if (!mbar_test(smem_u32(&bars.v_full[s]), par)) {
-                        CNT(2);
-                    } else {
-                        TRACE(2 + i, tv, 1);
-                        tc_fence_after_sync();
-                        const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
-                        const uint32_t p_col = t_tile + C::COL_P + (tv & 1) * 32;
+            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
+            int col, tag, g = 0, t = 0;
+            while (ok && wk.next(col, tag)) {
+                const int s = g % C::NK;
+                ok = mbar_wait(smem_u32(&bars.k_full[s]), (g / C::NK) & 1, abortp);
+                if (!ok) break;
+                if ((tag >> i) & 1) {
+                    // the softmax warps must have copied the scores of the previous block out of S
+                    if (t > 0) ok = mbar_wait(smem_u32(&bars.s_free[i]), (t - 1) & 1, abortp);
+                    if (!ok) break;
+                    TRACE(2 + i, t, 0);
+                    tc_fence_after_sync();
+                    const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
-                        for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
-                            mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
-                                        (tv > 0 || k > 0) ? 1u : 0u);
-                        tc_commit(smem_u32(&bars.v_empty[s]));
-                        tc_commit(smem_u32(&bars.pv_done[i][tv & 1]));
-                        ++tv;
-                        if (tv == len) tc_commit(smem_u32(&bars.o_final[i]));
-                        TRACE(2 + i, tv - 1, 2);
-                        progress = true;
-                    }
-                    if (progress) { ++vs.g; vs.have = vs.wk.next(vs.col, vs.tag); }
+                    for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
+                        mma_ss_lohi(t_tile + C::COL_S, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
+                    tc_commit(smem_u32(&bars.s_full[i]));
+                    tc_commit(smem_u32(&bars.k_empty[s]));
+                    TRACE(2 + i, t, 3);
+                    ++t;
+                } else {
+                    mbar_arrive(smem_u32(&bars.k_empty[s]));      // a block of the other tile only
                 }
-                if (ks.have) {
-                    const int s = ks.g % C::NK;
-                    const uint32_t par = (ks.g / C::NK) & 1;
-                    bool done = false;
-                    if (!((ks.tag >> i) & 1)) {
-                        if (mbar_test(smem_u32(&bars.k_full[s]), par)) {
-                            mbar_arrive(smem_u32(&bars.k_empty[s]));
-                            done = true;
-                        }
-                    } else if (tk >= tv + 2) {
-                        CNT(4);
-                    } else if (!mbar_test(smem_u32(&bars.k_full[s]), par)) {
-                        CNT(3);
-                    } else {
-                        // S buffer tk & 1 is free: O += P V of block tk - 2 has been issued
-                        TRACE(2 + i, tk, 0);
-                        tc_fence_after_sync();
-                        const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
-                        const uint32_t d_col = t_tile + C::COL_S;
-#pragma unroll
-                        for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
-                            mma_ss_lohi(d_col, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
-                                        kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                        tc_commit(smem_u32(&bars.s_full[i]));
-                        tc_commit(smem_u32(&bars.k_empty[s]));
-                        ++tk;
-                        TRACE(2 + i, tk - 1, 3);
-                        done = true;
-                    }
-                    if (done) { ++ks.g; ks.have = ks.wk.next(ks.col, ks.tag); progress = true; }
-                }
-                if (progress) {
-                    idle = 0; CNT(5);
-                } else if ((++idle & 255u) == 0u) {
-                    if (idle == 256u) idle_t0 = global_timer_ns();
-                    if (*abortp != 0) ok = false;
-                    else if (global_timer_ns() - idle_t0 > 1000000000ull) { *abortp = 1; ok = false; }
-                }
+                ++g;
             }
-#ifdef SALAD_TRACE
-            if (blockIdx.x == 700) for (int j = 0; j < 6; ++j) reinterpret_cast<long long*>(p.lse)[3000 + i * 8 + j] = cnt[j];
-#endif
+        }
+    } else if (warp == 4 || warp == 5) {
+        // ============================================================== issuer of O += P V, tile i
+        if (lane == 0) {
+            const int i = warp - 4;
+            const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+            const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
+            constexpr uint32_t HI = sdesc_hi_sw128(1024);
+            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
+            const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
+            const uint32_t t_tile = tmem + i * 256;
+            const int len = le[i] - ls[i];
+            bool ok = true;
+            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
+            int col, tag, g = 0, t = 0;
+            while (ok && wk.next(col, tag)) {
+                const int s = g % C::NV;
+                ok = mbar_wait(smem_u32(&bars.v_full[s]), (g / C::NV) & 1, abortp);
+                if (!ok) break;
+                if ((tag >> i) & 1) {
+                    ok = mbar_wait(smem_u32(&bars.p_ready[i][t & 1]), (t >> 1) & 1, abortp);
+                    if (!ok) break;
+                    TRACE(2 + i, t, 1);
+                    tc_fence_after_sync();
+                    const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
+                    const uint32_t p_col = t_tile + C::COL_P + (t & 1) * 32;
+#pragma unroll
+                    for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
+                        mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
+                                    (t > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&bars.v_empty[s]));
+                    tc_commit(smem_u32(&bars.pv_done[i][t & 1]));
+                    ++t;
+                    if (t == len) tc_commit(smem_u32(&bars.o_final[i]));
+                    TRACE(2 + i, t - 1, 2);
+                } else {
+                    mbar_arrive(smem_u32(&bars.v_empty[s]));
+                }
+                ++g;
+            }
             if (ok && linear && qb[i] < p.nQb) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
                 if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
@@ -355,10 +327,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 8) {
         // ============================================================== softmax + epilogue
-        const int i = (warp - 4) >> 2;            // tile
-        const int row = tid - 128 - 128 * i;      // query row within the tile = TMEM lane
+        const int i = (warp - 8) >> 2;            // tile
+        const int row = tid - 256 - 128 * i;      // query row within the tile = TMEM lane
         const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
         const uint32_t t_tile = tmem + i * 256 + lane_addr;
         const bool tile_valid = qb[i] < p.nQb;
@@ -420,41 +392,36 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 return s0 + s1;
             };
-            float row_sum;
+            // the block max first (the running max only moves when it grows by more than 2^8),
+            // then one pass of exponentials: the scores die as P is packed
+            const float msc = row_max_scaled();
             if (t == 0) {
-                m_run = row_max_scaled();
-                row_sum = exp_row(m_run);
-            } else {
-                // exponentials against the running max of the earlier blocks start at once; the
-                // max of this block is found alongside and only matters if it is 2^8 larger
-                row_sum = exp_row(m_run);
-                const float msc = row_max_scaled();
-                if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
-                    // bring the accumulator of this warp's rows to the new running max, once the
-                    // previous P V product has landed in it.  pv_done[b] completes a phase for
-                    // every second block; the product of block t cannot be issued before this
-                    // thread hands over P of block t, so the barrier is at most one phase past
-                    // the one tested here and the parity test is exact.
-                    ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const float m_new = fmaxf(m_run, msc);
-                    const float alpha = ex2_approx(m_run - m_new);
-                    l_run *= alpha;
-                    m_run = m_new;
+                m_run = msc;
+            } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
+                // bring the accumulator of this warp's rows to the new running max, once the
+                // previous P V product has landed in it.  pv_done[b] completes a phase for
+                // every second block; the product of block t cannot be issued before this
+                // thread hands over P of block t, so the barrier is at most one phase past
+                // the one tested here and the parity test is exact.
+                ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const float m_new = fmaxf(m_run, msc);
+                const float alpha = ex2_approx(m_run - m_new);
+                l_run *= alpha;
+                m_run = m_new;
 #pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t orr[32];
-                        tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
-                        tmem_wait_ld();
+                for (int cc = 0; cc < D / 16; ++cc) {
+                    uint32_t orr[16];
+                    tmem_ld16(t_tile + C::COL_O + cc * 16, orr);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        tmem_st32(t_tile + C::COL_O + cc * 32, orr);
-                    }
-                    tmem_wait_st();
-                    row_sum = exp_row(m_run);
+                    for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                    tmem_st16(t_tile + C::COL_O + cc * 16, orr);
                 }
+                tmem_wait_st();
             }
+            const float row_sum = exp_row(m_run);
             l_run += row_sum;
             if (row == 0) TRACE(i, t, 4);
             if (t >= 2) {
@@ -515,13 +482,13 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // O = O_acc / l + lin_coef * num, rounded once to bf16, staged in the Q tile
             const float inv_l = (len > 0) ? 1.0f / l_run : 0.f;
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
-                uint32_t orr[32], nr[32];
-                if (len > 0) tmem_ld32(t_tile + C::COL_O + cc * 32, orr);
-                if (linear) tmem_ld32(t_tile + cc * 32, nr);
+            for (int cc = 0; cc < D / 16; ++cc) {
+                uint32_t orr[16], nr[16];
+                if (len > 0) tmem_ld16(t_tile + C::COL_O + cc * 16, orr);
+                if (linear) tmem_ld16(t_tile + cc * 16, nr);
                 tmem_wait_ld();
 #pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
+                for (int c8 = 0; c8 < 2; ++c8) {
                     uint32_t w[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -534,7 +501,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                         w[e] = pack_bf16x2(o0, o1);
                     }
-                    const int col16 = (cc * 32 + c8 * 8) / 8;      // 16-byte chunk index within the row
+                    const int col16 = (cc * 16 + c8 * 8) / 8;      // 16-byte chunk index within the row
                     const int ch = col16 / 8, c16 = col16 % 8;
                     *reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
@@ -574,7 +541,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
         __syncthreads();
     }
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace salad
