@@ -122,6 +122,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __shared__ FusedBarriers bars;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ float z_s[D];          // linear normaliser state of this head
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t s_base = smem_u32(smem);
@@ -184,6 +185,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         fence_proxy_async_smem();
     }
     if (warp == 2) { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
+    if (linear && tid >= 256 && tid < 256 + D) z_s[tid - 256] = __ldg(p.z + size_t(bh) * D + (tid - 256));
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -436,17 +438,13 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i][t & 1]));   // one arrival per warp
             if (row == 0) TRACE(i, t, 5);
         }
-        if (ok && len > 0) {
-            ok = wait_uniform(&bars.o_final[i], 0);
-            tc_fence_after_sync();
-        }
-
         float lin_coef = 0.f;
         if (ok && tile_valid && linear) {
-            // ReLU of this thread's Q row in place, and the denominator ReLU(Q_n) . Z
+            // ReLU of this thread's Q row in place, and the denominator ReLU(Q_n) . Z.  Every
+            // Q K^T of this tile has completed (its scores were consumed above), so Q is no
+            // longer read; the last P V product may still be running meanwhile.
             ok = wait_uniform(&bars.q_full[i], 0);
             if (ok) {
-                const float* zrow = p.z + size_t(bh) * D;
                 float den = 0.f;
 #pragma unroll
                 for (int ch = 0; ch < C::CH; ++ch) {
@@ -461,8 +459,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
                             const float2 f = __bfloat1622float2(hv[e]);
                             const int a = ch * 64 + c16 * 8 + e * 2;
-                            den = fmaf(f.x, __ldg(zrow + a), den);
-                            den = fmaf(f.y, __ldg(zrow + a + 1), den);
+                            den = fmaf(f.x, z_s[a], den);
+                            den = fmaf(f.y, z_s[a + 1], den);
                         }
                         *ptr = v;
                     }
@@ -473,9 +471,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 lin_coef = c_scale / (den + p.eps);
                 fence_proxy_async_smem();
                 mbar_arrive(smem_u32(&bars.lin_ready[i]));
-                ok = wait_uniform(&bars.lin_done[i], 0);
-                tc_fence_after_sync();
             }
+        }
+        if (ok && len > 0) {
+            ok = wait_uniform(&bars.o_final[i], 0);
+            tc_fence_after_sync();
+        }
+        if (ok && tile_valid && linear) {
+            ok = wait_uniform(&bars.lin_done[i], 0);
+            tc_fence_after_sync();
         }
 
         if (ok && tile_valid) {
