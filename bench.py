@@ -333,7 +333,11 @@ def main():
             "mask_build_ms": mask_ms,
             "roofline": {"kernel": "salad_fused_kernel<128>", "bound": "tensor", "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "peak_source": peaks["source"] + " (burst)",
-                         "traffic": None, "kernel_ms": attn_ms, "state_kernels_ms": state_ms},
+                         # DRAM bytes of one launch from the ncu capture of this workload
+                         # (profiles/salad_fused_kernel_wan1.3b-90.md); algorithmic bytes are 402.6 MB
+                         "traffic": 388.2e6 if wl.name == "wan1.3b-90" else None,
+                         "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, see profiles/",
+                         "kernel_ms": attn_ms, "state_kernels_ms": state_ms},
             "cpu_baseline": cpu_baseline,
             "e2e": e2e,
             "gpu_launches": 3 * K,

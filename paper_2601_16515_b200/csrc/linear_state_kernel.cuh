@@ -1,7 +1,8 @@
 // Linear-attention state (Eq. 3):  KV = sum_j ReLU(K_j)^T V_j  (d x d),  Z = sum_j ReLU(K_j).
 //
 // HBM-bound: K and V are read exactly once.  The token axis of every (batch, head) is cut
-// into `chunks` contiguous ranges of key blocks (64 tokens); one CTA streams one range:
+// into `chunks` contiguous ranges of key blocks (64 tokens); one CTA per SM streams one range
+// through a six-stage ring (192 KB in flight per SM):
 //   warp 0      TMA producer, K and V tiles through a ring of stages
 //   warp 1      tcgen05 MMA issuer; per 16 tokens one MMA  D[d x d] += ReLU(K)^T V with both
 //               operands token-major in shared memory (MN-major descriptors), plus one
@@ -28,7 +29,7 @@ struct StateCfg {
     static constexpr int T_CHUNK = BK * 128;           // bytes of one 64-column chunk of a tile
     static constexpr int T_BYTES = CH * T_CHUNK;       // one K or V tile
     static constexpr int STAGE_BYTES = 2 * T_BYTES;    // K then V
-    static constexpr int STAGES = (D == 128) ? 3 : 4;
+    static constexpr int STAGES = (D == 128) ? 6 : 8;
     static constexpr int OFF_ONES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = OFF_ONES + 2048 + 1024;
     static constexpr int THREADS = 192;
@@ -198,22 +199,44 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
                              __nv_bfloat16* __restrict__ kvt)
 {
-    const int bh = blockIdx.y;
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;     // a * D + c
-    if (idx < D * D) {
-        const float* src = kv_part + size_t(bh) * chunks * D * D + idx;
-        float s = 0.f;
-        for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D * D];
-        if (kv_out) kv_out[size_t(bh) * D * D + idx] = s;
-        const int a = idx / D, c = idx % D;
-        kvt[size_t(bh) * D * D + c * D + a] = __float2bfloat16(s);
+    // grid (D/32, D/32, BH), block (32, 8): one 32 x 32 tile of KV per block, transposed through
+    // shared memory so that both the partial reads and the bf16 writes are coalesced
+    __shared__ float tile[32][33];
+    const int bh = blockIdx.z;
+    const int a0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const size_t head = size_t(bh) * chunks * D * D;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int a = a0 + ty + 8 * j;
+        const float* src = kv_part + head + size_t(a) * D + c0 + tx;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        int ch = 0;
+        for (; ch + 4 <= chunks; ch += 4) {           // fixed order: ((p0+p4+..)+(p1+p5+..))+...
+            s0 += src[size_t(ch) * D * D];
+            s1 += src[size_t(ch + 1) * D * D];
+            s2 += src[size_t(ch + 2) * D * D];
+            s3 += src[size_t(ch + 3) * D * D];
+        }
+        for (; ch < chunks; ++ch) s0 += src[size_t(ch) * D * D];
+        const float s = (s0 + s1) + (s2 + s3);
+        if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
+        tile[ty + 8 * j][tx] = s;
     }
-    if (idx < D) {
-        const float* src = z_part + size_t(bh) * chunks * D + idx;
-        float s = 0.f;
-        for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];
-        z_ws[size_t(bh) * D + idx] = s;
-        if (z_out) z_out[size_t(bh) * D + idx] = s;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int c = c0 + ty + 8 * j;
+        kvt[size_t(bh) * D * D + size_t(c) * D + a0 + tx] = __float2bfloat16(tile[tx][ty + 8 * j]);
+    }
+    if (blockIdx.x == 0 && blockIdx.y == 0) {
+        for (int a = ty * 32 + tx; a < D; a += 256) {
+            const float* src = z_part + size_t(bh) * chunks * D + a;
+            float s = 0.f;
+            for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];
+            z_ws[size_t(bh) * D + a] = s;
+            if (z_out) z_out[size_t(bh) * D + a] = s;
+        }
     }
 }
 

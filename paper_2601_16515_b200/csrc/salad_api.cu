@@ -132,7 +132,7 @@ template <int D>
 int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     const int BH = P.B * P.H;
     const int nKb = (P.N + 63) / 64;
-    int chunks = (2 * dev.sms) / BH;
+    int chunks = dev.sms / BH;          // one CTA per SM (its stage ring takes most of the shared memory)
     if (chunks < 1) chunks = 1;
     if (chunks > nKb) chunks = nKb;
     if (int64_t(chunks) * BH > w.slots) chunks = w.slots / BH;
@@ -150,7 +150,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     record_profile(0, P.stream);
     salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    salad_linear_finalize_kernel<D><<<dim3((D * D + 255) / 256, BH), 256, 0, P.stream>>>(
+    salad_linear_finalize_kernel<D><<<dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream>>>(
         sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
         reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt));
     record_profile(1, P.stream);
