@@ -31,7 +31,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2601_16515_b200 import workloads as wlmod  # noqa: E402
+from paper_2601_16515_b200 import dist_util, workloads as wlmod  # noqa: E402
 
 METRIC = "fused_salad_attn_kept_block_tflops"
 UNIT = "TFLOP/s"
@@ -250,11 +250,10 @@ def main():
     total_ms = t_start.elapsed_time(t_stop)
     state_ms = float(np.mean([g[0].elapsed_time(g[1]) for g in evs]))
     attn_ms = float(np.mean([g[2].elapsed_time(g[3]) for g in evs]))
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / K
-    value = flops * world / (ms_per_step * 1e-3) / 1e12
+    # every rank did `flops` of work; the job took the slowest rank's time (weak scaling)
+    flops_per_s, total_ms_max = dist_util.aggregate_throughput(flops * K, total_ms, dev)
+    ms_per_step = total_ms_max / K
+    value = flops_per_s / 1e12
 
     # ---------------- end to end: host buffers in, host buffer out, every step
     def e2e_step():
@@ -271,10 +270,7 @@ def main():
         e2e_step()
     t_stop.record()
     barrier()
-    te = torch.tensor([t_start.elapsed_time(t_stop)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_ms = float(te.item()) / Ke
+    e2e_ms = dist_util.max_over_ranks(t_start.elapsed_time(t_stop), dev) / Ke
     tensor_bytes = q_h.numel() * q_h.element_size()
     e2e = {"value": flops * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": 3 * tensor_bytes, "d2h_bytes_per_step": tensor_bytes}
