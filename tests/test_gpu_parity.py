@@ -299,3 +299,45 @@ def test_fused_cfg_pair_sparsity_sweep(salad, wl):
 
 def test_fused_cfg_pair_dense(salad):
     sampled_fused_check(salad, wlmod.C5_DENSE, heads=[8], nrows=120)
+
+
+# ------------------------------------------------------------------------------ API behaviour
+
+def test_runs_on_a_side_stream_and_is_deterministic(salad):
+    B, H, N, d = 2, 2, 1500, 128
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), 128, 64, (), 1)
+    q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 77))
+    rp, ci = random_csr(wl.nQb, wl.nKb, 5, lo=1, hi=wl.nKb)          # one mask for all heads and batch items
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = torch.tensor([0.3, 0.9], dtype=torch.float32, device="cuda")
+    s = torch.tensor([0.5, 0.25], dtype=torch.float32, device="cuda")
+    ws = salad.alloc_workspace(B, H, N, d)
+    side = torch.cuda.Stream()
+    outs = []
+    for _ in range(2):
+        out = torch.empty_like(q)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            salad.salad_fused_fwd(q, k, v, rp_d, ci_d, 1, lam, s, out=out, workspace=ws, stream=side)
+        side.synchronize()
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])                               # same launch, same bits
+    ref = orc.salad_fused(f32(q.cpu()), f32(k.cpu()), f32(v.cpu()), 128, 64, rp, ci, 1,
+                          lam.cpu().numpy(), s.cpu().numpy())
+    assert_close(f32(outs[0].cpu()).reshape(-1, d), ref, "side stream")
+
+
+def test_binding_rejects_bad_tensors(salad):
+    q, k, v = (t.cuda() for t in rand_qkv(1, 1, 128, 64, 3))
+    rp, ci = dev_csr(*wlmod.dense_csr(1, 2, 1))
+    with pytest.raises(ValueError):
+        salad.salad_sparse_attn_fwd(q.float(), k, v, rp, ci, 1)                 # not bf16
+    with pytest.raises(ValueError):
+        salad.salad_sparse_attn_fwd(q, k[:, :, :64], v, rp, ci, 1)               # shape mismatch
+    with pytest.raises(salad.SaladError) as err:
+        salad.salad_sparse_attn_fwd(q, k, v, rp, ci, 1, Bq=32)                   # unsupported block size
+    assert err.value.code in (salad.SALAD_ERR_UNSUPPORTED, salad.SALAD_ERR_WORKSPACE)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(salad.SaladError) as err:
+        salad.salad_sparse_attn_fwd(q, k, v, rp, ci, 1, workspace=small)
+    assert err.value.code == salad.SALAD_ERR_WORKSPACE
