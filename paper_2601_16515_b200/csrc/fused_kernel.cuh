@@ -371,28 +371,35 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
             }
             auto row_max_scaled = [&]() -> float {
-                float mx[8];
+                float mx[4] = {x[0], x[1], x[2], x[3]};
 #pragma unroll
-                for (int c = 0; c < 8; ++c) mx[c] = x[c];
+                for (int c = 4; c < C::BK - 4; c += 8) {
 #pragma unroll
-                for (int c = 8; c < C::BK; c += 8) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) mx[e] = fmaxf(mx[e], x[c + e]);
+                    for (int e = 0; e < 4; ++e) mx[e] = fmaxf(fmaxf(mx[e], x[c + e]), x[c + 4 + e]);
                 }
-                return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                             fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[C::BK - 4 + e]);
+                return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
             };
             uint32_t pk[32];
             auto exp_row = [&](float m_ref) -> float {    // P = exp2(x * scale - m_ref), packed bf16; returns the row sum
-                float s0 = 0.f, s1 = 0.f;
+                const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(-m_ref, -m_ref);
+                uint64_t acc0 = pack_f32x2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
-                for (int c = 0; c < C::BK; c += 2) {
-                    const float p0 = ex2_approx(fmaf(x[c], p.scale_log2, -m_ref));
-                    const float p1 = ex2_approx(fmaf(x[c + 1], p.scale_log2, -m_ref));
-                    s0 += p0; s1 += p1;
+                for (int c = 0; c < C::BK; c += 4) {              // scale-and-shift and the row sum two at a time
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), sc2, nm2), a0, a1);
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), sc2, nm2), a2, a3);
+                    const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(a2), p3 = ex2_approx(a3);
+                    acc0 = add_f32x2(acc0, pack_f32x2(p0, p1));
+                    acc1 = add_f32x2(acc1, pack_f32x2(p2, p3));
                     pk[c >> 1] = pack_bf16x2(p0, p1);
+                    pk[(c >> 1) + 1] = pack_bf16x2(p2, p3);
                 }
-                return s0 + s1;
+                float s0, s1, s2, s3;
+                unpack_f32x2(acc0, s0, s1);
+                unpack_f32x2(acc1, s2, s3);
+                return (s0 + s1) + (s2 + s3);
             };
             // the block max first (the running max only moves when it grows by more than 2^8),
             // then one pass of exponentials: the scores die as P is packed
