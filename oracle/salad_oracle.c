@@ -249,3 +249,46 @@ ORACLE_API void oracle_salad_fused(const float* q, const float* k, const float* 
     }
     free(kv); free(z); free(ol);
 }
+
+/*
+ * oracle_dynamic_scale: the input- and timestep-aware scaling factor of Algorithm 1, Level 2,
+ *     s[b] = Mean_n sigmoid( <X_t[b,n,:], w> + bias ),
+ * one scalar per batch item (a token average of a sigmoid of a D -> 1 linear layer, Sec. 4.2).
+ * The paper counts D x 1 weights and does not mention a bias; bias is an argument (0 = none).
+ *   x  [B, N, D] (bf16-representable values widened to fp32),  w [D],  s [B] out.
+ */
+ORACLE_API void oracle_dynamic_scale(const float* x, const float* w, double bias, int B, int N, int D,
+                                     double* s)
+{
+    for (int b = 0; b < B; ++b) {
+        double total = 0.0;
+#pragma omp parallel for reduction(+ : total) schedule(static)
+        for (int n = 0; n < N; ++n) {
+            const float* xn = x + ((int64_t)b * N + n) * (int64_t)D;
+            double z = bias;
+            for (int c = 0; c < D; ++c) z += (double)xn[c] * (double)w[c];
+            total += 1.0 / (1.0 + exp(-z));
+        }
+        s[b] = total / (double)N;
+    }
+}
+
+/*
+ * oracle_salad_fused_drop: Algorithm 1 with post-tuning branch dropping (Sec. 4.3, Appendix
+ * A.3): the linear branch of a batch item is skipped when its scaling factor is below the
+ * threshold,
+ *     O[b,h,n] = O_s[b,h,n] + [s[b] >= tau] * s[b] * lambda[h] * O_l[b,h,n].
+ */
+ORACLE_API void oracle_salad_fused_drop(const float* q, const float* k, const float* v,
+                                        int B, int H, int N, int d, int Bq, int Bk,
+                                        const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                        const double* lambda_h, const double* s_b, double tau,
+                                        double scale, double eps,
+                                        const int64_t* sel, int64_t nsel, double* o)
+{
+    double* s_eff = (double*)malloc(sizeof(double) * (size_t)B);
+    for (int b = 0; b < B; ++b) s_eff[b] = (s_b[b] >= tau) ? s_b[b] : 0.0;
+    oracle_salad_fused(q, k, v, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_eff, scale, eps,
+                       sel, nsel, o);
+    free(s_eff);
+}

@@ -48,6 +48,11 @@ def _load():
         lib.oracle_salad_fused.restype = None
         lib.oracle_salad_fused.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64,
                                                                     p, i64, p])
+        lib.oracle_dynamic_scale.restype = None
+        lib.oracle_dynamic_scale.argtypes = [p, p, f64, i32, i32, i32, p]
+        lib.oracle_salad_fused_drop.restype = None
+        lib.oracle_salad_fused_drop.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
+                                                                         p, i64, p])
         _lib = lib
     return _lib
 
@@ -153,4 +158,33 @@ def salad_fused(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, scale=None
         scale = 1.0 / np.sqrt(d)
     lib.oracle_salad_fused(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
                            sb.ctypes.data, float(scale), float(eps), sp, nsel, o.ctypes.data)
+    return o
+
+
+def dynamic_scale(x, w, bias=0.0):
+    """Alg. 1 Level 2: s[b] = mean_n sigmoid(<x[b,n,:], w> + bias).  x [B,N,D], w [D] -> [B] float64."""
+    lib = _load()
+    x, xp = _f32(x); w, wp = _f32(w)
+    B, N, D = x.shape
+    assert w.size == D
+    s = np.empty(B, dtype=np.float64)
+    lib.oracle_dynamic_scale(xp, wp, float(bias), B, N, D, s.ctypes.data)
+    return s
+
+
+def salad_fused_drop(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, tau, scale=None, eps=1e-6,
+                     sel=None):
+    """Fused output with branch dropping: the linear branch of batch item b is skipped when s_b < tau."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = q.shape
+    rp, rpp = _i32(row_ptr); ci, cip = _i32(col_idx if len(col_idx) else np.zeros(1, np.int32))
+    lam = np.ascontiguousarray(lambda_h, dtype=np.float64); sb = np.ascontiguousarray(s_b, dtype=np.float64)
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    lib.oracle_salad_fused_drop(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
+                                sb.ctypes.data, float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
     return o

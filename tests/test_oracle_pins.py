@@ -304,3 +304,40 @@ def test_workloads_are_seeded_and_sliceable():
         assert (np.diff(row) > 0).all() and row.min() >= 0 and row.max() < small.nKb
         i = r % small.nQb
         assert 2 * i in row
+
+
+# ----------------------------------------------------------------------------- scale producer, branch drop
+
+def test_dynamic_scale_pins():
+    rng = np.random.default_rng(31)
+    B, N, D = 3, 257, 96
+    x = bf16_round(rng.standard_normal((B, N, D)))
+    w = bf16_round(rng.standard_normal(D) * 0.2)
+    s = orc.dynamic_scale(x, w, bias=0.3)
+    z = np.einsum("bnd,d->bn", x.astype(np.float64), w.astype(np.float64)) + 0.3
+    ref = torch.sigmoid(torch.from_numpy(z)).mean(dim=1).numpy()          # library sigmoid as witness
+    np.testing.assert_allclose(s, ref, rtol=1e-12)
+    assert ((s > 0) & (s < 1)).all()                                       # the paper's s in (0, 1)
+    # closed forms: w = 0 -> sigmoid(bias); x -> -x with zero bias -> 1 - s
+    np.testing.assert_allclose(orc.dynamic_scale(x, np.zeros(D), bias=0.0), 0.5, rtol=1e-15)
+    np.testing.assert_allclose(orc.dynamic_scale(x, np.zeros(D), bias=2.0), 1 / (1 + np.exp(-2.0)), rtol=1e-14)
+    np.testing.assert_allclose(orc.dynamic_scale(-x, w) + orc.dynamic_scale(x, w), 1.0, rtol=1e-13)
+    # a mean over tokens, per batch item: permuting tokens changes nothing, batch items are independent
+    perm = rng.permutation(N)
+    np.testing.assert_allclose(orc.dynamic_scale(x[:, perm], w), orc.dynamic_scale(x, w), rtol=1e-13)
+    np.testing.assert_allclose(orc.dynamic_scale(x[1:2], w, 0.3), s[1:2], rtol=1e-15)
+
+
+def test_fused_branch_drop_pins():
+    B, H, N, d = 3, 2, 128, 32
+    q, k, v = rand_qkv(B, H, N, d, 41)
+    rp, ci = wlmod.dense_csr(2, 2, 1)
+    lam = np.array([0.7, 0.2]); s = np.array([0.10, 0.50, 0.90])
+    full = orc.salad_fused(q, k, v, 64, 64, rp, ci, 1, lam, s).reshape(B, H, N, d)
+    sparse = orc.sparse_attn(q, k, v, 64, 64, rp, ci, 1)[0].reshape(B, H, N, d)
+    drop = orc.salad_fused_drop(q, k, v, 64, 64, rp, ci, 1, lam, s, tau=0.5).reshape(B, H, N, d)
+    np.testing.assert_array_equal(drop[0], sparse[0])          # s < tau: exactly the sparse branch
+    np.testing.assert_array_equal(drop[1], full[1])            # s == tau is kept ("below" is dropped)
+    np.testing.assert_array_equal(drop[2], full[2])
+    np.testing.assert_array_equal(orc.salad_fused_drop(q, k, v, 64, 64, rp, ci, 1, lam, s, tau=-1.0).reshape(B, H, N, d), full)
+    np.testing.assert_array_equal(orc.salad_fused_drop(q, k, v, 64, 64, rp, ci, 1, lam, s, tau=2.0).reshape(B, H, N, d), sparse)
