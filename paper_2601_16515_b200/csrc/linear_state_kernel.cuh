@@ -194,22 +194,21 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 //   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
 //           num = ReLU(Q) KV in the fused kernel.
 template <int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
                              __nv_bfloat16* __restrict__ kvt)
 {
-    // grid (D/32, D/32, BH), block (32, 8): one 32 x 32 tile of KV per block, transposed through
-    // shared memory so that both the partial reads and the bf16 writes are coalesced
+    // grid (D/32, D/32, BH), block (32, 32): one 32 x 32 tile of KV per block, one element per
+    // thread, transposed through shared memory so that both the partial reads and the bf16
+    // writes are coalesced
     __shared__ float tile[32][33];
     const int bh = blockIdx.z;
     const int a0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
     const int tx = threadIdx.x, ty = threadIdx.y;
-    const size_t head = size_t(bh) * chunks * D * D;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int a = a0 + ty + 8 * j;
-        const float* src = kv_part + head + size_t(a) * D + c0 + tx;
+    {
+        const int a = a0 + ty;
+        const float* src = kv_part + size_t(bh) * chunks * D * D + size_t(a) * D + c0 + tx;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
         int ch = 0;
         for (; ch + 4 <= chunks; ch += 4) {           // fixed order: ((p0+p4+..)+(p1+p5+..))+...
@@ -221,16 +220,12 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
         for (; ch < chunks; ++ch) s0 += src[size_t(ch) * D * D];
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
-        tile[ty + 8 * j][tx] = s;
+        tile[ty][tx] = s;
     }
     __syncthreads();
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int c = c0 + ty + 8 * j;
-        kvt[size_t(bh) * D * D + size_t(c) * D + a0 + tx] = __float2bfloat16(tile[tx][ty + 8 * j]);
-    }
+    kvt[size_t(bh) * D * D + size_t(c0 + ty) * D + a0 + tx] = __float2bfloat16(tile[tx][ty]);
     if (blockIdx.x == 0 && blockIdx.y == 0) {
-        for (int a = ty * 32 + tx; a < D; a += 256) {
+        for (int a = ty * 32 + tx; a < D; a += 1024) {
             const float* src = z_part + size_t(bh) * chunks * D + a;
             float s = 0.f;
             for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];

@@ -101,8 +101,15 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
 // blocks sorted by decreasing cost (the longer of the two kept lists), so that the long items
 // start first and the short ones fill the tail.  Counting sort in shared memory; one CTA per
 // mask head.  The order among equal costs is arbitrary (it only affects scheduling).
+// It is the first kernel of a call, so it also clears the status words the later kernels test.
 __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
-                                                          int nPairs, int32_t* __restrict__ order) {
+                                                          int nPairs, int32_t* __restrict__ order,
+                                                          int32_t* __restrict__ ws_status,
+                                                          int32_t* __restrict__ user_status) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *ws_status = 0;
+        if (user_status) *user_status = 0;
+    }
     constexpr int BINS = 2048;
     __shared__ int hist[BINS];
     const int hm = blockIdx.x, tid = threadIdx.x;
@@ -116,10 +123,21 @@ __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restr
     __syncthreads();
     for (int pr = tid; pr < nPairs; pr += blockDim.x) atomicAdd(&hist[cost_of(pr)], 1);
     __syncthreads();
-    if (tid == 0) {                       // start position of every cost, largest cost first
-        int run = 0;
-        for (int c = BINS - 1; c >= 0; --c) { const int n = hist[c]; hist[c] = run; run += n; }
+    // start position of every cost, largest cost first: an exclusive suffix sum over the bins,
+    // two bins per thread, Hillis-Steele over the per-thread totals
+    __shared__ int part[1024];
+    const int h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+    part[tid] = h0 + h1;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        const int add = (tid + off < 1024) ? part[tid + off] : 0;
+        __syncthreads();
+        part[tid] += add;
+        __syncthreads();
     }
+    const int above = part[tid] - (h0 + h1);      // items with a cost in a higher pair of bins
+    hist[2 * tid + 1] = above;
+    hist[2 * tid] = above + h1;
     __syncthreads();
     for (int pr = tid; pr < nPairs; pr += blockDim.x)
         order[size_t(hm) * nPairs + atomicAdd(&hist[cost_of(pr)], 1)] = pr;

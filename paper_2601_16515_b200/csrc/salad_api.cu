@@ -150,7 +150,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     record_profile(0, P.stream);
     salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    salad_linear_finalize_kernel<D><<<dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream>>>(
+    salad_linear_finalize_kernel<D><<<dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream>>>(
         sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
         reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt));
     record_profile(1, P.stream);
@@ -174,13 +174,7 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
     fp.BH = BH;
     fp.order = nullptr;
-    if (P.mode & MODE_SPARSE) {
-        // longest work items first (the mask is an input of every call, so is its order)
-        int32_t* order = reinterpret_cast<int32_t*>(ws + w.off_order);
-        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, fp.nQb, fp.nPairs, order);
-        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-        fp.order = order;
-    }
+    if (P.mode & MODE_SPARSE) fp.order = reinterpret_cast<const int32_t*>(ws + w.off_order);   // written by run()
     fp.static_scale = P.static_scale; fp.dyn_scale = P.dyn_scale;
     fp.z = reinterpret_cast<const float*>(ws + w.off_z);
     fp.lse = P.lse;
@@ -206,10 +200,20 @@ int run(const Problem& P) {
     if (rc != SALAD_OK) return rc;
     const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
-    if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
-    if (P.d_status && cudaMemsetAsync(P.d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
-        cudaGetLastError();
-        return SALAD_ERR_CUDA;
+    if (P.mode & MODE_SPARSE) {
+        // first kernel of the call: longest work items first (the mask is an input of every call,
+        // so is its order); it also clears the status words
+        const int nQb = (P.N + P.Bq - 1) / P.Bq;
+        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb, (nQb + 1) / 2,
+                                                      reinterpret_cast<int32_t*>(ws + w.off_order),
+                                                      reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
+        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    } else {
+        if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+        if (P.d_status && cudaMemsetAsync(P.d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
+            cudaGetLastError();
+            return SALAD_ERR_CUDA;
+        }
     }
     if (P.mode & MODE_LINEAR) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
