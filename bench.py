@@ -307,6 +307,19 @@ def main():
                                   "frac": kv_bytes / (state_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                   "frac_of_nominal_8tbs": kv_bytes / (state_ms * 1e-3) / 1e9 / 8000.0}
 
+        # dynamic-scale producer (Alg. 1 Level 2) on hidden states of the DiT this workload comes from:
+        # a CFG pair of [N, D = H*d] token matrices (larger than L2), read once
+        xt = torch.randn(2, wl.N, wl.H * wl.d, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        w_dyn = torch.randn(wl.H * wl.d, device=dev, dtype=torch.float32) / (wl.H * wl.d) ** 0.5
+        s_out = torch.empty(2, device=dev, dtype=torch.float32)
+        dyn_ws = torch.empty(salad.DYN_SCALE_WS_BYTES, dtype=torch.uint8, device=dev)
+        dyn_ms = timed(lambda: salad.salad_dynamic_scale(xt, w_dyn, 0.0, out=s_out, workspace=dyn_ws), 20)
+        x_bytes = xt.numel() * 2
+        extras["dynamic_scale"] = {"ms": dyn_ms, "algorithmic_bytes": x_bytes,
+                                   "achieved_gbs": x_bytes / (dyn_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                                   "frac": x_bytes / (dyn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del xt
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline, _ = oracle_sample(wl, 1, 0, rank)
@@ -336,7 +349,7 @@ def main():
                          "kernel_ms": attn_ms, "state_kernels_ms": state_ms},
             "cpu_baseline": cpu_baseline,
             "e2e": e2e,
-            "gpu_launches": 3 * K,
+            "gpu_launches": 4 * K,      # per call: work order, linear state, state finalize, attention
             "clocks": sampler.result(),
         }
         line.update(extras)

@@ -123,6 +123,37 @@ int salad_fused_fwd(const void* q, const void* k, const void* v, void* o,
                     int32_t* d_status, void* stream);
 
 /*
+ * salad_fused_drop_fwd -- salad_fused_fwd with post-tuning branch dropping (Sec. 4.3, Appendix
+ * A.3): the linear branch of batch item b is skipped when its scaling factor is below the
+ * threshold,
+ *     O[b,h,n] = O_s[b,h,n] + [d_dyn_scale[b] >= drop_tau] * d_dyn_scale[b] * d_static_scale[h] * O_l[b,h,n].
+ * The comparison happens on the device (the scale is produced there), so there is no host
+ * synchronisation: the linear-state kernels of a dropped batch item return at once and the
+ * attention kernel does no linear work for it; its output equals salad_sparse_attn_fwd bit
+ * for bit.  drop_tau is the calibrated per-timestep threshold tau_t (a host float).
+ */
+int salad_fused_drop_fwd(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int N, int d, int Bq, int Bk,
+                         const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                         const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                         float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                         int32_t* d_status, void* stream);
+
+/*
+ * salad_dynamic_scale -- the input- and timestep-aware scaling factor of Algorithm 1, Level 2
+ * (Sec. 4.2): a D -> 1 linear layer on the modulated hidden states, a sigmoid, a token average:
+ *     s[b] = (1/N) sum_n sigmoid( <x[b,n,:], w> + bias ),   s in (0, 1).
+ *   x          bf16 [B, N, D], contiguous, 16-byte aligned; D a multiple of 8, D <= 8192.
+ *   w          fp32 [D] (device).   bias: the paper counts D x 1 weights only; pass 0 for none.
+ *   s_out      fp32 [B] (device), written; it can be passed on as d_dyn_scale.
+ *   workspace  at least SALAD_DYN_SCALE_WS_BYTES bytes of device memory, 256-byte aligned.
+ * HBM-bound (x is read once); the result is deterministic.  B <= 2048.
+ */
+#define SALAD_DYN_SCALE_WS_BYTES 8192
+int salad_dynamic_scale(const void* x, const float* w, float bias, int B, int N, int D,
+                        float* s_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide
  * scratch memory (the paper has no counterpart; this is a deployment convenience).
  * Some hosts of this library may not call cudaMalloc at the point where attention runs: a

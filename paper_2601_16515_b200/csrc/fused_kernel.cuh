@@ -59,6 +59,7 @@ struct FusedParams {
     float* lse;                  // optional [B*H, N]
     float scale_log2;            // softmax_scale * log2(e)
     float eps;
+    float drop_tau;              // linear branch of batch item b skipped when dyn_scale[b] < drop_tau
     int32_t* ws_status;          // library status word (never null)
     int32_t* user_status;        // optional
 };
@@ -134,7 +135,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int h = bh % p.H, b = bh / p.H;
     const int hm = (p.Hm == 1) ? 0 : h;
     const int pair = p.order ? __ldg(p.order + size_t(hm) * p.nPairs + rank) : rank;
-    const bool sparse = (p.mode & MODE_SPARSE) != 0, linear = (p.mode & MODE_LINEAR) != 0;
+    const bool sparse = (p.mode & MODE_SPARSE) != 0;
+    // post-tuning branch dropping (Sec. 4.3): no linear work at all for a dropped batch item
+    const bool linear = (p.mode & MODE_LINEAR) != 0 &&
+                        !(p.dyn_scale != nullptr && __ldg(p.dyn_scale + b) < p.drop_tau);
 
     // kept lists of the two tiles
     int qb[2], ls[2], le[2];
@@ -202,6 +206,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 prefetch_tmap(&map_q); prefetch_tmap(&map_k);
                 for (int i = 0; i < 2; ++i) {
                     if (qb[i] >= p.nQb) continue;
+                    // A tile with no kept block and no linear branch never reads Q: its epilogue
+                    // stages zeros in the Q tile without waiting for q_full, so nothing may land there.
+                    if (le[i] == ls[i] && !linear) continue;
                     const uint32_t bar = smem_u32(&bars.q_full[i]);
                     mbar_arrive_expect_tx(bar, uint32_t(p.Bq) * D * 2);
                     for (int ch = 0; ch < C::CH; ++ch)

@@ -42,7 +42,16 @@ struct StateParams {
     float* z_part;        // [BH][chunks][D]
     int32_t* ws_status;
     int32_t* user_status;
+    const float* dyn_scale;   // [B] or null: with drop_tau, batch items whose scale is below it are skipped
+    float drop_tau;
+    int H;
 };
+
+// Post-tuning branch dropping (Sec. 4.3): the linear branch of a batch item is skipped when its
+// dynamic scale is below the threshold.  Decided on the device, so no host synchronisation.
+__device__ __forceinline__ bool branch_dropped(const float* dyn_scale, float tau, int b) {
+    return dyn_scale != nullptr && __ldg(dyn_scale + b) < tau;
+}
 
 template <int D>
 __global__ void __launch_bounds__(192)
@@ -59,6 +68,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x, bh = blockIdx.y;
+    if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) return;     // whole CTA, before any allocation
     const int kb0 = chunk * p.blocks_per_chunk;
     const int kb1 = min(p.nKb, kb0 + p.blocks_per_chunk);
     const int nblk = max(0, kb1 - kb0);
@@ -197,8 +207,9 @@ template <int D>
 __global__ void __launch_bounds__(1024)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
-                             __nv_bfloat16* __restrict__ kvt)
+                             __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
+    if (branch_dropped(dyn_scale, drop_tau, blockIdx.z / H)) return;
     // grid (D/32, D/32, BH), block (32, 32): one 32 x 32 tile of KV per block, one element per
     // thread, transposed through shared memory so that both the partial reads and the bf16
     // writes are coalesced

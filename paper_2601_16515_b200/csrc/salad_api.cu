@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 
+#include "dynamic_scale_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "linear_state_kernel.cuh"
 #include "mask_kernels.cuh"
@@ -102,7 +103,7 @@ struct Problem {
     int B, H, N, d, Bq, Bk, Hm, mode;
     const int32_t *row_ptr, *col_idx;
     const float *static_scale, *dyn_scale;
-    float softmax_scale, eps;
+    float softmax_scale, eps, drop_tau;
     float *kv_out, *z_out;
     void* ws; size_t ws_bytes; int32_t* d_status; cudaStream_t stream;
 };
@@ -147,12 +148,13 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.z_part = reinterpret_cast<float*>(ws + w.off_zp);
     sp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     sp.user_status = P.d_status;
+    sp.dyn_scale = P.dyn_scale; sp.drop_tau = P.drop_tau; sp.H = P.H;
     record_profile(0, P.stream);
     salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     salad_linear_finalize_kernel<D><<<dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream>>>(
         sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
-        reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt));
+        reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt), P.dyn_scale, P.drop_tau, P.H);
     record_profile(1, P.stream);
     return check_launch();
 }
@@ -181,6 +183,7 @@ int launch_fused(const Problem& P, const Workspace& w) {
     const float sc = (P.softmax_scale > 0.f) ? P.softmax_scale : 1.0f / sqrtf(float(D));
     fp.scale_log2 = sc * 1.4426950408889634f;
     fp.eps = P.eps;
+    fp.drop_tau = P.drop_tau;
     fp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     fp.user_status = P.d_status;
     const int64_t grid = int64_t(fp.nPairs) * BH;
@@ -347,6 +350,7 @@ SALAD_EXPORT int salad_sparse_attn_fwd(const void* q, const void* k, const void*
                                        float softmax_scale, void* workspace, size_t workspace_bytes,
                                        int32_t* d_status, void* stream) {
     Problem P{};
+    P.drop_tau = -INFINITY;
     P.q = q; P.k = k; P.v = v; P.o = o; P.lse = lse;
     P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_SPARSE;
     P.row_ptr = row_ptr; P.col_idx = col_idx;
@@ -361,9 +365,28 @@ SALAD_EXPORT int salad_linear_attn_fwd(const void* q, const void* k, const void*
                                        void* workspace, size_t workspace_bytes, int32_t* d_status,
                                        void* stream) {
     Problem P{};
+    P.drop_tau = -INFINITY;
     P.q = q; P.k = k; P.v = v; P.o = o_l;
     P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
     P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_fused_drop_fwd(const void* q, const void* k, const void* v, void* o,
+                                      int B, int H, int N, int d, int Bq, int Bk,
+                                      const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                      const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                                      float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                                      int32_t* d_status, void* stream) {
+    if (isnan(drop_tau)) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
+    P.softmax_scale = softmax_scale; P.eps = eps;
     P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
     P.stream = static_cast<cudaStream_t>(stream);
     return run(P);
@@ -375,15 +398,34 @@ SALAD_EXPORT int salad_fused_fwd(const void* q, const void* k, const void* v, vo
                                  const float* d_static_scale, const float* d_dyn_scale,
                                  float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
                                  int32_t* d_status, void* stream) {
-    Problem P{};
-    P.q = q; P.k = k; P.v = v; P.o = o;
-    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
-    P.row_ptr = row_ptr; P.col_idx = col_idx;
-    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale;
-    P.softmax_scale = softmax_scale; P.eps = eps;
-    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
-    P.stream = static_cast<cudaStream_t>(stream);
-    return run(P);
+    // no threshold: every branch is kept, whatever the value of its scale
+    return salad_fused_drop_fwd(q, k, v, o, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, d_static_scale, d_dyn_scale,
+                                -INFINITY, softmax_scale, eps, workspace, workspace_bytes, d_status, stream);
+}
+
+SALAD_EXPORT int salad_dynamic_scale(const void* x, const float* w, float bias, int B, int N, int D,
+                                     float* s_out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!x || !w || !s_out || B <= 0 || N <= 0 || D <= 0 || !isfinite(bias)) return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(x)) return SALAD_ERR_INVALID_ARG;
+    if (D % 8 != 0 || D > 8192 || B > 2048) return SALAD_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 ||
+        workspace_bytes < SALAD_DYN_SCALE_WS_BYTES)
+        return SALAD_ERR_WORKSPACE;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int slots = SALAD_DYN_SCALE_WS_BYTES / 4;
+    int G = (8 * dev.sms) / B;                       // about eight CTAs per SM in flight
+    if (G > slots / B) G = slots / B;
+    if (G > (N + 7) / 8) G = (N + 7) / 8;            // at least one token per warp
+    if (G < 1) G = 1;
+    float* partial = static_cast<float*>(workspace);
+    dynamic_scale_partial_kernel<<<dim3(G, B), kDynScaleThreads, size_t(D) * 4, st>>>(
+        static_cast<const uint4*>(x), w, bias, N, D, partial);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    dynamic_scale_finalize_kernel<<<B, 32, 0, st>>>(partial, G, N, s_out);
+    return check_launch();
 }
 
 SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o_l,
@@ -405,6 +447,7 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     if (w.total > kNoAllocBytes) return SALAD_ERR_UNSUPPORTED;
 
     Problem P{};
+    P.drop_tau = -INFINITY;
     P.q = q; P.k = k; P.v = v; P.o = o_l;
     P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
     P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;

@@ -26,7 +26,8 @@ SALAD_ERR_TIMEOUT = -6
 
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
-           "salad_set_profile_events", "salad_linear_attn_fwd_noalloc")
+           "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
+           "salad_dynamic_scale")
 
 
 class SaladError(RuntimeError):
@@ -56,6 +57,10 @@ def _load() -> ctypes.CDLL:
     lib.salad_fused_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, p, sz, p, p]
     lib.salad_linear_attn_fwd_noalloc.restype = i32
     lib.salad_linear_attn_fwd_noalloc.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [f32, p, p]
+    lib.salad_fused_drop_fwd.restype = i32
+    lib.salad_fused_drop_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, f32, p, sz, p, p]
+    lib.salad_dynamic_scale.restype = i32
+    lib.salad_dynamic_scale.argtypes = [p, p, f32, i32, i32, i32, p, p, sz, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -201,10 +206,31 @@ def salad_linear_attn_fwd_noalloc(q, k, v, eps: float = 1e-6, out=None, kv_out=N
     return out
 
 
+DYN_SCALE_WS_BYTES = 8192
+
+
+def salad_dynamic_scale(x, w, bias: float = 0.0, out=None, workspace=None, stream=None):
+    """s[b] = mean over tokens of sigmoid(<x[b,n,:], w> + bias).  x bf16 [B,N,D], w fp32 [D] -> fp32 [B]."""
+    if x.dtype != torch.bfloat16 or x.dim() != 3 or not x.is_contiguous() or not x.is_cuda:
+        raise ValueError("x must be a contiguous CUDA bf16 tensor [B, N, D]")
+    B, N, D = x.shape
+    if w.dtype != torch.float32 or not w.is_cuda or w.numel() != D or not w.is_contiguous():
+        raise ValueError("w must be a contiguous CUDA fp32 tensor with D elements")
+    if out is None:
+        out = torch.empty(B, dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(DYN_SCALE_WS_BYTES, dtype=torch.uint8, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(_lib.salad_dynamic_scale(_ptr(x), _ptr(w), float(bias), B, N, D, _ptr(out), _ptr(workspace),
+                                        workspace.numel(), _stream(stream)), "salad_dynamic_scale")
+    return out
+
+
 def salad_fused_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_scale, Bq: int = 128,
                     Bk: int = 64, softmax_scale: float = 0.0, eps: float = 1e-6, out=None,
-                    workspace=None, status=None, stream=None):
-    """O = O_sparse + dyn_scale[b] * static_scale[h] * O_linear, one bf16 write."""
+                    workspace=None, status=None, stream=None, drop_tau: Optional[float] = None):
+    """O = O_sparse + dyn_scale[b] * static_scale[h] * O_linear, one bf16 write.  With `drop_tau`
+    the linear branch of batch items whose dyn_scale is below it is skipped (salad_fused_drop_fwd)."""
     B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
     _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
     for name, t, n in (("static_scale", static_scale, H), ("dyn_scale", dyn_scale, B)):
@@ -213,8 +239,15 @@ def salad_fused_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_scale,
     if out is None:
         out = torch.empty_like(q)
     with torch.cuda.device(q.device):
-        _check(_lib.salad_fused_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
-                                    _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale),
-                                    float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
-                                    _ptr(status), _stream(stream)), "salad_fused_fwd")
+        if drop_tau is None:
+            _check(_lib.salad_fused_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                        _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale),
+                                        float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
+                                        _ptr(status), _stream(stream)), "salad_fused_fwd")
+        else:
+            _check(_lib.salad_fused_drop_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                             _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale),
+                                             float(drop_tau), float(softmax_scale), float(eps), _ptr(workspace),
+                                             workspace.numel(), _ptr(status), _stream(stream)),
+                   "salad_fused_drop_fwd")
     return out

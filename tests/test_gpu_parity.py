@@ -142,6 +142,31 @@ def test_sparse_random_lists(salad, B, H, N, d, Bq, Hm):
     np.testing.assert_allclose(got_lse[~empty], ref_lse[~empty], atol=2e-3, rtol=1e-4)
 
 
+def test_sparse_empty_rows_write_exact_zeros(salad):
+    # Query blocks with no kept key block: Eq. 2 sums over nothing, the output row is exactly zero.
+    # Half of the rows are empty, the others keep everything; repeated, on a buffer prefilled with
+    # ones, so that a query tile landing in the staging buffer late would show up.
+    B, H, N, d, Bq = 2, 3, 1000, 128, 128
+    q, k, v = rand_qkv(B, H, N, d, 31)
+    nQb, nKb = -(-N // Bq), -(-N // 64)
+    lens = np.array([nKb if (r % 3 == 1) else 0 for r in range(H * nQb)], dtype=np.int32)
+    rp = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ci = np.concatenate([np.arange(n, dtype=np.int32) for n in lens if n] or [np.zeros(0, np.int32)])
+    rp_d, ci_d = dev_csr(rp, ci)
+    ref, _ = orc.sparse_attn(f32(q), f32(k), f32(v), Bq, 64, rp, ci, H)
+    ref = ref.reshape(B, H, N, d)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    for _ in range(5):
+        out = torch.ones_like(qd)
+        salad.salad_sparse_attn_fwd(qd, kd, vd, rp_d, ci_d, H, Bq=Bq, out=out)
+        got = f32(out.cpu()).reshape(B, H, N, d)
+        for h in range(H):
+            for i in range(nQb):
+                if lens[h * nQb + i] == 0:
+                    assert not got[:, h, i * Bq:(i + 1) * Bq].any(), (h, i)
+        assert_close(got.reshape(-1, d), ref.reshape(-1, d), "half-empty")
+
+
 def test_sparse_all_kept_is_full_attention(salad):
     B, H, N, d = 1, 2, 1000, 128
     q, k, v = rand_qkv(B, H, N, d, 5)
@@ -341,3 +366,58 @@ def test_binding_rejects_bad_tensors(salad):
     with pytest.raises(salad.SaladError) as err:
         salad.salad_sparse_attn_fwd(q, k, v, rp, ci, 1, workspace=small)
     assert err.value.code == salad.SALAD_ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------------------ scale producer, branch drop
+
+@pytest.mark.parametrize("B,N,D", [(2, 1000, 96), (3, 7, 8), (1, 32760, 1536), (2, 4099, 5120)])
+def test_dynamic_scale(salad, B, N, D):
+    rng = np.random.default_rng(B * 1000 + D)
+    x = bf16(rng.standard_normal((B, N, D)))
+    w = (rng.standard_normal(D) * (2.0 / np.sqrt(D))).astype(np.float32)
+    got = salad.salad_dynamic_scale(x.cuda(), torch.from_numpy(w).cuda(), bias=-0.2)
+    ref = orc.dynamic_scale(f32(x), w, bias=-0.2)
+    # fp32 dot products of D terms and a fast exp: a few 1e-6 on a value in (0, 1)
+    np.testing.assert_allclose(got.cpu().numpy(), ref, rtol=0, atol=2e-5)
+    again = salad.salad_dynamic_scale(x.cuda(), torch.from_numpy(w).cuda(), bias=-0.2)
+    assert torch.equal(got, again)                       # fixed reduction order
+
+
+def test_fused_branch_drop(salad):
+    B, H, N, d = 3, 2, 1100, 128
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), 128, 64, (), 1)
+    q, k, v = rand_qkv(B, H, N, d, 91)
+    rp, ci = random_csr(wl.nQb, wl.nKb, 3, lo=1, hi=wl.nKb)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = np.array([0.7, 0.2], np.float32); s = np.array([0.10, 0.50, 0.90], np.float32)
+    lam_d, s_d = torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda()
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    drop = salad.salad_fused_fwd(qd, kd, vd, rp_d, ci_d, 1, lam_d, s_d, drop_tau=0.5, status=status)
+    status_ok(status)
+    ref = orc.salad_fused_drop(f32(q), f32(k), f32(v), 128, 64, rp, ci, 1, lam, s, tau=0.5)
+    assert_close(f32(drop.cpu()).reshape(-1, d), ref, "drop")
+    sparse = salad.salad_sparse_attn_fwd(qd, kd, vd, rp_d, ci_d, 1)
+    full = salad.salad_fused_fwd(qd, kd, vd, rp_d, ci_d, 1, lam_d, s_d)
+    assert torch.equal(drop[0], sparse[0])               # below the threshold: the sparse branch, bit for bit
+    assert torch.equal(drop[1:], full[1:])               # at or above it: unchanged
+    none = salad.salad_fused_fwd(qd, kd, vd, rp_d, ci_d, 1, lam_d, s_d, drop_tau=2.0)
+    assert torch.equal(none, sparse)
+
+
+def test_scale_producer_feeds_the_fused_call(salad):
+    # s computed on the device by salad_dynamic_scale goes straight into the attention call
+    B, H, N, d, D = 2, 2, 640, 64, 128
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), 64, 64, (), 1)
+    q, k, v = rand_qkv(B, H, N, d, 17)
+    rng = np.random.default_rng(2)
+    x = bf16(rng.standard_normal((B, N, D)))
+    w = (rng.standard_normal(D) * 0.3).astype(np.float32)
+    rp, ci = random_csr(wl.nQb, wl.nKb, 8, lo=1, hi=wl.nKb)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = np.array([0.4, 0.8], np.float32)
+    s_d = salad.salad_dynamic_scale(x.cuda(), torch.from_numpy(w).cuda())
+    out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, torch.from_numpy(lam).cuda(), s_d, Bq=64)
+    s_ref = orc.dynamic_scale(f32(x), w)
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), 64, 64, rp, ci, 1, lam, s_ref)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "chain")
