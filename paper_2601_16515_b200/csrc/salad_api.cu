@@ -416,7 +416,14 @@ SALAD_EXPORT int salad_dynamic_scale(const void* x, const float* w, float bias, 
     if (rc != SALAD_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int slots = SALAD_DYN_SCALE_WS_BYTES / 4;
-    int G = (8 * dev.sms) / B;                       // about eight CTAs per SM in flight
+    // one wave: as many CTAs as the device holds at once, split over the batch items
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dynamic_scale_partial_kernel, kDynScaleThreads,
+                                                      size_t(D) * 4) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        return SALAD_ERR_CUDA;
+    }
+    int G = (per_sm * dev.sms) / B;
     if (G > slots / B) G = slots / B;
     if (G > (N + 7) / 8) G = (N + 7) / 8;            // at least one token per warp
     if (G < 1) G = 1;
