@@ -8,6 +8,7 @@
 
 #include "dynamic_scale_kernel.cuh"
 #include "fused_kernel.cuh"
+#include "linear_apply_kernel.cuh"
 #include "linear_state_kernel.cuh"
 #include "mask_kernels.cuh"
 #include "tmap.cuh"
@@ -85,6 +86,12 @@ int prepare_device(DeviceInfo* info) {
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_linear_state_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      StateCfg<64>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<128>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<64>::SMEM_BYTES);
         if (e != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
         sm_count[dev] = sms;
         attr_set[dev] = true;
@@ -195,6 +202,31 @@ int launch_fused(const Problem& P, const Workspace& w) {
     return check_launch();
 }
 
+// Linear-only calls: the stand-alone apply kernel, one persistent CTA per SM.
+template <int D>
+int launch_apply(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
+    const int BH = P.B * P.H;
+    uint8_t* ws = static_cast<uint8_t*>(P.ws);
+    CUtensorMap mq, mo, ms;
+    if (!make_tmap_bf16_3d(&mq, P.q, D, P.N, BH, 128) || !make_tmap_bf16_3d(&mo, P.o, D, P.N, BH, 128) ||
+        !make_tmap_bf16_3d(&ms, ws + w.off_kvt, D, D, BH, D))
+        return SALAD_ERR_CUDA;
+    ApplyParams ap;
+    ap.N = P.N; ap.H = P.H;
+    ap.nQb = (P.N + 127) / 128;
+    ap.tiles = (long long)ap.nQb * BH;
+    ap.z = reinterpret_cast<const float*>(ws + w.off_z);
+    ap.static_scale = P.static_scale; ap.dyn_scale = P.dyn_scale;
+    ap.eps = P.eps;
+    ap.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    ap.user_status = P.d_status;
+    const unsigned grid = unsigned(ap.tiles < dev.sms ? ap.tiles : dev.sms);
+    record_profile(2, P.stream);
+    salad_linear_apply_kernel<D><<<grid, ApplyCfg<D>::THREADS, ApplyCfg<D>::SMEM_BYTES, P.stream>>>(mq, ms, mo, ap);
+    record_profile(3, P.stream);
+    return check_launch();
+}
+
 int run(const Problem& P) {
     int rc = validate(P);
     if (rc != SALAD_OK) return rc;
@@ -222,6 +254,7 @@ int run(const Problem& P) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
         if (rc != SALAD_OK) return rc;
     }
+    if (P.mode == MODE_LINEAR) return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
     return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }
 
