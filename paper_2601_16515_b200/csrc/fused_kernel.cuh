@@ -128,6 +128,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    grid_dependency_wait();           // the order and the linear state come from the kernels before
+    grid_launch_dependents();
 
     // work item: head by head (K/V of one head stay hot in L2), within a head the pairs of query
     // blocks from the most to the least expensive, so that the kernel ends on short items

@@ -73,6 +73,8 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     // contiguous, balanced range of tiles (head-major, so the state changes rarely)
     const long long t0 = p.tiles * blockIdx.x / gridDim.x, t1 = p.tiles * (blockIdx.x + 1) / gridDim.x;
 
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (tid == 0) {
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int s = 0; s < C::NQ; ++s) {

@@ -68,6 +68,8 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x, bh = blockIdx.y;
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) return;     // whole CTA, before any allocation
     const int kb0 = chunk * p.blocks_per_chunk;
     const int kb1 = min(p.nKb, kb0 + p.blocks_per_chunk);
@@ -209,6 +211,8 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
                              __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (branch_dropped(dyn_scale, drop_tau, blockIdx.z / H)) return;
     // grid (D/32, D/32, BH), block (32, 32): one 32 x 32 tile of KV per block, one element per
     // thread, transposed through shared memory so that both the partial reads and the bf16

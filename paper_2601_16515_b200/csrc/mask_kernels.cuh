@@ -11,6 +11,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace salad {
 
 struct MaskGeom {
@@ -106,6 +108,7 @@ __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restr
                                                           int nPairs, int32_t* __restrict__ order,
                                                           int32_t* __restrict__ ws_status,
                                                           int32_t* __restrict__ user_status) {
+    grid_launch_dependents();         // the next kernel of the call may be placed now; it waits for this one
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         *ws_status = 0;
         if (user_status) *user_status = 0;

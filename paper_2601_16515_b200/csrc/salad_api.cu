@@ -101,6 +101,22 @@ int prepare_device(DeviceInfo* info) {
     return SALAD_OK;
 }
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may be set up and its CTAs
+// placed while the kernel before it in the stream drains.  Every kernel launched this way starts with
+// grid_dependency_wait(), so stream order is kept; only the launch latency between the kernels of a
+// call goes away.
+template <typename... KArgs, typename... Args>
+void launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                      Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);     // errors are read by check_launch()
+}
+
 int check_launch() {
     return cudaGetLastError() == cudaSuccess ? SALAD_OK : SALAD_ERR_CUDA;
 }
@@ -157,11 +173,12 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.user_status = P.d_status;
     sp.dyn_scale = P.dyn_scale; sp.drop_tau = P.drop_tau; sp.H = P.H;
     record_profile(0, P.stream);
-    salad_linear_state_kernel<D><<<dim3(chunks, BH), StateCfg<D>::THREADS, StateCfg<D>::SMEM_BYTES, P.stream>>>(mk, mv, sp);
+    launch_dependent(salad_linear_state_kernel<D>, dim3(chunks, BH), dim3(StateCfg<D>::THREADS),
+                     StateCfg<D>::SMEM_BYTES, P.stream, mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    salad_linear_finalize_kernel<D><<<dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream>>>(
-        sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
-        reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt), P.dyn_scale, P.drop_tau, P.H);
+    launch_dependent(salad_linear_finalize_kernel<D>, dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream,
+                     sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
+                     reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt), P.dyn_scale, P.drop_tau, P.H);
     record_profile(1, P.stream);
     return check_launch();
 }
@@ -196,8 +213,8 @@ int launch_fused(const Problem& P, const Workspace& w) {
     const int64_t grid = int64_t(fp.nPairs) * BH;
     if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
     record_profile(2, P.stream);
-    salad_fused_kernel<D><<<unsigned(grid), FusedCfg<D>::THREADS, FusedCfg<D>::SMEM_BYTES, P.stream>>>(
-        mq, mk, mv, mo, ms, fp);
+    launch_dependent(salad_fused_kernel<D>, dim3(unsigned(grid)), dim3(FusedCfg<D>::THREADS),
+                     FusedCfg<D>::SMEM_BYTES, P.stream, mq, mk, mv, mo, ms, fp);
     record_profile(3, P.stream);
     return check_launch();
 }
@@ -222,7 +239,8 @@ int launch_apply(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     ap.user_status = P.d_status;
     const unsigned grid = unsigned(ap.tiles < dev.sms ? ap.tiles : dev.sms);
     record_profile(2, P.stream);
-    salad_linear_apply_kernel<D><<<grid, ApplyCfg<D>::THREADS, ApplyCfg<D>::SMEM_BYTES, P.stream>>>(mq, ms, mo, ap);
+    launch_dependent(salad_linear_apply_kernel<D>, dim3(grid), dim3(ApplyCfg<D>::THREADS), ApplyCfg<D>::SMEM_BYTES,
+                     P.stream, mq, ms, mo, ap);
     record_profile(3, P.stream);
     return check_launch();
 }
