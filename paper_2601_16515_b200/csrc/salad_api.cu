@@ -184,7 +184,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
 }
 
 template <int D>
-int launch_fused(const Problem& P, const Workspace& w) {
+int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     const int BH = P.B * P.H;
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
     CUtensorMap mq, mk, mv, mo, ms;
@@ -197,6 +197,12 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.nQb = (P.N + P.Bq - 1) / P.Bq;
     fp.nKb = (P.N + 63) / 64;
     fp.nPairs = (fp.nQb + 1) / 2;
+    {
+        // about two waves of the cheapest items of all heads form the tail of the launch
+        int tail = (2 * dev.sms + BH - 1) / BH;
+        if (tail > fp.nPairs) tail = fp.nPairs;
+        fp.head_major_ranks = (P.mode & MODE_SPARSE) ? fp.nPairs - tail : fp.nPairs;
+    }
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
     fp.BH = BH;
     fp.order = nullptr;
@@ -273,7 +279,7 @@ int run(const Problem& P) {
         if (rc != SALAD_OK) return rc;
     }
     if (P.mode == MODE_LINEAR) return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
-    return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
+    return (P.d == 128) ? launch_fused<128>(P, w, dev) : launch_fused<64>(P, w, dev);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -520,5 +526,5 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     }
     rc = (d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
     if (rc != SALAD_OK) return rc;
-    return (d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
+    return (d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
 }
