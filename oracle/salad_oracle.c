@@ -125,8 +125,10 @@ ORACLE_API void oracle_sparse_attn(const float* q, const float* k, const float* 
             int64_t bh; int n;
             decode_row(sel, s, N, &bh, &n);
             int h = (int)(bh % H);
-            int hm = (Hm == 1) ? 0 : h;
-            int64_t r = (int64_t)hm * nQb + n / Bq;
+            /* one mask for all heads (Hm = 1), one per head (Hm = H), or one per batch item
+             * and head (Hm = B*H: input-dependent masks such as the Top-K selection) */
+            int64_t hm = (Hm == 1) ? 0 : (Hm == H ? h : bh);
+            int64_t r = hm * nQb + n / Bq;
             const float* qn = q + (bh * N + n) * (int64_t)d;
             const float* kb = k + bh * (int64_t)N * d;
             const float* vb = v + bh * (int64_t)N * d;
@@ -291,4 +293,64 @@ ORACLE_API void oracle_salad_fused_drop(const float* q, const float* k, const fl
     oracle_salad_fused(q, k, v, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_eff, scale, eps,
                        sel, nsel, o);
     free(s_eff);
+}
+
+/*
+ * oracle_topk_mask: the dynamic Top-K block mask (Sec. 3, Appendix A.1), per batch item and head:
+ *   Step 1  tokens are partitioned into blocks; the mean of every key block is formed,
+ *               kbar_j = mean_{m in key block j} K_m          (the last block may be short);
+ *   Step 2  similarity of the queries with the key-block means, top k blocks kept.  The attention
+ *           kernel is block-granular on the query side as well, so a query block scores a key
+ *           block with the average of its tokens' similarities,
+ *               s[i][j] = mean_{n in query block i} <Q_n, kbar_j>  ( = <qbar_i, kbar_j> ),
+ *           and keeps the k key blocks with the largest s (a tie goes to the lower block index);
+ *   Step 3  is the block-sparse attention itself (oracle_sparse_attn on the lists built here).
+ * Every row keeps kk = min(topk, nKb) blocks, so row_ptr[r] = r * kk; col_idx
+ * [B*H*nQb][kk] holds each row's blocks in ascending order.  scores (may be NULL) receives
+ * s as [B*H][nQb][nKb] for the tests.
+ */
+ORACLE_API void oracle_topk_mask(const float* q, const float* k, int B, int H, int N, int d,
+                                 int Bq, int Bk, int topk, int32_t* col_idx, double* scores)
+{
+    int nQb = (N + Bq - 1) / Bq, nKb = (N + Bk - 1) / Bk;
+    int kk = topk < nKb ? topk : nKb;
+    int64_t BH = (int64_t)B * H;
+#pragma omp parallel for schedule(static)
+    for (int64_t bh = 0; bh < BH; ++bh) {
+        const float* qb = q + bh * (int64_t)N * d;
+        const float* kb = k + bh * (int64_t)N * d;
+        double* kbar = (double*)calloc((size_t)nKb * d, sizeof(double));
+        double* s = (double*)malloc(sizeof(double) * (size_t)nKb);
+        char* taken = (char*)malloc((size_t)nKb);
+        for (int j = 0; j < nKb; ++j) {                                  /* Step 1 */
+            int m1 = (j + 1) * Bk; if (m1 > N) m1 = N;
+            for (int m = j * Bk; m < m1; ++m)
+                for (int c = 0; c < d; ++c) kbar[(int64_t)j * d + c] += (double)kb[(int64_t)m * d + c];
+            for (int c = 0; c < d; ++c) kbar[(int64_t)j * d + c] /= (double)(m1 - j * Bk);
+        }
+        for (int i = 0; i < nQb; ++i) {                                  /* Step 2 */
+            int n1 = (i + 1) * Bq; if (n1 > N) n1 = N;
+            for (int j = 0; j < nKb; ++j) {
+                double acc = 0.0;
+                for (int n = i * Bq; n < n1; ++n) {
+                    double dot = 0.0;
+                    for (int c = 0; c < d; ++c) dot += (double)qb[(int64_t)n * d + c] * kbar[(int64_t)j * d + c];
+                    acc += dot;
+                }
+                s[j] = acc / (double)(n1 - i * Bq);
+                if (scores) scores[(bh * nQb + i) * (int64_t)nKb + j] = s[j];
+            }
+            memset(taken, 0, (size_t)nKb);
+            for (int t = 0; t < kk; ++t) {                               /* k times: the largest left */
+                int best = -1;
+                for (int j = 0; j < nKb; ++j)
+                    if (!taken[j] && (best < 0 || s[j] > s[best])) best = j;
+                taken[best] = 1;
+            }
+            int32_t* out = col_idx + (bh * nQb + i) * (int64_t)kk;
+            int w = 0;
+            for (int j = 0; j < nKb; ++j) if (taken[j]) out[w++] = j;    /* ascending */
+        }
+        free(kbar); free(s); free(taken);
+    }
 }

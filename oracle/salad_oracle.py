@@ -53,6 +53,8 @@ def _load():
         lib.oracle_salad_fused_drop.restype = None
         lib.oracle_salad_fused_drop.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
                                                                          p, i64, p])
+        lib.oracle_topk_mask.restype = None
+        lib.oracle_topk_mask.argtypes = [p, p] + [i32] * 7 + [p, p]
         _lib = lib
     return _lib
 
@@ -188,3 +190,21 @@ def salad_fused_drop(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, tau, 
     lib.oracle_salad_fused_drop(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
                                 sb.ctypes.data, float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
     return o
+
+
+def topk_mask(q, k, Bq, Bk, topk, return_scores=False):
+    """Dynamic Top-K block mask (Appendix A.1): per (batch, head) and query block the `topk` key blocks
+    whose mean has the largest average similarity with the block's queries.
+    Returns (row_ptr[B*H*nQb+1], col_idx[B*H*nQb*kk]) int32 (Hm = B*H), optionally the fp64 scores."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k)
+    B, H, N, d = q.shape
+    nQb, nKb = -(-N // Bq), -(-N // Bk)
+    kk = min(int(topk), nKb)
+    rows = B * H * nQb
+    col_idx = np.zeros(rows * kk, dtype=np.int32)
+    scores = np.zeros((B * H, nQb, nKb), dtype=np.float64) if return_scores else None
+    lib.oracle_topk_mask(qp, kp, B, H, N, d, Bq, Bk, int(topk), col_idx.ctypes.data,
+                         scores.ctypes.data if return_scores else None)
+    row_ptr = (np.arange(rows + 1, dtype=np.int64) * kk).astype(np.int32)
+    return (row_ptr, col_idx, scores) if return_scores else (row_ptr, col_idx)

@@ -1,6 +1,8 @@
 """Pins of the CPU oracle against things other than itself: the equations written out as
 dense N x N matrices in numpy, torch's SDPA routine, closed forms and hand-counted masks.
 CPU only."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -341,3 +343,93 @@ def test_fused_branch_drop_pins():
     np.testing.assert_array_equal(drop[2], full[2])
     np.testing.assert_array_equal(orc.salad_fused_drop(q, k, v, 64, 64, rp, ci, 1, lam, s, tau=-1.0).reshape(B, H, N, d), full)
     np.testing.assert_array_equal(orc.salad_fused_drop(q, k, v, 64, 64, rp, ci, 1, lam, s, tau=2.0).reshape(B, H, N, d), sparse)
+
+
+# ----------------------------------------------------------------------------- Top-K block mask
+
+def _golden(name):
+    out = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", name)):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *vals = line.split()
+        out[key] = np.array([float(v) for v in vals])
+    return out
+
+
+def test_topk_mask_hand_example():
+    g = _golden("topk_hand_example.txt")
+    q = g["Q"].reshape(1, 1, 6, 1)
+    for kname in ("K", "K2"):
+        k = g[kname].reshape(1, 1, 6, 1)
+        rp, ci, sc = orc.topk_mask(q, k, 2, 2, 2, return_scores=True)
+        assert rp.tolist() == [0, 2, 4, 6]
+        assert ci.tolist() == g["TOP2_" + kname].astype(int).tolist()
+        assert orc.topk_mask(q, k, 2, 2, 1)[1].tolist() == g["TOP1_" + kname].astype(int).tolist()
+        if kname == "K":
+            np.testing.assert_allclose(sc.reshape(-1), g["SCORES_K"], rtol=0, atol=1e-15)
+
+
+def test_topk_mask_matches_per_token_brute_force():
+    # Step 2 taken literally: every query token's similarity with the key-block means, averaged
+    # over the tokens of the query block, then argsort.  Ragged last blocks on both sides.
+    rng = np.random.default_rng(77)
+    B, H, N, d, Bq, Bk, topk = 2, 3, 150, 16, 32, 16, 3
+    q = bf16_round(rng.standard_normal((B, H, N, d))); k = bf16_round(rng.standard_normal((B, H, N, d)))
+    rp, ci, sc = orc.topk_mask(q, k, Bq, Bk, topk, return_scores=True)
+    nQb, nKb = -(-N // Bq), -(-N // Bk)
+    assert len(rp) == B * H * nQb + 1 and (np.diff(rp) == topk).all()
+    q64, k64 = q.astype(np.float64), k.astype(np.float64)
+    for b in range(B):
+        for h in range(H):
+            kbar = np.stack([k64[b, h, j * Bk:(j + 1) * Bk].mean(0) for j in range(nKb)])       # [nKb, d]
+            tok = q64[b, h] @ kbar.T                                                          # [N, nKb]
+            for i in range(nQb):
+                s = tok[i * Bq:(i + 1) * Bq].mean(0)
+                np.testing.assert_allclose(sc[b * H + h, i], s, rtol=1e-12, atol=1e-13)
+                want = np.sort(np.argsort(-s, kind="stable")[:topk])
+                r = (b * H + h) * nQb + i
+                assert ci[rp[r]:rp[r + 1]].tolist() == want.tolist()
+
+
+def test_topk_mask_special_cases():
+    rng = np.random.default_rng(78)
+    B, H, N, d, Bq, Bk = 1, 2, 128, 8, 32, 16
+    q = bf16_round(rng.standard_normal((B, H, N, d))); k = bf16_round(rng.standard_normal((B, H, N, d)))
+    nQb, nKb = N // Bq, N // Bk
+    # k >= number of key blocks: everything is kept, i.e. the dense lists
+    rp, ci = orc.topk_mask(q, k, Bq, Bk, nKb + 5)
+    drp, dci = wlmod.dense_csr(nQb, nKb, B * H)
+    assert rp.tolist() == drp.tolist() and ci.tolist() == dci.tolist()
+    # a planted key block: its tokens all equal c * qbar_i, c large -> query block i must select it
+    k2 = k.copy()
+    i, j = 2, 5
+    qbar = q[0, 1, i * Bq:(i + 1) * Bq].astype(np.float64).mean(0)
+    k2[0, 1, j * Bk:(j + 1) * Bk] = bf16_round(50.0 * qbar)
+    rp2, ci2 = orc.topk_mask(q, k2, Bq, Bk, 1)
+    assert ci2[(1 * nQb + i)] == j
+    # positive rescaling of the queries changes no selection; heads and batch items are independent
+    rp3, ci3 = orc.topk_mask(4.0 * q, k, Bq, Bk, 3)
+    assert ci3.tolist() == orc.topk_mask(q, k, Bq, Bk, 3)[1].tolist()
+    sub = orc.topk_mask(q[:, 1:2], k[:, 1:2], Bq, Bk, 3)[1]
+    assert sub.tolist() == orc.topk_mask(q, k, Bq, Bk, 3)[1].reshape(H, -1)[1].tolist()
+
+
+def test_sparse_attn_with_per_batch_and_head_masks():
+    # Hm = B*H: head (b, h) uses list block b*H + h.  Against a dense masked softmax built per head.
+    rng = np.random.default_rng(79)
+    B, H, N, d, Bq, Bk = 2, 2, 64, 8, 16, 16
+    q, k, v = rand_qkv(B, H, N, d, 79)
+    rp, ci = orc.topk_mask(q, k, Bq, Bk, 2)
+    out = orc.sparse_attn(q, k, v, Bq, Bk, rp, ci, B * H)[0].reshape(B, H, N, d)
+    nQb = N // Bq
+    for b in range(B):
+        for h in range(H):
+            M = np.full((N, N), -np.inf)
+            for i in range(nQb):
+                r = (b * H + h) * nQb + i
+                for j in ci[rp[r]:rp[r + 1]]:
+                    M[i * Bq:(i + 1) * Bq, j * Bk:(j + 1) * Bk] = 0.0
+            x = q[b, h].astype(np.float64) @ k[b, h].astype(np.float64).T / np.sqrt(d) + M
+            p = np.exp(x - x.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
+            np.testing.assert_allclose(out[b, h], p @ v[b, h].astype(np.float64), rtol=1e-10, atol=1e-12)
