@@ -326,6 +326,21 @@ def main():
                                    "achieved_gbs": x_bytes / (dyn_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
                                    "frac": x_bytes / (dyn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del xt
+        # Top-K mask producer (App. A.1 steps 1-2) at this shape, k chosen for the same 90 % sparsity:
+        # block means read Q and K once (the HBM-bound part), then scores and selection
+        topk = max(1, round(wl.nKb * (1.0 - sparsity)))
+        tk_ws = torch.empty(int(salad._lib.salad_topk_workspace_bytes(wl.B, wl.H, wl.N, wl.d, wl.Bq, wl.Bk)),
+                            dtype=torch.uint8, device=dev)
+        tk_rp = torch.empty(wl.B * wl.H * wl.nQb + 1, dtype=torch.int32, device=dev)
+        tk_ci = torch.empty(wl.B * wl.H * wl.nQb * topk, dtype=torch.int32, device=dev)
+        tk_ms = timed(lambda: salad.salad_topk_mask_build(q, k, topk, Bq=wl.Bq, Bk=wl.Bk, row_ptr=tk_rp,
+                                                          col_idx=tk_ci, workspace=tk_ws), 20)
+        extras["topk_mask"] = {"k": topk, "ms": tk_ms, "algorithmic_bytes": 2 * tensor_bytes,
+                               "achieved_gbs": 2 * tensor_bytes / (tk_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                               "frac": 2 * tensor_bytes / (tk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        tk_fused_ms = timed(lambda: salad.salad_fused_fwd(q, k, v, tk_rp, tk_ci, wl.B * wl.H, lam_d, s_d, Bq=wl.Bq,
+                                                          Bk=wl.Bk, out=out, workspace=ws), 10)
+        extras["topk_mask"]["fused_on_topk_lists_ms"] = tk_fused_ms
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -16,8 +16,10 @@
  *   - The sparsity mask is block granular: query block i covers tokens [i*Bq, (i+1)*Bq),
  *     key block j covers [j*Bk, (j+1)*Bk).  It is passed as CSR lists: row r = hm*nQb + i
  *     (nQb = ceil(N/Bq)) owns col_idx[row_ptr[r] .. row_ptr[r+1]), the kept key blocks,
- *     ascending and unique, each in [0, ceil(N/Bk)).  Hm is 1 (one mask for all heads) or H.
- *     The mask is shared by all batch items.  An empty row is legal: its O_s is zero.
+ *     ascending and unique, each in [0, ceil(N/Bk)).  Hm is 1 (one mask for all heads), H
+ *     (one per head, shared by the batch items; hm = h) or B*H (one per batch item and head,
+ *     hm = b*H + h: input-dependent masks such as salad_topk_mask_build's).  An empty row is
+ *     legal: its O_s is zero.
  *   - Every pointer is DEVICE memory owned by the caller unless its name starts with h_
  *     (host).  Nothing is allocated or freed by the library; scratch comes from a caller
  *     workspace of at least salad_workspace_bytes() bytes, 256-byte aligned, which must
@@ -152,6 +154,27 @@ int salad_fused_drop_fwd(const void* q, const void* k, const void* v, void* o,
 #define SALAD_DYN_SCALE_WS_BYTES 8192
 int salad_dynamic_scale(const void* x, const float* w, float bias, int B, int N, int D,
                         float* s_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * salad_topk_mask_build -- the dynamic Top-K block mask (Sec. 3; Appendix A.1, Steps 1-2), as
+ * CSR lists for the attention entry points (Hm = B*H).  Per batch item and head:
+ *     kbar_j = mean of the key tokens of block j,   qbar_i = mean of the query tokens of block i,
+ *     s[i][j] = <qbar_i, kbar_j>   (= the block's average of its tokens' similarity with kbar_j),
+ *     row i keeps the kk = min(topk, nKb) key blocks with the largest s, a tie going to the
+ *     lower block index; the kept blocks are written in ascending order.
+ * Arithmetic: fp32 sums and FMAs in a fixed order (deterministic).  Scores are assumed finite.
+ *   q, k           bf16 [B, H, N, d], d in {64, 128}; Bq, Bk <= 1024.
+ *   d_row_ptr      device int32 [B*H*nQb + 1], written (row r starts at r*kk).
+ *   d_col_idx      device int32, capacity col_capacity entries; B*H*nQb*kk are written,
+ *                  SALAD_ERR_CAPACITY if it is smaller (nothing is launched).
+ *   workspace      at least salad_topk_workspace_bytes() bytes, 256-byte aligned (block means and
+ *                  the B*H*nQb*nKb scores).
+ * Asynchronous on `stream`; no host synchronisation (the list sizes are known in advance).
+ */
+size_t salad_topk_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk);
+int salad_topk_mask_build(const void* q, const void* k, int B, int H, int N, int d, int Bq, int Bk,
+                          int topk, int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
+                          void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide

@@ -147,7 +147,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     }
     const int h = bh % p.H, b = bh / p.H;
-    const int hm = (p.Hm == 1) ? 0 : h;
+    const int hm = (p.Hm == 1) ? 0 : (p.Hm == p.H ? h : bh);   // one mask, one per head, or one per (batch, head)
     const int pair = p.order ? __ldg(p.order + size_t(hm) * p.nPairs + rank) : rank;
     const bool sparse = (p.mode & MODE_SPARSE) != 0;
     // post-tuning branch dropping (Sec. 4.3): no linear work at all for a dropped batch item
@@ -161,8 +161,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         qb[i] = 2 * pair + i;
         ls[i] = le[i] = 0;
         if (sparse && qb[i] < p.nQb) {
-            ls[i] = __ldg(p.row_ptr + hm * p.nQb + qb[i]);
-            le[i] = __ldg(p.row_ptr + hm * p.nQb + qb[i] + 1);
+            ls[i] = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb[i]);
+            le[i] = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb[i] + 1);
         }
     }
 

@@ -12,6 +12,7 @@
 #include "linear_state_kernel.cuh"
 #include "mask_kernels.cuh"
 #include "tmap.cuh"
+#include "topk_mask_kernels.cuh"
 
 using namespace salad;
 
@@ -47,7 +48,7 @@ Workspace carve(int B, int H, int N, int d, int Bq) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = w.off_zp + align_up(size_t(w.slots) * d * 4);
-    w.total = w.off_order + align_up(size_t(H) * nPairs * 4);       // launch order, per mask head
+    w.total = w.off_order + align_up(BH * nPairs * 4);              // launch order, per mask (at most B*H)
     return w;
 }
 
@@ -139,7 +140,7 @@ int validate(const Problem& P) {
     if (int64_t(P.B) * P.H > 65535) return SALAD_ERR_UNSUPPORTED;
     if (P.mode & MODE_SPARSE) {
         if (!P.row_ptr || !P.col_idx) return SALAD_ERR_INVALID_ARG;
-        if (P.Hm != 1 && P.Hm != P.H) return SALAD_ERR_INVALID_ARG;
+        if (P.Hm != 1 && P.Hm != P.H && P.Hm != P.B * P.H) return SALAD_ERR_INVALID_ARG;
         if (!(P.softmax_scale >= 0.f) || !isfinite(P.softmax_scale)) return SALAD_ERR_INVALID_ARG;
     }
     if (P.mode & MODE_LINEAR) {
@@ -489,6 +490,72 @@ SALAD_EXPORT int salad_dynamic_scale(const void* x, const float* w, float bias, 
         static_cast<const uint4*>(x), w, bias, N, D, partial);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     dynamic_scale_finalize_kernel<<<B, 32, 0, st>>>(partial, G, N, s_out);
+    return check_launch();
+}
+
+SALAD_EXPORT size_t salad_topk_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk) {
+    if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || Bq <= 0 || Bk <= 0) return 0;
+    const size_t BH = size_t(B) * H;
+    const size_t nQb = (size_t(N) + Bq - 1) / Bq, nKb = (size_t(N) + Bk - 1) / Bk;
+    const size_t ldk = (nKb + kScoreTile - 1) / kScoreTile * kScoreTile;
+    // query-block means | key-block means, channel-major, rows padded to whole tiles | scores
+    return align_up(BH * nQb * d * 4) + align_up(BH * d * ldk * 4) + align_up(BH * nQb * nKb * 4);
+}
+
+SALAD_EXPORT int salad_topk_mask_build(const void* q, const void* k, int B, int H, int N, int d, int Bq, int Bk,
+                                       int topk, int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (!q || !k || !d_row_ptr || !d_col_idx || B <= 0 || H <= 0 || N <= 0 || d <= 0 || Bq <= 0 || Bk <= 0 ||
+        topk <= 0)
+        return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k)) return SALAD_ERR_INVALID_ARG;
+    if ((d != 64 && d != 128) || Bq > 1024 || Bk > 1024) return SALAD_ERR_UNSUPPORTED;
+    const int64_t BH = int64_t(B) * H;
+    const int64_t nQb = (int64_t(N) + Bq - 1) / Bq, nKb = (int64_t(N) + Bk - 1) / Bk;
+    const int64_t kk = topk < nKb ? topk : nKb;
+    const int64_t rows = BH * nQb;
+    if (BH > 65535 || nQb > 65535 * int64_t(kScoreRows) || rows * kk > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
+    if (col_capacity < rows * kk) return SALAD_ERR_CAPACITY;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 ||
+        workspace_bytes < salad_topk_workspace_bytes(B, H, N, d, Bq, Bk))
+        return SALAD_ERR_WORKSPACE;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int ldk = int((nKb + kScoreTile - 1) / kScoreTile * kScoreTile);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* qmean = reinterpret_cast<float*>(ws);
+    float* kmeanT = reinterpret_cast<float*>(ws + align_up(size_t(BH) * nQb * d * 4));
+    uint32_t* score = reinterpret_cast<uint32_t*>(ws + align_up(size_t(BH) * nQb * d * 4) +
+                                                  align_up(size_t(BH) * d * ldk * 4));
+    MeanJob jq{static_cast<const uint4*>(q), qmean, Bq, int(nQb), 0};
+    MeanJob jk{static_cast<const uint4*>(k), kmeanT, Bk, int(nKb), ldk};
+    block_mean_kernel<<<dim3(unsigned(nQb > nKb ? nQb : nKb), unsigned(BH), 2), kMeanThreads, 0, st>>>(jq, jk, N, d);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    const size_t smem = size_t(d) * (kScoreRows + kScoreTile) * 4;          // 80 KB at d = 128
+    static bool smem_set[64] = {};
+    int devi = 0;
+    cudaGetDevice(&devi);
+    if (devi >= 0 && devi < 64 && !smem_set[devi]) {
+        if (cudaFuncSetAttribute(topk_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 160 * 4) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return SALAD_ERR_CUDA;
+        }
+        smem_set[devi] = true;
+    }
+    launch_dependent(topk_score_kernel, dim3(unsigned(ldk / kScoreTile), unsigned((nQb + kScoreRows - 1) / kScoreRows),
+                                             unsigned(BH)),
+                     dim3(256), smem, st, qmean, kmeanT, int(nQb), int(nKb), ldk, d, score);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    const dim3 pgrid(unsigned((rows + 7) / 8));
+    if (nKb <= 512)
+        launch_dependent(topk_pick_kernel<16>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+    else if (nKb <= 1024)
+        launch_dependent(topk_pick_kernel<32>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+    else
+        launch_dependent(topk_pick_kernel<0>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
     return check_launch();
 }
 

@@ -27,7 +27,7 @@ SALAD_ERR_TIMEOUT = -6
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
-           "salad_dynamic_scale")
+           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build")
 
 
 class SaladError(RuntimeError):
@@ -61,6 +61,10 @@ def _load() -> ctypes.CDLL:
     lib.salad_fused_drop_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, f32, p, sz, p, p]
     lib.salad_dynamic_scale.restype = i32
     lib.salad_dynamic_scale.argtypes = [p, p, f32, i32, i32, i32, p, p, sz, p]
+    lib.salad_topk_workspace_bytes.restype = sz
+    lib.salad_topk_workspace_bytes.argtypes = [i32] * 6
+    lib.salad_topk_mask_build.restype = i32
+    lib.salad_topk_mask_build.argtypes = [p, p] + [i32] * 7 + [p, p, ctypes.c_int64, p, sz, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -204,6 +208,33 @@ def salad_linear_attn_fwd_noalloc(q, k, v, eps: float = 1e-6, out=None, kv_out=N
                                                   B, H, N, d, float(eps), _ptr(status), _stream(stream)),
                "salad_linear_attn_fwd_noalloc")
     return out
+
+
+def salad_topk_mask_build(q, k, topk: int, Bq: int = 128, Bk: int = 64, row_ptr=None, col_idx=None,
+                          workspace=None, stream=None):
+    """Top-K block mask of every (batch, head): returns (row_ptr, col_idx) int32 device tensors, to be
+    passed to the attention calls with Hm = B*H."""
+    for name, t in (("q", q), ("k", k)):
+        _bf16_4d(name, t)
+    if q.shape != k.shape:
+        raise ValueError("q and k must have the same shape")
+    B, H, N, d = q.shape
+    nQb, nKb = -(-N // Bq), -(-N // Bk)
+    kk = min(int(topk), nKb)
+    rows = B * H * nQb
+    if row_ptr is None:
+        row_ptr = torch.empty(rows + 1, dtype=torch.int32, device=q.device)
+    if col_idx is None:
+        col_idx = torch.empty(max(rows * kk, 1), dtype=torch.int32, device=q.device)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    if workspace is None:
+        nbytes = int(_lib.salad_topk_workspace_bytes(B, H, N, d, Bq, Bk))
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_topk_mask_build(_ptr(q), _ptr(k), B, H, N, d, Bq, Bk, int(topk), _ptr(row_ptr),
+                                          _ptr(col_idx), col_idx.numel(), _ptr(workspace), workspace.numel(),
+                                          _stream(stream)), "salad_topk_mask_build")
+    return row_ptr, col_idx[:rows * kk]
 
 
 DYN_SCALE_WS_BYTES = 8192

@@ -421,3 +421,81 @@ def test_scale_producer_feeds_the_fused_call(salad):
     s_ref = orc.dynamic_scale(f32(x), w)
     ref = orc.salad_fused(f32(q), f32(k), f32(v), 64, 64, rp, ci, 1, lam, s_ref)
     assert_close(f32(out.cpu()).reshape(-1, d), ref, "chain")
+
+
+# ------------------------------------------------------------------------------ Top-K mask producer
+
+def _check_topk_lists(rp_g, ci_g, rp_o, ci_o, scores, kk):
+    """Bit-exact where the selection is unique.  The device scores are fp32, the oracle's fp64: a row
+    may differ only where the scores of the swapped blocks agree to fp32 rounding (a near tie), and
+    every list must still be a valid selection (kk blocks, ascending, in range)."""
+    assert np.array_equal(rp_g, rp_o)
+    rows = len(rp_o) - 1
+    g = ci_g.reshape(rows, kk); o = ci_o.reshape(rows, kk)
+    nKb = scores.shape[-1]
+    assert (np.diff(g, axis=1) > 0).all() and g.min() >= 0 and g.max() < nKb
+    bad = np.nonzero((g != o).any(axis=1))[0]
+    sc = scores.reshape(rows, nKb)
+    for r in bad:
+        only_g = np.setdiff1d(g[r], o[r]); only_o = np.setdiff1d(o[r], g[r])
+        assert len(only_g) == len(only_o)
+        tol = 1e-5 * max(1.0, np.abs(sc[r]).max())
+        # whatever the device took instead scores within rounding of what the oracle took
+        assert np.abs(np.sort(sc[r][only_g]) - np.sort(sc[r][only_o])).max() <= tol, (r, g[r], o[r])
+    return len(bad)
+
+
+@pytest.mark.parametrize("B,H,N,d,Bq,Bk,topk", [
+    (1, 2, 1024, 64, 64, 64, 4),
+    (2, 3, 1000, 128, 128, 64, 4),      # ragged last blocks on both sides
+    (1, 2, 2500, 128, 128, 64, 8),
+    (1, 1, 700, 64, 64, 64, 100),       # k above the number of key blocks: dense lists
+])
+def test_topk_mask_build(salad, B, H, N, d, Bq, Bk, topk):
+    q, k, _ = rand_qkv(B, H, N, d, 900 + N)
+    rp_o, ci_o, sc = orc.topk_mask(f32(q), f32(k), Bq, Bk, topk, return_scores=True)
+    rp_g, ci_g = salad.salad_topk_mask_build(q.cuda(), k.cuda(), topk, Bq=Bq, Bk=Bk)
+    kk = min(topk, -(-N // Bk))
+    ndiff = _check_topk_lists(rp_g.cpu().numpy(), ci_g.cpu().numpy(), rp_o, ci_o, sc, kk)
+    assert ndiff <= max(1, (len(rp_o) - 1) // 50)            # near ties are rare
+
+
+def test_topk_mask_wan13b_shape(salad):
+    # full size, the configuration the benchmark times: k = 51 of 512 key blocks (90 % block sparsity)
+    wl = wlmod.C2
+    q, k, _ = wlmod.make_qkv(wl)
+    rp_o, ci_o, sc = orc.topk_mask(f32(q), f32(k), wl.Bq, wl.Bk, 51, return_scores=True)
+    rp_g, ci_g = salad.salad_topk_mask_build(q.cuda(), k.cuda(), 51, Bq=wl.Bq, Bk=wl.Bk)
+    ndiff = _check_topk_lists(rp_g.cpu().numpy(), ci_g.cpu().numpy(), rp_o, ci_o, sc, 51)
+    assert ndiff <= (len(rp_o) - 1) // 50
+
+
+def test_topk_mask_feeds_the_fused_call(salad):
+    # producer -> consumer on the device with per-(batch, head) lists (Hm = B*H); the oracle runs the
+    # same lists the device built, so a near tie cannot fail this test
+    B, H, N, d, Bq = 2, 3, 1000, 128, 128
+    q, k, v = rand_qkv(B, H, N, d, 77)
+    lam = np.array([0.3, 0.8, 0.5], dtype=np.float32); s = np.array([0.6, 0.2], dtype=np.float32)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    rp, ci = salad.salad_topk_mask_build(qd, kd, 5, Bq=Bq)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_fwd(qd, kd, vd, rp, ci, B * H, torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda(),
+                                Bq=Bq, status=status)
+    status_ok(status)
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), Bq, 64, rp.cpu().numpy(), ci.cpu().numpy(), B * H,
+                          lam.astype(np.float64), s.astype(np.float64))
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "fused on top-k lists")
+    sp = salad.salad_sparse_attn_fwd(qd, kd, vd, rp, ci, B * H, Bq=Bq)
+    ref_s, _ = orc.sparse_attn(f32(q), f32(k), f32(v), Bq, 64, rp.cpu().numpy(), ci.cpu().numpy(), B * H)
+    assert_close(f32(sp.cpu()).reshape(-1, d), ref_s, "sparse on top-k lists")
+
+
+def test_topk_mask_capacity_and_arguments(salad):
+    q, k, _ = rand_qkv(1, 1, 256, 64, 3)
+    small = torch.empty(3, dtype=torch.int32, device="cuda")
+    with pytest.raises(salad.SaladError) as e:
+        salad.salad_topk_mask_build(q.cuda(), k.cuda(), 2, Bq=64, col_idx=small)
+    assert e.value.code == salad.SALAD_ERR_CAPACITY
+    with pytest.raises(salad.SaladError) as e:
+        salad.salad_topk_mask_build(q.cuda(), k.cuda(), 0, Bq=64)
+    assert e.value.code == salad.SALAD_ERR_INVALID_ARG
