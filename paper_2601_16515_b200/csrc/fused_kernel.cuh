@@ -30,8 +30,10 @@
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
 //
-// TMEM columns (512 allocated), tile i at 256 i:  [0,64) S;  [64,96) and [96,128) the two P
-// buffers;  [128,128+D) O.  The linear numerator reuses [0,D).
+// TMEM columns (512 allocated), tile i at 256 i:  [0,64) and [64,128) two score buffers (block t
+// uses buffer t & 1; its probabilities, packed bf16, overwrite the first 32 columns of the same
+// buffer, so the scores of block t + 1 can be computed while block t is still in the softmax);
+// [128,128+D) O.  The linear numerator reuses [0,D).
 #pragma once
 #include "ptx.cuh"
 
@@ -81,13 +83,15 @@ struct FusedCfg {
     static constexpr int OFF_K = OFF_ST + ST_BYTES;
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
-    static constexpr int THREADS = 512;
-    static constexpr uint32_t COL_S = 0, COL_P = 64, COL_O = 128;     // TMEM columns within a tile's 256
+    static constexpr int THREADS = 768;
+    // TMEM columns within a tile's 256: two score buffers of 64 (P overwrites the first 32 columns
+    // of the buffer its scores came from), then the output accumulator
+    static constexpr uint32_t COL_SP = 0, SP_STRIDE = 64, COL_O = 128;
 };
 
 struct FusedBarriers {
     uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], s_free[2], p_ready[2][2], pv_done[2][2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
+    uint64_t s_full[2][2], p_ready[2][2], pv_done[2][2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
 };
 
 // Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
@@ -114,7 +118,7 @@ struct MergeWalk {
 };
 
 template <int D>
-__global__ void __launch_bounds__(512, 1)
+__global__ void __launch_bounds__(768, 1)
 salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                    const __grid_constant__ CUtensorMap map_st, const FusedParams p)
@@ -172,14 +176,13 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.s_free[i]), 4);              // one arrival per softmax warp
             mbar_init(smem_u32(&bars.o_final[i]), 1);
-            mbar_init(smem_u32(&bars.lin_ready[i]), 128);
+            mbar_init(smem_u32(&bars.lin_ready[i]), 256);
             mbar_init(smem_u32(&bars.lin_done[i]), 1);
-            mbar_init(smem_u32(&bars.out_staged[i]), 128);
+            mbar_init(smem_u32(&bars.out_staged[i]), 256);
             for (int j = 0; j < 2; ++j) {
-                mbar_init(smem_u32(&bars.p_ready[i][j]), 4);
+                mbar_init(smem_u32(&bars.s_full[i][j]), 1);
+                mbar_init(smem_u32(&bars.p_ready[i][j]), 8);          // one arrival per softmax warp
                 mbar_init(smem_u32(&bars.pv_done[i][j]), 1);
             }
         }
@@ -277,17 +280,17 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars.k_full[s]), (g / C::NK) & 1, abortp);
                 if (!ok) break;
                 if ((tag >> i) & 1) {
-                    // the softmax warps must have copied the scores of the previous block out of S
-                    if (t > 0) ok = mbar_wait(smem_u32(&bars.s_free[i]), (t - 1) & 1, abortp);
+                    // score buffer t & 1 held P of block t - 2: its P V product must have read it
+                    if (t >= 2) ok = mbar_wait(smem_u32(&bars.pv_done[i][t & 1]), ((t >> 1) - 1) & 1, abortp);
                     if (!ok) break;
                     TRACE(2 + i, t, 0);
                     tc_fence_after_sync();
                     const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
-                        mma_ss_lohi(t_tile + C::COL_S, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                        mma_ss_lohi(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
                                     kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                    tc_commit(smem_u32(&bars.s_full[i]));
+                    tc_commit(smem_u32(&bars.s_full[i][t & 1]));
                     tc_commit(smem_u32(&bars.k_empty[s]));
                     TRACE(2 + i, t, 3);
                     ++t;
@@ -321,7 +324,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     TRACE(2 + i, t, 1);
                     tc_fence_after_sync();
                     const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
-                    const uint32_t p_col = t_tile + C::COL_P + (t & 1) * 32;
+                    const uint32_t p_col = t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE;
 #pragma unroll
                     for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
                         mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
@@ -352,151 +355,172 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp >= 8) {
         // ============================================================== softmax + epilogue
-        const int i = (warp - 8) >> 2;            // tile
-        const int row = tid - 256 - 128 * i;      // query row within the tile = TMEM lane
-        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t t_tile = tmem + i * 256 + lane_addr;
+        // Eight warps per tile.  A warp works on 16 TMEM lanes (query rows) with the 16-lane
+        // load/store shapes: four threads share a row, each holding a quarter of its columns,
+        // and every thread serves two rows (a and a + 8).  Row maxima and sums are combined
+        // with two shuffles inside the group of four.
+        const int sw = warp - 8;
+        const int i = sw >> 3;                                  // tile
+        const int q4 = lane & 3;                                // position in the group of four
+        const int lane0 = (warp & 3) * 32 + ((sw >> 2) & 1) * 16;          // first TMEM lane of this warp
+        const int ra = lane0 + (lane >> 2), rb = ra + 8;        // the thread's two query rows
+        const uint32_t t_tile = tmem + i * 256 + (uint32_t(lane0) << 16);
         const bool tile_valid = qb[i] < p.nQb;
         const int len = le[i] - ls[i];
         uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_a = -INFINITY, m_b = -INFINITY;                 // running maxima (log2 domain)
+        float l_a = 0.f, l_b = 0.f;                             // this thread's share of the row sums
         bool ok = true;
         // every lane of a warp must take the same path around the warp-collective tcgen05
         // loads/stores, so the outcome of a bounded wait is made warp-uniform
         auto wait_uniform = [&](uint64_t* bar, uint32_t parity) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, abortp));
         };
+        auto quad_max = [](float v) -> float {
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+        };
+        auto quad_sum = [](float v) -> float {
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            return v + __shfl_xor_sync(0xffffffffu, v, 2);
+        };
 
         const bool ragged_keys = (p.N % C::BK) != 0;
         for (int t = 0; t < len && ok; ++t) {
-            if (row == 0) TRACE(i, t, 0);
+            if (ra == 0 && q4 == 0) TRACE(i, t, 0);
             // only the last key block can be short; its id is needed only then
             const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
-            ok = wait_uniform(&bars.s_full[i], t & 1);
+            ok = wait_uniform(&bars.s_full[i][t & 1], (t >> 1) & 1);
             if (!ok) break;
-            if (row == 0) TRACE(i, t, 1);
+            if (ra == 0 && q4 == 0) TRACE(i, t, 1);
             tc_fence_after_sync();
-            uint32_t xr[64];
-            tmem_ld32(t_tile + C::COL_S, xr);
-            tmem_ld32(t_tile + C::COL_S + 32, xr + 32);
+            // x[4n], x[4n+1] = S(row a, keys 8n + 2 q4, + 1);  x[4n+2], x[4n+3] = the same keys of row b
+            uint32_t xr[32];
+            tmem_ld_16x256b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, xr);
             tmem_wait_ld();
-            // the scores are in registers: the S buffer may take the next block's
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[i]));
-            if (row == 0) TRACE(i, t, 2);
+            if (ra == 0 && q4 == 0) TRACE(i, t, 2);
             float* x = reinterpret_cast<float*>(xr);
-            const int valid = p.N - col * C::BK;          // keys of this block that exist
+            const int valid = p.N - col * C::BK;              // keys of this block that exist
             if (ragged_keys && valid < C::BK) {
 #pragma unroll
-                for (int c = 0; c < C::BK; ++c) if (c >= valid) x[c] = -INFINITY;
+                for (int n = 0; n < 8; ++n) {
+                    const int key = 8 * n + 2 * q4;
+                    if (key >= valid) { x[4 * n] = -INFINITY; x[4 * n + 2] = -INFINITY; }
+                    if (key + 1 >= valid) { x[4 * n + 1] = -INFINITY; x[4 * n + 3] = -INFINITY; }
+                }
             }
-            auto row_max_scaled = [&]() -> float {
-                float mx[4] = {x[0], x[1], x[2], x[3]};
+            // block maxima of the two rows
+            float mxa = fmaxf(x[0], x[1]), mxb = fmaxf(x[2], x[3]);
 #pragma unroll
-                for (int c = 4; c < C::BK - 4; c += 8) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) mx[e] = fmaxf(fmaxf(mx[e], x[c + e]), x[c + 4 + e]);
-                }
-#pragma unroll
-                for (int e = 0; e < 4; ++e) mx[e] = fmaxf(mx[e], x[C::BK - 4 + e]);
-                return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
-            };
-            uint32_t pk[32];
-            auto exp_row = [&](float m_ref) -> float {    // P = exp2(x * scale - m_ref), packed bf16; returns the row sum
-                const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(-m_ref, -m_ref);
-                uint64_t acc0 = pack_f32x2(0.f, 0.f), acc1 = acc0;
-#pragma unroll
-                for (int c = 0; c < C::BK; c += 4) {              // scale-and-shift and the row sum two at a time
-                    float a0, a1, a2, a3;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(x[c], x[c + 1]), sc2, nm2), a0, a1);
-                    unpack_f32x2(fma_f32x2(pack_f32x2(x[c + 2], x[c + 3]), sc2, nm2), a2, a3);
-                    const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(a2), p3 = ex2_approx(a3);
-                    acc0 = add_f32x2(acc0, pack_f32x2(p0, p1));
-                    acc1 = add_f32x2(acc1, pack_f32x2(p2, p3));
-                    pk[c >> 1] = pack_bf16x2(p0, p1);
-                    pk[(c >> 1) + 1] = pack_bf16x2(p2, p3);
-                }
-                float s0, s1, s2, s3;
-                unpack_f32x2(acc0, s0, s1);
-                unpack_f32x2(acc1, s2, s3);
-                return (s0 + s1) + (s2 + s3);
-            };
-            // the block max first (the running max only moves when it grows by more than 2^8),
-            // then one pass of exponentials: the scores die as P is packed
-            const float msc = row_max_scaled();
+            for (int n = 1; n < 8; ++n) {
+                mxa = fmaxf(mxa, fmaxf(x[4 * n], x[4 * n + 1]));
+                mxb = fmaxf(mxb, fmaxf(x[4 * n + 2], x[4 * n + 3]));
+            }
+            const float msa = quad_max(mxa) * p.scale_log2, msb = quad_max(mxb) * p.scale_log2;
+            // The running max only moves when it grows by more than 2^8: then the accumulator of this
+            // warp's rows is brought to the new max, once the previous P V product has landed in it.
+            // pv_done[b] completes a phase for every second block; the product of block t cannot be
+            // issued before this warp hands over P of block t, so the barrier is at most one phase
+            // past the one tested here and the parity test is exact.
             if (t == 0) {
-                m_run = msc;
-            } else if (__any_sync(0xffffffffu, msc > m_run + 8.0f)) {
-                // bring the accumulator of this warp's rows to the new running max, once the
-                // previous P V product has landed in it.  pv_done[b] completes a phase for
-                // every second block; the product of block t cannot be issued before this
-                // thread hands over P of block t, so the barrier is at most one phase past
-                // the one tested here and the parity test is exact.
+                m_a = msa; m_b = msb;
+            } else if (__any_sync(0xffffffffu, msa > m_a + 8.0f || msb > m_b + 8.0f)) {
                 ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const float m_new = fmaxf(m_run, msc);
-                const float alpha = ex2_approx(m_run - m_new);
-                l_run *= alpha;
-                m_run = m_new;
+                const float na = fmaxf(m_a, msa), nb = fmaxf(m_b, msb);
+                const float al_a = ex2_approx(m_a - na), al_b = ex2_approx(m_b - nb);
+                l_a *= al_a; l_b *= al_b;
+                m_a = na; m_b = nb;
 #pragma unroll
-                for (int cc = 0; cc < D / 16; ++cc) {
+                for (int cc = 0; cc < D / 32; ++cc) {
                     uint32_t orr[16];
-                    tmem_ld16(t_tile + C::COL_O + cc * 16, orr);
+                    tmem_ld_16x256b_x4(t_tile + C::COL_O + cc * 32, orr);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                    tmem_st16(t_tile + C::COL_O + cc * 16, orr);
+                    for (int n = 0; n < 4; ++n) {
+                        orr[4 * n] = __float_as_uint(__uint_as_float(orr[4 * n]) * al_a);
+                        orr[4 * n + 1] = __float_as_uint(__uint_as_float(orr[4 * n + 1]) * al_a);
+                        orr[4 * n + 2] = __float_as_uint(__uint_as_float(orr[4 * n + 2]) * al_b);
+                        orr[4 * n + 3] = __float_as_uint(__uint_as_float(orr[4 * n + 3]) * al_b);
+                    }
+                    tmem_st_16x256b_x4(t_tile + C::COL_O + cc * 32, orr);
                 }
                 tmem_wait_st();
             }
-            const float row_sum = exp_row(m_run);
-            l_run += row_sum;
-            if (row == 0) TRACE(i, t, 4);
-            if (t >= 2) {
-                // P buffer t & 1 was read by the P V product of block t - 2
-                ok = wait_uniform(&bars.pv_done[i][t & 1], ((t >> 1) - 1) & 1);
-                if (!ok) break;
+            if (ra == 0 && q4 == 0) TRACE(i, t, 3);
+            // P = exp2(x * scale - m), packed bf16: word 2n = row a, keys (8n + 2 q4, + 1) = packed
+            // column 4n + q4 of the P tile, word 2n + 1 the same of row b -- the 16x128b layout
+            uint32_t pk[16];
+            {
+                const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2);
+                const uint64_t nma = pack_f32x2(-m_a, -m_a), nmb = pack_f32x2(-m_b, -m_b);
+                uint64_t acc_a = pack_f32x2(0.f, 0.f), acc_b = acc_a;
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                    float a0, a1, b0, b1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x[4 * n], x[4 * n + 1]), sc2, nma), a0, a1);
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x[4 * n + 2], x[4 * n + 3]), sc2, nmb), b0, b1);
+                    const float pa0 = ex2_approx(a0), pa1 = ex2_approx(a1), pb0 = ex2_approx(b0), pb1 = ex2_approx(b1);
+                    acc_a = add_f32x2(acc_a, pack_f32x2(pa0, pa1));
+                    acc_b = add_f32x2(acc_b, pack_f32x2(pb0, pb1));
+                    pk[2 * n] = pack_bf16x2(pa0, pa1);
+                    pk[2 * n + 1] = pack_bf16x2(pb0, pb1);
+                }
+                float s0, s1;
+                unpack_f32x2(acc_a, s0, s1); l_a += s0 + s1;
+                unpack_f32x2(acc_b, s0, s1); l_b += s0 + s1;
             }
-            tmem_st32(t_tile + C::COL_P + (t & 1) * 32, pk);
+            if (ra == 0 && q4 == 0) TRACE(i, t, 4);
+            // P goes over the scores it was computed from (this warp's own lanes, already in registers)
+            tmem_st_16x128b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i][t & 1]));   // one arrival per warp
-            if (row == 0) TRACE(i, t, 5);
+            if (ra == 0 && q4 == 0) TRACE(i, t, 5);
         }
-        float lin_coef = 0.f;
+        float coef_a = 0.f, coef_b = 0.f;
         if (ok && tile_valid && linear) {
-            // ReLU of this thread's Q row in place, and the denominator ReLU(Q_n) . Z.  Every
-            // Q K^T of this tile has completed (its scores were consumed above), so Q is no
-            // longer read; the last P V product may still be running meanwhile.
+            // ReLU of the Q rows in place, and the denominators ReLU(Q_n) . Z: the four threads of a
+            // row take two 16-byte groups of every 64 channels each.  Every Q K^T of this tile has
+            // completed (its scores were consumed above), so Q is no longer read; the last P V
+            // product may still be running meanwhile.
             ok = wait_uniform(&bars.q_full[i], 0);
             if (ok) {
-                float den = 0.f;
+                float den_a = 0.f, den_b = 0.f;
 #pragma unroll
                 for (int ch = 0; ch < C::CH; ++ch) {
 #pragma unroll
-                    for (int c16 = 0; c16 < 8; ++c16) {
-                        uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
-                                                              ((c16 ^ (row & 7)) << 4));
-                        uint4 v = *ptr;
-                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+                    for (int j = 0; j < 2; ++j) {
+                        const int c16 = q4 + 4 * j;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
-                            const float2 f = __bfloat1622float2(hv[e]);
-                            const int a = ch * 64 + c16 * 8 + e * 2;
-                            den = fmaf(f.x, z_s[a], den);
-                            den = fmaf(f.y, z_s[a + 1], den);
+                        for (int e2 = 0; e2 < 2; ++e2) {
+                            const int row = e2 ? rb : ra;
+                            uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
+                                                                  ((c16 ^ (row & 7)) << 4));
+                            uint4 v = *ptr;
+                            __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+                            float den = 0.f;
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
+                                const float2 f = __bfloat1622float2(hv[e]);
+                                const int a = ch * 64 + c16 * 8 + e * 2;
+                                den = fmaf(f.x, z_s[a], den);
+                                den = fmaf(f.y, z_s[a + 1], den);
+                            }
+                            *ptr = v;
+                            if (e2) den_b += den; else den_a += den;
                         }
-                        *ptr = v;
                     }
                 }
+                den_a = quad_sum(den_a); den_b = quad_sum(den_b);
                 float c_scale = 1.f;
                 if (p.static_scale) c_scale *= __ldg(p.static_scale + h);
                 if (p.dyn_scale) c_scale *= __ldg(p.dyn_scale + b);
-                lin_coef = c_scale / (den + p.eps);
+                coef_a = c_scale / (den_a + p.eps);
+                coef_b = c_scale / (den_b + p.eps);
                 fence_proxy_async_smem();
                 mbar_arrive(smem_u32(&bars.lin_ready[i]));
             }
@@ -511,37 +535,37 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
 
         if (ok && tile_valid) {
-            // O = O_acc / l + lin_coef * num, rounded once to bf16, staged in the Q tile
-            const float inv_l = (len > 0) ? 1.0f / l_run : 0.f;
+            // O = O_acc / l + coef * num, rounded once to bf16, staged in the Q tile
+            const float lt_a = quad_sum(l_a), lt_b = quad_sum(l_b);
+            const float inv_a = (len > 0) ? 1.0f / lt_a : 0.f, inv_b = (len > 0) ? 1.0f / lt_b : 0.f;
 #pragma unroll
-            for (int cc = 0; cc < D / 16; ++cc) {
+            for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t orr[16], nr[16];
-                if (len > 0) tmem_ld16(t_tile + C::COL_O + cc * 16, orr);
-                if (linear) tmem_ld16(t_tile + cc * 16, nr);
+                if (len > 0) tmem_ld_16x256b_x4(t_tile + C::COL_O + cc * 32, orr);
+                if (linear) tmem_ld_16x256b_x4(t_tile + cc * 32, nr);
                 tmem_wait_ld();
 #pragma unroll
-                for (int c8 = 0; c8 < 2; ++c8) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int c = c8 * 8 + e * 2;
-                        float o0 = (len > 0) ? __uint_as_float(orr[c]) * inv_l : 0.f;
-                        float o1 = (len > 0) ? __uint_as_float(orr[c + 1]) * inv_l : 0.f;
-                        if (linear) {
-                            o0 = fmaf(lin_coef, __uint_as_float(nr[c]), o0);
-                            o1 = fmaf(lin_coef, __uint_as_float(nr[c + 1]), o1);
-                        }
-                        w[e] = pack_bf16x2(o0, o1);
+                for (int n = 0; n < 4; ++n) {
+                    float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+                    if (len > 0) {
+                        a0 = __uint_as_float(orr[4 * n]) * inv_a;     a1 = __uint_as_float(orr[4 * n + 1]) * inv_a;
+                        b0 = __uint_as_float(orr[4 * n + 2]) * inv_b; b1 = __uint_as_float(orr[4 * n + 3]) * inv_b;
                     }
-                    const int col16 = (cc * 16 + c8 * 8) / 8;      // 16-byte chunk index within the row
+                    if (linear) {
+                        a0 = fmaf(coef_a, __uint_as_float(nr[4 * n]), a0);     a1 = fmaf(coef_a, __uint_as_float(nr[4 * n + 1]), a1);
+                        b0 = fmaf(coef_b, __uint_as_float(nr[4 * n + 2]), b0); b1 = fmaf(coef_b, __uint_as_float(nr[4 * n + 3]), b1);
+                    }
+                    const int col16 = cc * 4 + n;                  // 16-byte group (8 columns) within the row
                     const int ch = col16 / 8, c16 = col16 % 8;
-                    *reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4)) =
-                        make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint32_t*>(qtile + ch * C::Q_CHUNK + ra * 128 + ((c16 ^ (ra & 7)) << 4) + q4 * 4) =
+                        pack_bf16x2(a0, a1);
+                    *reinterpret_cast<uint32_t*>(qtile + ch * C::Q_CHUNK + rb * 128 + ((c16 ^ (rb & 7)) << 4) + q4 * 4) =
+                        pack_bf16x2(b0, b1);
                 }
             }
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bars.out_staged[i]));
-            if (row == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
+            if (ra == 0 && q4 == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
                 for (int ch = 0; ch < C::CH; ++ch)
                     tma_store_3d(&map_o, s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, ch * 64,
                                  qb[i] * p.Bq, bh);
@@ -549,11 +573,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tma_store_wait_all();
             }
 #ifndef SALAD_TRACE
-            if (p.lse != nullptr) {
-                const int n = qb[i] * p.Bq + row;
-                if (row < p.Bq && n < p.N)
-                    p.lse[size_t(bh) * p.N + n] =
-                        (len > 0) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            if (p.lse != nullptr && q4 == 0) {
+#pragma unroll
+                for (int e2 = 0; e2 < 2; ++e2) {
+                    const int row = e2 ? rb : ra;
+                    const int n = qb[i] * p.Bq + row;
+                    if (row < p.Bq && n < p.N)
+                        p.lse[size_t(bh) * p.N + n] =
+                            (len > 0) ? ((e2 ? m_b : m_a) + log2f(e2 ? lt_b : lt_a)) * 0.6931471805599453f : -INFINITY;
+                }
             }
 #endif
         }

@@ -63,7 +63,10 @@ C5_80 = Workload("cfg-80", 2, 12, 128, (21, 30, 52), 128, 64, ((5, 5, 24),), 100
 C5_90 = replace(C5_80, name="cfg-90", windows=((2, 5, 24),))
 C5_95 = replace(C5_80, name="cfg-95", windows=((1, 4, 24),))
 C5_DENSE = replace(C5_80, name="cfg-dense", windows=((21, 30, 52),))
-ALL = {w.name: w for w in (C1, C2, C3, C4, C5_80, C5_90, C5_95, C5_DENSE)}
+# Not one of the five: the 1.3B model at the higher resolution the paper also reports (Sec. 5.1), i.e.
+# its 12 heads on the 21 x 45 x 80 latent grid (75 600 tokens), same window as the 14B-shaped config.
+C6 = Workload("wan1.3b-720p-90", 1, 12, 128, (21, 45, 80), 128, 64, ((2, 10, 36),), 1006)
+ALL = {w.name: w for w in (C1, C2, C3, C4, C5_80, C5_90, C5_95, C5_DENSE, C6)}
 
 
 def _smooth_field(rng: np.random.Generator, grid, d: int) -> np.ndarray:

@@ -317,6 +317,10 @@ def test_fused_wan14b_90(salad):
     sampled_fused_check(salad, wlmod.C4, heads=[0, 39], nrows=600)
 
 
+def test_fused_wan13b_720p_90(salad):
+    sampled_fused_check(salad, wlmod.C6, heads=[3, 11], nrows=600)
+
+
 @pytest.mark.parametrize("wl", [wlmod.C5_80, wlmod.C5_90, wlmod.C5_95])
 def test_fused_cfg_pair_sparsity_sweep(salad, wl):
     sampled_fused_check(salad, wl, heads=[3], nrows=600)
