@@ -8,18 +8,21 @@
 //   warps 2, 3    tcgen05 issuers of S = Q K^T for tile 0 and tile 1 (one thread each); warp 2
 //                 owns the TMEM allocation
 //   warps 4, 5    tcgen05 issuers of O += P V (and of the linear numerator) for tile 0 and 1
-//   warps 8-11    softmax + epilogue warpgroup of tile 0 (thread = query row = TMEM lane)
-//   warps 12-15   the same for tile 1
+//   warps 8-15    softmax + epilogue warps of tile 0: a warp works on 16 query rows (TMEM lanes)
+//                 with the 16-lane load/store shapes, four threads share a row and each thread
+//                 serves two rows; row maxima and sums are combined with two shuffles
+//   warps 16-23   the same for tile 1
 // The kept lists of the two query blocks are walked as one sorted merge, so a key block that
 // both keep is fetched once and multiplied against both tiles.  Masked blocks are never
 // loaded.
 //
-// Per tile, S = Q K^T (128x64xd, operands in shared memory) lands in one TMEM buffer that the
-// softmax warps copy to registers at once and hand back, so the scores of block t+1 are
-// computed while the softmax of block t runs.  P = exp2(.) goes, as bf16, to one of two P
-// buffers in TMEM (so O += P V of block t, which reads P from TMEM, overlaps the softmax of
-// block t+1).  The running max lives in the log2 domain; exponentials start against the max of the
-// earlier blocks and the O accumulator is rescaled only when the max grows by more than 2^8.
+// Per tile, S = Q K^T (128x64xd, operands in shared memory) of block t lands in TMEM score
+// buffer t & 1; the softmax warps copy it to registers and write P = exp2(.), as bf16, over the
+// first half of the same buffer, which O += P V then reads.  The scores of block t + 1 go to the
+// other buffer as soon as the P V product of block t - 1 has read it, so both products of the
+// neighbouring blocks overlap the softmax of block t.  The running max lives in the log2 domain;
+// exponentials start against the max of the earlier blocks and the O accumulator is rescaled only
+// when the max grows by more than 2^8.
 // The two products of a tile have their own issuing threads: each walks the merged list,
 // waits only for what its next MMA series needs (so it reacts as soon as that arrives), and
 // releases the ring stages of the other tile's blocks, always after waiting for the stage to
