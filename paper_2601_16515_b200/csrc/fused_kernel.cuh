@@ -419,15 +419,16 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 mxa = fmaxf(mxa, fmaxf(x[4 * n], x[4 * n + 1]));
                 mxb = fmaxf(mxb, fmaxf(x[4 * n + 2], x[4 * n + 3]));
             }
-            const float msa = quad_max(mxa) * p.scale_log2, msb = quad_max(mxb) * p.scale_log2;
-            // The running max only moves when it grows by more than 2^8: then the accumulator of this
-            // warp's rows is brought to the new max, once the previous P V product has landed in it.
-            // pv_done[b] completes a phase for every second block; the product of block t cannot be
-            // issued before this warp hands over P of block t, so the barrier is at most one phase
-            // past the one tested here and the parity test is exact.
+            // The running max only moves when it grows by more than 2^8 (checked on the threads' own
+            // columns first: the shuffles that form the row maxima are needed only then).  The accumulator
+            // of this warp's rows is then brought to the new max, once the previous P V product has
+            // landed in it.  pv_done[b] completes a phase for every second block; the product of block t
+            // cannot be issued before this warp hands over P of block t, so the barrier is at most one
+            // phase past the one tested here and the parity test is exact.
             if (t == 0) {
-                m_a = msa; m_b = msb;
-            } else if (__any_sync(0xffffffffu, msa > m_a + 8.0f || msb > m_b + 8.0f)) {
+                m_a = quad_max(mxa) * p.scale_log2; m_b = quad_max(mxb) * p.scale_log2;
+            } else if (__any_sync(0xffffffffu, mxa * p.scale_log2 > m_a + 8.0f || mxb * p.scale_log2 > m_b + 8.0f)) {
+                const float msa = quad_max(mxa) * p.scale_log2, msb = quad_max(mxb) * p.scale_log2;
                 ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
