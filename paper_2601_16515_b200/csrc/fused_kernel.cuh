@@ -54,7 +54,6 @@ enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
 
 struct FusedParams {
     int N, H, nQb, nKb, nPairs, Bq, Hm, mode;
-    int head_major_ranks;        // ranks below this run head by head, the rest rank by rank across the heads
     const int32_t* row_ptr;
     const int32_t* col_idx;
     const int32_t* order;        // [Hm][nPairs] launch order of the query-block pairs, or null (identity)
@@ -139,20 +138,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     grid_dependency_wait();           // the order and the linear state come from the kernels before
     grid_launch_dependents();
 
-    // Work item.  Most of the launch goes head by head (K/V of one head stay hot in L2), inside a head
-    // from the most to the least expensive pair of query blocks.  The cheapest pairs of ALL heads come
-    // last, rank by rank across the heads, so that the final, partly filled wave of the launch is made
-    // of the shortest items there are.
-    int rank, bh;
-    {
-        const long long major = (long long)p.head_major_ranks * p.BH;
-        if (blockIdx.x < major) {
-            rank = blockIdx.x % p.head_major_ranks; bh = blockIdx.x / p.head_major_ranks;
-        } else {
-            const long long idx = blockIdx.x - major;
-            rank = p.head_major_ranks + int(idx / p.BH); bh = int(idx % p.BH);
-        }
-    }
+    // work item: head by head (K/V of one head stay hot in L2: ordering the cheapest items of all
+    // heads last instead was measured to shorten the launch by 0.3 % and to raise its DRAM traffic by
+    // half), within a head the pairs of query blocks from the most to the least expensive, so that
+    // the kernel ends on short items
+    const int rank = blockIdx.x % p.nPairs, bh = blockIdx.x / p.nPairs;
     const int h = bh % p.H, b = bh / p.H;
     const int hm = (p.Hm == 1) ? 0 : (p.Hm == p.H ? h : bh);   // one mask, one per head, or one per (batch, head)
     const int pair = p.order ? __ldg(p.order + size_t(hm) * p.nPairs + rank) : rank;

@@ -185,7 +185,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
 }
 
 template <int D>
-int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
+int launch_fused(const Problem& P, const Workspace& w) {
     const int BH = P.B * P.H;
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
     CUtensorMap mq, mk, mv, mo, ms;
@@ -198,12 +198,6 @@ int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     fp.nQb = (P.N + P.Bq - 1) / P.Bq;
     fp.nKb = (P.N + 63) / 64;
     fp.nPairs = (fp.nQb + 1) / 2;
-    {
-        // about two waves of the cheapest items of all heads form the tail of the launch
-        int tail = (2 * dev.sms + BH - 1) / BH;
-        if (tail > fp.nPairs) tail = fp.nPairs;
-        fp.head_major_ranks = (P.mode & MODE_SPARSE) ? fp.nPairs - tail : fp.nPairs;
-    }
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
     fp.BH = BH;
     fp.order = nullptr;
@@ -280,7 +274,7 @@ int run(const Problem& P) {
         if (rc != SALAD_OK) return rc;
     }
     if (P.mode == MODE_LINEAR) return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
-    return (P.d == 128) ? launch_fused<128>(P, w, dev) : launch_fused<64>(P, w, dev);
+    return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }
 
 // ---------------------------------------------------------------------------------------
