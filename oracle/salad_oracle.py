@@ -208,3 +208,32 @@ def topk_mask(q, k, Bq, Bk, topk, return_scores=False):
                          scores.ctypes.data if return_scores else None)
     row_ptr = (np.arange(rows + 1, dtype=np.int64) * kk).astype(np.int32)
     return (row_ptr, col_idx, scores) if return_scores else (row_ptr, col_idx)
+
+
+def temporal_order(grid):
+    """Appendix A.1 token permutation for heads with temporal locality: the flattening with time
+    slowest, n = t*(Hs*Ws) + s, is replaced by one that groups tokens by spatial location, so that
+    temporal neighbours are consecutive.  Returns perm with perm[m] = n: position m of the
+    permuted sequence holds original token n, m = s*T + t."""
+    T, Hs, Ws = grid
+    S = Hs * Ws
+    perm = np.empty(T * S, dtype=np.int64)
+    for s in range(S):
+        for t in range(T):
+            perm[s * T + t] = t * S + s
+    return perm
+
+
+def permute_tokens(x, grid, head_flags, inverse=False):
+    """x [B, H, N, d].  Heads with a non-zero flag are re-ordered along the token axis by
+    temporal_order (forward: y[m] = x[perm[m]]; inverse: y[perm[m]] = x[m]); the others are copied."""
+    x = np.asarray(x)
+    perm = temporal_order(grid)
+    y = x.copy()
+    for h, flag in enumerate(head_flags):
+        if flag:
+            if inverse:
+                y[:, h, perm] = x[:, h]
+            else:
+                y[:, h] = x[:, h, perm]
+    return y

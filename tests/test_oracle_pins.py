@@ -433,3 +433,43 @@ def test_sparse_attn_with_per_batch_and_head_masks():
             x = q[b, h].astype(np.float64) @ k[b, h].astype(np.float64).T / np.sqrt(d) + M
             p = np.exp(x - x.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
             np.testing.assert_allclose(out[b, h], p @ v[b, h].astype(np.float64), rtol=1e-10, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- temporal-head permutation
+
+def test_temporal_order_hand_example_and_inverse():
+    # T = 2 frames of a 1 x 3 grid: tokens (t, s) = 0:(0,0) 1:(0,1) 2:(0,2) 3:(1,0) 4:(1,1) 5:(1,2);
+    # grouped by spatial location: (0,0) (1,0) (0,1) (1,1) (0,2) (1,2) = tokens 0 3 1 4 2 5
+    assert orc.temporal_order((2, 1, 3)).tolist() == [0, 3, 1, 4, 2, 5]
+    rng = np.random.default_rng(5)
+    grid = (3, 2, 4)
+    x = rng.standard_normal((2, 3, 24, 4)).astype(np.float32)
+    flags = [1, 0, 1]
+    y = orc.permute_tokens(x, grid, flags)
+    assert np.array_equal(y[:, 1], x[:, 1])                                  # unflagged head untouched
+    assert not np.array_equal(y[:, 0], x[:, 0])
+    assert np.array_equal(orc.permute_tokens(y, grid, flags, inverse=True), x)
+    # temporal neighbours become adjacent: positions m, m+1 (same s) are one frame apart
+    perm = orc.temporal_order(grid)
+    S = grid[1] * grid[2]
+    d = np.diff(perm.reshape(S, grid[0]), axis=1)
+    assert (d == S).all()
+
+
+def test_attention_commutes_with_the_permutation():
+    # attention is equivariant under a joint re-ordering of the tokens of Q, K, V: dense attention
+    # on the permuted tensors, un-permuted, equals dense attention on the originals
+    grid = (4, 2, 4)
+    B, H, N, d = 1, 2, 32, 8
+    q, k, v = rand_qkv(B, H, N, d, 91)
+    flags = [1, 1]
+    qp, kp, vp = (orc.permute_tokens(t, grid, flags) for t in (q, k, v))
+    rp, ci = wlmod.dense_csr(2, 2, 1)
+    o_perm = orc.sparse_attn(qp, kp, vp, 16, 16, rp, ci, 1)[0].reshape(B, H, N, d)
+    o_ref = orc.sparse_attn(q, k, v, 16, 16, rp, ci, 1)[0].reshape(B, H, N, d)
+    np.testing.assert_allclose(orc.permute_tokens(o_perm, grid, flags, inverse=True), o_ref, rtol=1e-12, atol=1e-14)
+    # and the 1-D window on the permuted order reaches temporal neighbours the same window misses on
+    # the original order: token (t, s) and (t+1, s) are 1 apart after, Hs*Ws apart before
+    perm = orc.temporal_order(grid)
+    pos = np.empty_like(perm); pos[perm] = np.arange(len(perm))
+    assert abs(pos[0 * 8 + 3] - pos[1 * 8 + 3]) == 1
