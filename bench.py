@@ -326,6 +326,14 @@ def main():
                                    "achieved_gbs": x_bytes / (dyn_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
                                    "frac": x_bytes / (dyn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del xt
+        # temporal-head permutation (App. A.1): one read and one write of a [B,H,N,d] tensor
+        flags = [1] * wl.H
+        perm_out = torch.empty_like(q)
+        perm_ms = timed(lambda: salad.salad_permute_tokens(q, wl.grid, flags, out=perm_out), 20)
+        extras["permute_tokens"] = {"ms": perm_ms, "algorithmic_bytes": 2 * tensor_bytes,
+                                    "achieved_gbs": 2 * tensor_bytes / (perm_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                                    "frac": 2 * tensor_bytes / (perm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del perm_out
         # Top-K mask producer (App. A.1 steps 1-2) at this shape, k chosen for the same 90 % sparsity:
         # block means read Q and K once (the HBM-bound part), then scores and selection
         topk = max(1, round(wl.nKb * (1.0 - sparsity)))

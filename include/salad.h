@@ -177,6 +177,21 @@ int salad_topk_mask_build(const void* q, const void* k, int B, int H, int N, int
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * salad_permute_tokens -- the token re-ordering of Appendix A.1 for heads with temporal locality.
+ * Tokens arrive flattened with time slowest, n = t*(Hs*Ws) + s; a flagged head is re-ordered to
+ * m = s*T + t (tokens grouped by spatial location, temporal neighbours adjacent), so that a 1-D
+ * sliding-window mask (salad_mask_build on the grid 1 x 1 x N) captures temporal locality:
+ *     inverse == 0:  y[b,h,m,:] = x[b,h,n,:]        inverse != 0:  y[b,h,n,:] = x[b,h,m,:]
+ * Heads whose flag is 0 are copied unchanged.  Use: permute Q, K, V, run an attention entry
+ * point with per-head 1-D windows, permute O back with inverse = 1.
+ *   x, y           bf16 [B, H, N, d], N == T*Hs*Ws, d in {64, 128}; y must not alias x.
+ *   h_head_flags   HOST int32 [H]; H <= 1024.
+ * HBM-bound (one read and one write of the tensor); asynchronous on `stream`.
+ */
+int salad_permute_tokens(const void* x, void* y, int B, int H, int N, int d, int T, int Hs, int Ws,
+                         const int32_t* h_head_flags, int inverse, void* stream);
+
+/*
  * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide
  * scratch memory (the paper has no counterpart; this is a deployment convenience).
  * Some hosts of this library may not call cudaMalloc at the point where attention runs: a

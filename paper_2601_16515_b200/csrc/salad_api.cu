@@ -11,6 +11,7 @@
 #include "linear_apply_kernel.cuh"
 #include "linear_state_kernel.cuh"
 #include "mask_kernels.cuh"
+#include "permute_kernel.cuh"
 #include "tmap.cuh"
 #include "topk_mask_kernels.cuh"
 
@@ -550,6 +551,25 @@ SALAD_EXPORT int salad_topk_mask_build(const void* q, const void* k, int B, int 
         launch_dependent(topk_pick_kernel<32>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
     else
         launch_dependent(topk_pick_kernel<0>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+    return check_launch();
+}
+
+SALAD_EXPORT int salad_permute_tokens(const void* x, void* y, int B, int H, int N, int d, int T, int Hs, int Ws,
+                                      const int32_t* h_head_flags, int inverse, void* stream) {
+    if (!x || !y || x == y || !h_head_flags || B <= 0 || H <= 0 || N <= 0 || T <= 0 || Hs <= 0 || Ws <= 0)
+        return SALAD_ERR_INVALID_ARG;
+    if (int64_t(T) * Hs * Ws != N) return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return SALAD_ERR_INVALID_ARG;
+    if ((d != 64 && d != 128) || H > kPermuteMaxHeads || int64_t(B) * H > 65535) return SALAD_ERR_UNSUPPORTED;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    PermuteParams pp{};
+    pp.N = N; pp.T = T; pp.S = Hs * Ws; pp.H = H; pp.vec_per_row = d / 8; pp.inverse = inverse ? 1 : 0;
+    for (int h = 0; h < H; ++h)
+        if (h_head_flags[h]) pp.flag_bits[h >> 5] |= 1u << (h & 31);
+    permute_tokens_kernel<<<dim3(unsigned((N + kPermuteRows - 1) / kPermuteRows), unsigned(B * H)), kPermuteThreads, 0,
+                            static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(x), static_cast<uint4*>(y), pp);
     return check_launch();
 }
 

@@ -27,7 +27,7 @@ SALAD_ERR_TIMEOUT = -6
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
-           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build")
+           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens")
 
 
 class SaladError(RuntimeError):
@@ -65,6 +65,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_topk_workspace_bytes.argtypes = [i32] * 6
     lib.salad_topk_mask_build.restype = i32
     lib.salad_topk_mask_build.argtypes = [p, p] + [i32] * 7 + [p, p, ctypes.c_int64, p, sz, p]
+    lib.salad_permute_tokens.restype = i32
+    lib.salad_permute_tokens.argtypes = [p, p] + [i32] * 7 + [p, i32, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -235,6 +237,23 @@ def salad_topk_mask_build(q, k, topk: int, Bq: int = 128, Bk: int = 64, row_ptr=
                                           _ptr(col_idx), col_idx.numel(), _ptr(workspace), workspace.numel(),
                                           _stream(stream)), "salad_topk_mask_build")
     return row_ptr, col_idx[:rows * kk]
+
+
+def salad_permute_tokens(x, grid, head_flags, inverse: bool = False, out=None, stream=None):
+    """Re-order the tokens of the flagged heads from time-slowest to grouped-by-spatial-location order
+    (inverse=True: back).  x bf16 [B,H,N,d]; grid = (T, Hs, Ws); head_flags: H ints."""
+    _bf16_4d("x", x)
+    B, H, N, d = x.shape
+    T, Hs, Ws = grid
+    flags = (ctypes.c_int32 * H)(*[int(bool(f)) for f in head_flags])
+    if len(head_flags) != H:
+        raise ValueError("head_flags must have one entry per head")
+    if out is None:
+        out = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        _check(_lib.salad_permute_tokens(_ptr(x), _ptr(out), B, H, N, d, T, Hs, Ws, flags, int(bool(inverse)),
+                                         _stream(stream)), "salad_permute_tokens")
+    return out
 
 
 DYN_SCALE_WS_BYTES = 8192

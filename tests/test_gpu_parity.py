@@ -503,3 +503,38 @@ def test_topk_mask_capacity_and_arguments(salad):
     with pytest.raises(salad.SaladError) as e:
         salad.salad_topk_mask_build(q.cuda(), k.cuda(), 0, Bq=64)
     assert e.value.code == salad.SALAD_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------------------ temporal-head permutation
+
+@pytest.mark.parametrize("B,H,grid,d", [(2, 3, (5, 6, 7), 128), (1, 2, (4, 16, 16), 64), (1, 4, (21, 9, 13), 128)])
+def test_permute_tokens_bit_exact(salad, B, H, grid, d):
+    N = grid[0] * grid[1] * grid[2]
+    x, _, _ = rand_qkv(B, H, N, d, 300 + N)
+    flags = [(h % 2) == 0 for h in range(H)]
+    y = salad.salad_permute_tokens(x.cuda(), grid, flags)
+    ref = orc.permute_tokens(f32(x), grid, flags)
+    assert np.array_equal(f32(y.cpu()), ref)
+    back = salad.salad_permute_tokens(y, grid, flags, inverse=True)
+    assert torch.equal(back.cpu(), x)
+
+
+def test_permuted_sliding_window_pipeline(salad):
+    # The paper's ST-SWA: temporal heads are re-ordered, every head then gets a 1-D sliding window,
+    # the output goes back to the original order.  Device pipeline against the oracle's.
+    grid = (8, 8, 16)                     # N = 1024
+    B, H, N, d, Bq = 1, 4, 1024, 128, 128
+    q, k, v = rand_qkv(B, H, N, d, 55)
+    flags = [1, 0, 1, 0]                  # heads 0 and 2 temporal
+    windows = [(0, 0, 64), (0, 0, 200), (0, 0, 24), (0, 0, 130)]       # 1-D half-widths per head
+    lam = np.array([0.5, 0.1, 0.9, 0.3], dtype=np.float32); s = np.array([0.4], dtype=np.float32)
+    qd, kd, vd = (salad.salad_permute_tokens(t.cuda(), grid, flags) for t in (q, k, v))
+    rp, ci = salad.salad_mask_build(1, 1, N, Bq, 64, windows)
+    out_p = salad.salad_fused_fwd(qd, kd, vd, rp, ci, H, torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda(), Bq=Bq)
+    out = salad.salad_permute_tokens(out_p, grid, flags, inverse=True)
+    qo, ko, vo = (orc.permute_tokens(f32(t), grid, flags) for t in (q, k, v))
+    rp_o, ci_o = orc.mask_build(1, 1, N, Bq, 64, windows)
+    assert np.array_equal(rp.cpu().numpy(), rp_o) and np.array_equal(ci.cpu().numpy(), ci_o)
+    ref_p = orc.salad_fused(qo, ko, vo, Bq, 64, rp_o, ci_o, H, lam.astype(np.float64), s.astype(np.float64))
+    ref = orc.permute_tokens(ref_p.reshape(B, H, N, d), grid, flags, inverse=True)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "permuted ST-SWA")
