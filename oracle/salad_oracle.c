@@ -354,3 +354,35 @@ ORACLE_API void oracle_topk_mask(const float* q, const float* k, int B, int H, i
         free(kbar); free(s); free(taken);
     }
 }
+
+/*
+ * oracle_proj_combine: Algorithm 1, Level 1 and the residual integration, with the full projection:
+ *     O'_l = Proj(O_l)        a linear layer on the head-concatenated linear-branch output
+ *                             (D = H*d channels in, D out; zero-initialised before tuning, Sec. 4.2),
+ *     O~   = O_s + s * O'_l   (s the dynamic scale of the batch item; Eq. 5's lambda is a further
+ *                             scalar on the same term and can be folded into s).
+ * Layouts: o_s, o_l, out [B, H, N, d]; channel j = h*d + c of the concatenation.
+ *   w     [D][D], w[j_out][j_in]      (y = x W^T, the usual linear-layer storage)
+ *   bias  [D] or NULL
+ *   s_b   [B]
+ */
+ORACLE_API void oracle_proj_combine(const float* o_s, const float* o_l, const float* w, const float* bias,
+                                    const double* s_b, int B, int H, int N, int d, double* out)
+{
+    int D = H * d;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b) {
+        for (int n = 0; n < N; ++n) {
+            for (int jo = 0; jo < D; ++jo) {
+                double acc = bias ? (double)bias[jo] : 0.0;
+                for (int h = 0; h < H; ++h) {
+                    const float* x = o_l + (((int64_t)b * H + h) * N + n) * (int64_t)d;
+                    const float* wr = w + (int64_t)jo * D + (int64_t)h * d;
+                    for (int c = 0; c < d; ++c) acc += (double)x[c] * (double)wr[c];
+                }
+                int64_t idx = (((int64_t)b * H + jo / d) * N + n) * (int64_t)d + jo % d;
+                out[idx] = (double)o_s[idx] + s_b[b] * acc;
+            }
+        }
+    }
+}

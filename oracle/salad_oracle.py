@@ -53,6 +53,8 @@ def _load():
         lib.oracle_salad_fused_drop.restype = None
         lib.oracle_salad_fused_drop.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
                                                                          p, i64, p])
+        lib.oracle_proj_combine.restype = None
+        lib.oracle_proj_combine.argtypes = [p, p, p, p, p, i32, i32, i32, i32, p]
         lib.oracle_topk_mask.restype = None
         lib.oracle_topk_mask.argtypes = [p, p] + [i32] * 7 + [p, p]
         _lib = lib
@@ -237,3 +239,20 @@ def permute_tokens(x, grid, head_flags, inverse=False):
             else:
                 y[:, h] = x[:, h, perm]
     return y
+
+
+def proj_combine(o_s, o_l, w, s_b, bias=None):
+    """Algorithm 1 with the full projection: O_s + s_b * Proj(O_l), Proj a D x D linear layer on the
+    head-concatenated O_l (w[j_out, j_in], optional bias).  o_s, o_l [B,H,N,d] -> [B,H,N,d] float64."""
+    lib = _load()
+    o_s, sp = _f32(o_s); o_l, lp = _f32(o_l); w, wp = _f32(w)
+    B, H, N, d = o_s.shape
+    assert o_l.shape == o_s.shape and w.shape == (H * d, H * d)
+    sb = np.ascontiguousarray(s_b, dtype=np.float64); assert sb.size == B
+    if bias is not None:
+        bias, bp = _f32(bias); assert bias.size == H * d
+    else:
+        bp = None
+    out = np.empty((B, H, N, d), dtype=np.float64)
+    lib.oracle_proj_combine(sp, lp, wp, bp, sb.ctypes.data, B, H, N, d, out.ctypes.data)
+    return out

@@ -473,3 +473,48 @@ def test_attention_commutes_with_the_permutation():
     perm = orc.temporal_order(grid)
     pos = np.empty_like(perm); pos[perm] = np.arange(len(perm))
     assert abs(pos[0 * 8 + 3] - pos[1 * 8 + 3]) == 1
+
+
+# ----------------------------------------------------------------------------- full projection (Alg. 1 level 1)
+
+def test_proj_combine_pins():
+    rng = np.random.default_rng(101)
+    B, H, N, d = 2, 3, 37, 8
+    D = H * d
+    o_s = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    o_l = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    w = (rng.standard_normal((D, D)) * 0.2).astype(np.float32)
+    bias = rng.standard_normal(D).astype(np.float32)
+    s = np.array([0.3, 0.8])
+    got = orc.proj_combine(o_s, o_l, w, s, bias)
+    # the definition with library routines: concatenate heads, y = x W^T + b, split heads again
+    x = np.transpose(o_l.astype(np.float64), (0, 2, 1, 3)).reshape(B, N, D)
+    y = x @ w.astype(np.float64).T + bias.astype(np.float64)
+    y = np.transpose(y.reshape(B, N, H, d), (0, 2, 1, 3))
+    np.testing.assert_allclose(got, o_s + s[:, None, None, None] * y, rtol=1e-12, atol=1e-13)
+    # zero-initialised layer: the sparse branch exactly (the starting point of tuning, Sec. 4.2)
+    assert np.array_equal(orc.proj_combine(o_s, o_l, np.zeros((D, D), np.float32), s), o_s.astype(np.float64))
+    # identity: the plain residual sum
+    np.testing.assert_allclose(orc.proj_combine(o_s, o_l, np.eye(D, dtype=np.float32), s),
+                               o_s + s[:, None, None, None] * o_l.astype(np.float64), rtol=1e-14)
+    # a matrix that moves head 1 to head 0 and nothing else
+    w2 = np.zeros((D, D), np.float32); w2[0:d, d:2 * d] = np.eye(d)
+    out2 = orc.proj_combine(o_s, o_l, w2, np.ones(B))
+    np.testing.assert_allclose(out2[:, 0], o_s[:, 0].astype(np.float64) + o_l[:, 1], rtol=1e-14)
+    assert np.array_equal(out2[:, 1:], o_s[:, 1:].astype(np.float64))
+
+
+def test_proj_combine_block_diagonal_is_the_fused_path():
+    # Proj = blockdiag(lambda_h I_d) turns the full projection into the per-head static scale of the
+    # fused call: O_s + s_b * lambda_h * O_l
+    B, H, N, d = 2, 2, 64, 16
+    q, k, v = rand_qkv(B, H, N, d, 103)
+    rp, ci = wlmod.dense_csr(4, 4, 1)
+    lam = np.array([0.7, 0.2]); s = np.array([0.4, 0.9])
+    o_s = orc.sparse_attn(q, k, v, 16, 16, rp, ci, 1)[0].reshape(B, H, N, d)
+    o_l = orc.linear_attn(q, k, v).reshape(B, H, N, d)
+    w = np.kron(np.diag(lam), np.eye(d))
+    got = orc.proj_combine(o_s, o_l, w, s)
+    # o_s and o_l pass through fp32 in the wrapper: compare at that precision
+    ref = orc.salad_fused(q, k, v, 16, 16, rp, ci, 1, lam, s).reshape(B, H, N, d)
+    np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
