@@ -326,6 +326,16 @@ def main():
                                    "achieved_gbs": x_bytes / (dyn_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
                                    "frac": x_bytes / (dyn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del xt
+        # full D x D projection of the linear branch + residual sum (Alg. 1 level 1): a tensor-core GEMM
+        Dm = wl.H * wl.d
+        w_proj = (torch.randn(Dm, Dm, device=dev) / Dm ** 0.5).to(torch.bfloat16)
+        o_l_buf = torch.randn_like(q)
+        proj_out = torch.empty_like(q)
+        proj_ms = timed(lambda: salad.salad_proj_combine_fwd(out, o_l_buf, w_proj, s_d, out=proj_out), 10)
+        proj_flops = 2.0 * wl.B * wl.N * Dm * Dm
+        extras["proj_combine"] = {"ms": proj_ms, "tflops": proj_flops / (proj_ms * 1e-3) / 1e12,
+                                  "frac_of_measured_bf16_peak": proj_flops / (proj_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        del w_proj, o_l_buf, proj_out
         # temporal-head permutation (App. A.1): one read and one write of a [B,H,N,d] tensor
         flags = [1] * wl.H
         perm_out = torch.empty_like(q)

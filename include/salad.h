@@ -192,6 +192,24 @@ int salad_permute_tokens(const void* x, void* y, int B, int H, int N, int d, int
                          const int32_t* h_head_flags, int inverse, void* stream);
 
 /*
+ * salad_proj_combine_fwd -- Algorithm 1 with the full Level-1 projection (Sec. 4.2): a linear layer
+ * on the head-concatenated output of the linear branch (zero-initialised before tuning), scaled by
+ * the dynamic factor and added to the sparse branch,
+ *     out[b, :, n, :] = O_s[b, :, n, :] + d_dyn_scale[b] * ( concat_h O_l[b, h, n, :] . W^T + bias ).
+ * salad_fused_fwd covers the case W = blockdiag(lambda_h I) in one pass over Q, K, V; a projection
+ * that mixes heads needs the two branch outputs first: salad_sparse_attn_fwd -> O_s,
+ * salad_linear_attn_fwd -> O_l, then this call (a [B*N x D] x [D x D] tensor-core GEMM, D = H*d,
+ * with the sum fused into its epilogue).
+ *   o_s, o_l, out  bf16 [B, H, N, d], d in {64, 128}.  out may alias o_s, not o_l.
+ *   w              bf16 [D][D], w[j_out][j_in], channel j = h*d + c (device).
+ *   d_bias         fp32 [D] or NULL;   d_dyn_scale fp32 [B] or NULL (= 1).
+ * Allocates nothing, needs no workspace.  fp32 accumulation, one rounding to bf16.
+ */
+int salad_proj_combine_fwd(const void* o_s, const void* o_l, const void* w, const float* d_bias,
+                           const float* d_dyn_scale, void* out, int B, int H, int N, int d,
+                           int32_t* d_status, void* stream);
+
+/*
  * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide
  * scratch memory (the paper has no counterpart; this is a deployment convenience).
  * Some hosts of this library may not call cudaMalloc at the point where attention runs: a

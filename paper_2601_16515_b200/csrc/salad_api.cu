@@ -12,6 +12,7 @@
 #include "linear_state_kernel.cuh"
 #include "mask_kernels.cuh"
 #include "permute_kernel.cuh"
+#include "proj_gemm_kernel.cuh"
 #include "tmap.cuh"
 #include "topk_mask_kernels.cuh"
 
@@ -570,6 +571,48 @@ SALAD_EXPORT int salad_permute_tokens(const void* x, void* y, int B, int H, int 
         if (h_head_flags[h]) pp.flag_bits[h >> 5] |= 1u << (h & 31);
     permute_tokens_kernel<<<dim3(unsigned((N + kPermuteRows - 1) / kPermuteRows), unsigned(B * H)), kPermuteThreads, 0,
                             static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(x), static_cast<uint4*>(y), pp);
+    return check_launch();
+}
+
+SALAD_EXPORT int salad_proj_combine_fwd(const void* o_s, const void* o_l, const void* w, const float* d_bias,
+                                        const float* d_dyn_scale, void* out, int B, int H, int N, int d,
+                                        int32_t* d_status, void* stream) {
+    if (!o_s || !o_l || !w || !out || B <= 0 || H <= 0 || N <= 0 || d <= 0) return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(o_s) || !aligned16(o_l) || !aligned16(w) || !aligned16(out)) return SALAD_ERR_INVALID_ARG;
+    if (out == o_l) return SALAD_ERR_INVALID_ARG;                 // the activation is re-read by other tiles
+    if (d != 64 && d != 128) return SALAD_ERR_UNSUPPORTED;
+    if (int64_t(B) * H > 65535 || int64_t(H) * d > 65536) return SALAD_ERR_UNSUPPORTED;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    static bool smem_set[64] = {};
+    int devi = 0;
+    cudaGetDevice(&devi);
+    if (devi >= 0 && devi < 64 && !smem_set[devi]) {
+        if (cudaFuncSetAttribute(salad_proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 ProjCfg::SMEM_BYTES) != cudaSuccess) {
+            cudaGetLastError();
+            return SALAD_ERR_CUDA;
+        }
+        smem_set[devi] = true;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (d_status && cudaMemsetAsync(d_status, 0, sizeof(int32_t), st) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
+    const int D = H * d;
+    CUtensorMap ma, mw;
+    if (!make_tmap_bf16_3d(&ma, o_l, d, N, int64_t(B) * H, ProjCfg::BM) || !make_tmap_bf16_3d(&mw, w, D, D, 1, ProjCfg::BN))
+        return SALAD_ERR_CUDA;
+    ProjParams pp;
+    pp.B = B; pp.H = H; pp.N = N; pp.d = d; pp.D = D;
+    pp.nMt = (N + ProjCfg::BM - 1) / ProjCfg::BM;
+    pp.nNt = (D + ProjCfg::BN - 1) / ProjCfg::BN;
+    pp.ksteps = D / ProjCfg::BK;
+    pp.tiles = (long long)B * pp.nMt * pp.nNt;
+    pp.o_s = static_cast<const __nv_bfloat16*>(o_s);
+    pp.out = static_cast<__nv_bfloat16*>(out);
+    pp.bias = d_bias; pp.s_b = d_dyn_scale; pp.status = d_status;
+    const unsigned grid = unsigned(pp.tiles < dev.sms ? pp.tiles : dev.sms);
+    salad_proj_gemm_kernel<<<grid, ProjCfg::THREADS, ProjCfg::SMEM_BYTES, st>>>(ma, mw, pp);
     return check_launch();
 }
 

@@ -27,7 +27,7 @@ SALAD_ERR_TIMEOUT = -6
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
-           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens")
+           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd")
 
 
 class SaladError(RuntimeError):
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_topk_mask_build.argtypes = [p, p] + [i32] * 7 + [p, p, ctypes.c_int64, p, sz, p]
     lib.salad_permute_tokens.restype = i32
     lib.salad_permute_tokens.argtypes = [p, p] + [i32] * 7 + [p, i32, p]
+    lib.salad_proj_combine_fwd.restype = i32
+    lib.salad_proj_combine_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -253,6 +255,26 @@ def salad_permute_tokens(x, grid, head_flags, inverse: bool = False, out=None, s
     with torch.cuda.device(x.device):
         _check(_lib.salad_permute_tokens(_ptr(x), _ptr(out), B, H, N, d, T, Hs, Ws, flags, int(bool(inverse)),
                                          _stream(stream)), "salad_permute_tokens")
+    return out
+
+
+def salad_proj_combine_fwd(o_s, o_l, w, dyn_scale=None, bias=None, out=None, status=None, stream=None):
+    """out = O_s + dyn_scale[b] * (concat_heads(O_l) @ w.T + bias), all [B,H,N,d] bf16; w bf16 [D,D]."""
+    _bf16_4d("o_s", o_s); _bf16_4d("o_l", o_l)
+    if o_s.shape != o_l.shape:
+        raise ValueError("o_s and o_l must have the same shape")
+    B, H, N, d = o_s.shape
+    D = H * d
+    if w.dtype != torch.bfloat16 or not w.is_cuda or not w.is_contiguous() or tuple(w.shape) != (D, D):
+        raise ValueError("w must be a contiguous CUDA bf16 tensor [H*d, H*d]")
+    for name, t, n in (("dyn_scale", dyn_scale, B), ("bias", bias, D)):
+        if t is not None and (t.dtype != torch.float32 or not t.is_cuda or t.numel() != n or not t.is_contiguous()):
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor with {n} elements")
+    if out is None:
+        out = torch.empty_like(o_s)
+    with torch.cuda.device(o_s.device):
+        _check(_lib.salad_proj_combine_fwd(_ptr(o_s), _ptr(o_l), _ptr(w), _ptr(bias), _ptr(dyn_scale), _ptr(out),
+                                           B, H, N, d, _ptr(status), _stream(stream)), "salad_proj_combine_fwd")
     return out
 
 

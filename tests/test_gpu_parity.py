@@ -538,3 +538,51 @@ def test_permuted_sliding_window_pipeline(salad):
     ref_p = orc.salad_fused(qo, ko, vo, Bq, 64, rp_o, ci_o, H, lam.astype(np.float64), s.astype(np.float64))
     ref = orc.permute_tokens(ref_p.reshape(B, H, N, d), grid, flags, inverse=True)
     assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "permuted ST-SWA")
+
+
+# ------------------------------------------------------------------------------ full projection (Alg. 1 level 1)
+
+@pytest.mark.parametrize("B,H,N,d,with_bias", [
+    (1, 2, 300, 128, True),        # one output tile, ragged token tile
+    (2, 3, 1000, 128, False),      # D = 384: the second column tile is half empty
+    (1, 12, 520, 64, True),        # D = 768, four heads per column tile
+    (1, 12, 2048, 128, True),      # the 1.3B width, several tiles per SM none
+])
+def test_proj_combine(salad, B, H, N, d, with_bias):
+    rng = np.random.default_rng(500 + N)
+    D = H * d
+    o_s = bf16(rng.standard_normal((B, H, N, d))); o_l = bf16(rng.standard_normal((B, H, N, d)))
+    w = bf16(rng.standard_normal((D, D)) / np.sqrt(D))
+    bias = torch.from_numpy(rng.standard_normal(D).astype(np.float32)) if with_bias else None
+    s = torch.from_numpy(rng.uniform(0.2, 0.9, B).astype(np.float32))
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_proj_combine_fwd(o_s.cuda(), o_l.cuda(), w.cuda(), s.cuda(),
+                                       bias.cuda() if with_bias else None, status=status)
+    status_ok(status)
+    ref = orc.proj_combine(f32(o_s), f32(o_l), f32(w), s.numpy().astype(np.float64),
+                           bias.numpy() if with_bias else None)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "proj_combine")
+    # in place on O_s, and the zero-initialised layer returns the sparse branch bit for bit
+    buf = o_s.cuda().clone()
+    salad.salad_proj_combine_fwd(buf, o_l.cuda(), w.cuda(), s.cuda(), bias.cuda() if with_bias else None, out=buf)
+    assert torch.equal(buf, out)
+    zero = salad.salad_proj_combine_fwd(o_s.cuda(), o_l.cuda(), torch.zeros_like(w).cuda(), s.cuda())
+    assert torch.equal(zero.cpu(), o_s)
+
+
+def test_full_projection_pipeline_matches_fused_for_block_diagonal(salad):
+    # sparse call + linear call + projection with W = blockdiag(lambda_h I) against the one-pass fused call
+    wl = wlmod.C1
+    q, k, v = wlmod.make_qkv(wl)
+    T, Hs, Ws = wl.grid
+    lam, s = wlmod.make_scales(wl)
+    rp, ci = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    lam_d, s_d = torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda()
+    fused = salad.salad_fused_fwd(qd, kd, vd, rp, ci, len(wl.windows), lam_d, s_d, Bq=wl.Bq, Bk=wl.Bk)
+    o_s = salad.salad_sparse_attn_fwd(qd, kd, vd, rp, ci, len(wl.windows), Bq=wl.Bq, Bk=wl.Bk)
+    o_l = salad.salad_linear_attn_fwd(qd, kd, vd)
+    w = torch.from_numpy(np.kron(np.diag(lam.astype(np.float64)), np.eye(wl.d))).to(torch.bfloat16).cuda()
+    out = salad.salad_proj_combine_fwd(o_s, o_l, w, s_d)
+    # lambda rounded to bf16 in W and O_l rounded to bf16 between the calls: not bit-equal, but close
+    assert_close(f32(out.cpu()).reshape(-1, wl.d), f32(fused.cpu()).reshape(-1, wl.d).astype(np.float64), "pipeline vs fused")
