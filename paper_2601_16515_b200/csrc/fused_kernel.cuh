@@ -564,7 +564,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tma_store_3d(&map_o, s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, ch * 64,
                                  qb[i] * p.Bq, bh);
                 tma_store_commit();
-                tma_store_wait_all();
+                // only the shared-memory source must have been read before the CTA may exit; the
+                // writes are complete, like all of the kernel's, when the grid is
+                tma_store_wait_read_all();
             }
 #ifndef SALAD_TRACE
             if (p.lse != nullptr && q4 == 0) {

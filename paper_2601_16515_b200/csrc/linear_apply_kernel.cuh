@@ -262,7 +262,7 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 }
             }
         }
-        if (row == 0) tma_store_wait_all();
+        if (row == 0) tma_store_wait_read_all();      // the staging tile must outlive the last store's read
     }
     }  // abort_flag == 0
 
