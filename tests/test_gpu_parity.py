@@ -586,3 +586,59 @@ def test_full_projection_pipeline_matches_fused_for_block_diagonal(salad):
     out = salad.salad_proj_combine_fwd(o_s, o_l, w, s_d)
     # lambda rounded to bf16 in W and O_l rounded to bf16 between the calls: not bit-equal, but close
     assert_close(f32(out.cpu()).reshape(-1, wl.d), f32(fused.cpu()).reshape(-1, wl.d).astype(np.float64), "pipeline vs fused")
+
+
+# ------------------------------------------------------------------------------ degenerate sizes
+
+@pytest.mark.parametrize("B,H,N,d,Bq", [
+    (1, 1, 1, 64, 64),          # a single token
+    (1, 2, 63, 128, 128),       # less than one key block
+    (3, 1, 65, 64, 128),        # one token into the second key block
+    (5, 1, 129, 128, 64),       # one row into the third query block, odd number of query blocks
+    (1, 20, 200, 64, 64),       # many heads, short sequence
+])
+def test_fused_degenerate_sizes(salad, B, H, N, d, Bq):
+    q, k, v = rand_qkv(B, H, N, d, 700 + N)
+    nQb, nKb = -(-N // Bq), -(-N // 64)
+    rp, ci = random_csr(nQb, nKb, 3 + N, lo=0, hi=nKb)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = np.linspace(0.2, 0.9, H).astype(np.float32); s = np.linspace(0.3, 0.7, B).astype(np.float32)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, torch.from_numpy(lam).cuda(),
+                                torch.from_numpy(s).cuda(), Bq=Bq, status=status)
+    status_ok(status)
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), Bq, 64, rp, ci, 1, lam.astype(np.float64), s.astype(np.float64))
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "degenerate fused")
+    lin = salad.salad_linear_attn_fwd(q.cuda(), k.cuda(), v.cuda())
+    assert_close(f32(lin.cpu()).reshape(-1, d), orc.linear_attn(f32(q), f32(k), f32(v)), "degenerate linear")
+
+
+def test_fused_with_no_kept_block_at_all_is_the_scaled_linear_branch(salad):
+    B, H, N, d = 1, 2, 640, 128
+    q, k, v = rand_qkv(B, H, N, d, 12)
+    nQb = -(-N // 128)
+    rp = np.zeros(nQb + 1, dtype=np.int32); ci = np.zeros(0, dtype=np.int32)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = np.array([0.5, 0.25], dtype=np.float32); s = np.array([0.5], dtype=np.float32)
+    out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, torch.from_numpy(lam).cuda(),
+                                torch.from_numpy(s).cuda())
+    ref = orc.linear_attn(f32(q), f32(k), f32(v)).reshape(B, H, N, d) * (lam * s[0])[None, :, None, None]
+    assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "linear only through the fused call")
+
+
+def test_long_sequence_linear_and_sparse_band(salad):
+    # 256k tokens of one head: the longest sequence the tests run; a narrow band keeps the oracle cheap
+    B, H, N, d = 1, 1, 262144, 128
+    rng = np.random.default_rng(99)
+    q, k, v = (bf16(rng.standard_normal((B, H, N, d))) for _ in range(3))
+    rp_d, ci_d = salad.salad_mask_build(1, 1, N, 128, 64, [(0, 0, 100)])
+    lam = torch.tensor([0.5], device="cuda"); s = torch.tensor([0.5], device="cuda")
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, lam, s, status=status)
+    status_ok(status)
+    wl = wlmod.Workload("long", B, H, d, (1, 1, N), 128, 64, ((0, 0, 100),), 0)
+    sel = np.concatenate([np.arange(0, 130), np.arange(N - 130, N), wlmod.sample_rows(wl, 300)])
+    ref = orc.salad_fused(f32(q), f32(k), f32(v), 128, 64, rp_d.cpu().numpy(), ci_d.cpu().numpy(), 1,
+                          np.array([0.5]), np.array([0.5]), sel=sel)
+    got = f32(out.cpu()).reshape(-1, d)[sel]
+    assert_close(got, ref, "long sequence")
