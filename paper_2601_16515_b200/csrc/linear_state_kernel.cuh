@@ -68,15 +68,25 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x, bh = blockIdx.y;
-    grid_dependency_wait();
-    grid_launch_dependents();
     if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) return;     // whole CTA, before any allocation
     const int kb0 = chunk * p.blocks_per_chunk;
     const int kb1 = min(p.nKb, kb0 + p.blocks_per_chunk);
     const int nblk = max(0, kb1 - kb0);
 
+    // K and V are inputs of the call, not products of the kernel before this one in the stream: the
+    // producer thread starts the first loads at once, ahead of the set-up below and of the dependency
+    // wait (this kernel is launched so that it may begin while its predecessor still runs).
+    auto load_stage = [&](int g) {
+        const int s = g % C::STAGES;
+        const uint32_t bar = smem_u32(&full[s]);
+        mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+        const uint32_t dst = s_base + s * C::STAGE_BYTES;
+        for (int ch = 0; ch < C::CH; ++ch) {
+            tma_load_3d(dst + ch * C::T_CHUNK, &map_k, bar, ch * 64, (kb0 + g) * C::BK, bh);
+            tma_load_3d(dst + C::T_BYTES + ch * C::T_CHUNK, &map_v, bar, ch * 64, (kb0 + g) * C::BK, bh);
+        }
+    };
     if (tid == 0) {
-        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
             mbar_init(smem_u32(&relu_done[s]), 128);
@@ -84,12 +94,17 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         }
         mbar_init(smem_u32(&acc_done), 1);
         fence_mbar_init();
+        prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+        for (int g = 0; g < min(nblk, C::STAGES); ++g) load_stage(g);
     }
     // all-ones bf16 tile (0x3F80 = 1.0)
     for (int i = tid; i < 2048 / 4; i += C::THREADS)
         reinterpret_cast<uint32_t*>(smem + C::OFF_ONES)[i] = 0x3F803F80u;
     fence_proxy_async_smem();
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
+    grid_dependency_wait();            // the status word is cleared by the kernel before
+    grid_launch_dependents();
+    if (tid == 0) abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -99,17 +114,10 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     if (abort_flag == 0) {
     if (warp == 0) {
         if (lane == 0) {
-            prefetch_tmap(&map_k); prefetch_tmap(&map_v);
-            for (int g = 0; g < nblk; ++g) {
+            for (int g = C::STAGES; g < nblk; ++g) {          // the first STAGES blocks are already on their way
                 const int s = g % C::STAGES;
                 if (!mbar_wait(smem_u32(&empty[s]), ((g / C::STAGES) & 1) ^ 1, abortp)) break;
-                const uint32_t bar = smem_u32(&full[s]);
-                mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-                const uint32_t dst = s_base + s * C::STAGE_BYTES;
-                for (int ch = 0; ch < C::CH; ++ch) {
-                    tma_load_3d(dst + ch * C::T_CHUNK, &map_k, bar, ch * 64, (kb0 + g) * C::BK, bh);
-                    tma_load_3d(dst + C::T_BYTES + ch * C::T_CHUNK, &map_v, bar, ch * 64, (kb0 + g) * C::BK, bh);
-                }
+                load_stage(g);
             }
         }
     } else if (warp == 1) {
