@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <math.h>
 
+#include <mutex>
+
 #include "dynamic_scale_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "linear_apply_kernel.cuh"
@@ -62,10 +64,14 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 struct DeviceInfo { int sms; bool ok; };
 
-// sm_100 check and shared-memory opt-in, once per device.
+// Guards the once-per-device initialisation below (the entry points may be called from several host threads).
+std::mutex g_init_mutex;
+
+// sm_100 check and shared-memory opt-in of every kernel, once per device.
 int prepare_device(DeviceInfo* info) {
     static bool attr_set[64] = {};
     static int sm_count[64] = {};
+    std::lock_guard<std::mutex> lock(g_init_mutex);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
     if (dev < 0 || dev >= 64) return SALAD_ERR_CUDA;
@@ -95,6 +101,12 @@ int prepare_device(DeviceInfo* info) {
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_linear_apply_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      ApplyCfg<64>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(topk_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     128 * (kScoreRows + kScoreTile) * 4);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ProjCfg::SMEM_BYTES);
         if (e != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
         sm_count[dev] = sms;
         attr_set[dev] = true;
@@ -315,6 +327,7 @@ Workspace carve_noalloc(int B, int H, int d) {
 // Device address of g_noalloc_scratch on the current device (looked up on first use).
 int noalloc_scratch_ptr(void** out) {
     static void* cached[64] = {};
+    std::lock_guard<std::mutex> lock(g_init_mutex);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return SALAD_ERR_CUDA; }
     if (!cached[dev]) {
@@ -530,17 +543,6 @@ SALAD_EXPORT int salad_topk_mask_build(const void* q, const void* k, int B, int 
     block_mean_kernel<<<dim3(unsigned(nQb > nKb ? nQb : nKb), unsigned(BH), 2), kMeanThreads, 0, st>>>(jq, jk, N, d);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     const size_t smem = size_t(d) * (kScoreRows + kScoreTile) * 4;          // 80 KB at d = 128
-    static bool smem_set[64] = {};
-    int devi = 0;
-    cudaGetDevice(&devi);
-    if (devi >= 0 && devi < 64 && !smem_set[devi]) {
-        if (cudaFuncSetAttribute(topk_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 160 * 4) !=
-            cudaSuccess) {
-            cudaGetLastError();
-            return SALAD_ERR_CUDA;
-        }
-        smem_set[devi] = true;
-    }
     launch_dependent(topk_score_kernel, dim3(unsigned(ldk / kScoreTile), unsigned((nQb + kScoreRows - 1) / kScoreRows),
                                              unsigned(BH)),
                      dim3(256), smem, st, qmean, kmeanT, int(nQb), int(nKb), ldk, d, score);
@@ -585,17 +587,6 @@ SALAD_EXPORT int salad_proj_combine_fwd(const void* o_s, const void* o_l, const 
     DeviceInfo dev{};
     int rc = prepare_device(&dev);
     if (rc != SALAD_OK) return rc;
-    static bool smem_set[64] = {};
-    int devi = 0;
-    cudaGetDevice(&devi);
-    if (devi >= 0 && devi < 64 && !smem_set[devi]) {
-        if (cudaFuncSetAttribute(salad_proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 ProjCfg::SMEM_BYTES) != cudaSuccess) {
-            cudaGetLastError();
-            return SALAD_ERR_CUDA;
-        }
-        smem_set[devi] = true;
-    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d_status && cudaMemsetAsync(d_status, 0, sizeof(int32_t), st) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
     const int D = H * d;
