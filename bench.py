@@ -348,6 +348,13 @@ def main():
         extras["sparse_only_ms"] = timed(lambda: salad.salad_sparse_attn_fwd(
             q, k, v, rp, ci, Hm, Bq=wl.Bq, Bk=wl.Bk, out=out, workspace=ws), 20)
         extras["linear_only_ms"] = timed(lambda: salad.salad_linear_attn_fwd(q, k, v, out=out, workspace=ws), 20)
+        # the whole linear branch as one call: K, V read (state), Q read and O written (apply)
+        lin_bytes = 4 * q_h.numel() * q_h.element_size()
+        extras["linear_branch"] = {"ms": extras["linear_only_ms"], "algorithmic_bytes": lin_bytes,
+                                   "achieved_gbs": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9,
+                                   "peak_gbs": peaks["hbm_gbs"],
+                                   "frac": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   "frac_of_nominal_8tbs": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9 / 8000.0}
         drp, dci = wlmod.dense_csr(wl.nQb, wl.nKb, 1)
         drp_d, dci_d = torch.from_numpy(drp).to(dev), torch.from_numpy(dci).to(dev)
         dense_ms = timed(lambda: salad.salad_fused_fwd(q, k, v, drp_d, dci_d, 1, lam_d, s_d, Bq=wl.Bq, Bk=wl.Bk,

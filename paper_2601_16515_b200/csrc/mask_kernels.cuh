@@ -104,6 +104,19 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
 // start first and the short ones fill the tail.  Counting sort in shared memory; one CTA per
 // mask head.  The order among equal costs is arbitrary (it only affects scheduling).
 // It is the first kernel of a call, so it also clears the status words the later kernels test.
+// First kernel of a call that has no work-order kernel: clears the status words (and the work-item
+// counter next to the library's).  The kernel after it in the stream is launched so that it can be
+// set up and start its input loads meanwhile.
+__global__ void __launch_bounds__(32) status_clear_kernel(int32_t* __restrict__ ws_status,
+                                                          int32_t* __restrict__ user_status) {
+    grid_launch_dependents();
+    if (threadIdx.x == 0) {
+        ws_status[0] = 0;
+        ws_status[1] = 0;
+        if (user_status) *user_status = 0;
+    }
+}
+
 __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
                                                           int nPairs, int32_t* __restrict__ order,
                                                           int32_t* __restrict__ ws_status,

@@ -277,11 +277,8 @@ int run(const Problem& P) {
                                                       reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
         if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     } else {
-        if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
-        if (P.d_status && cudaMemsetAsync(P.d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
-            cudaGetLastError();
-            return SALAD_ERR_CUDA;
-        }
+        status_clear_kernel<<<1, 32, 0, P.stream>>>(reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
+        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     }
     if (P.mode & MODE_LINEAR) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
@@ -634,11 +631,8 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     P.stream = static_cast<cudaStream_t>(stream);
     // the array keeps the last call's contents: the status word must start at zero
     uint8_t* ws = static_cast<uint8_t*>(scratch);
-    if (cudaMemsetAsync(ws + w.off_status, 0, kAlign, P.stream) != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
-    if (d_status && cudaMemsetAsync(d_status, 0, sizeof(int32_t), P.stream) != cudaSuccess) {
-        cudaGetLastError();
-        return SALAD_ERR_CUDA;
-    }
+    status_clear_kernel<<<1, 32, 0, P.stream>>>(reinterpret_cast<int32_t*>(ws + w.off_status), d_status);
+    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     rc = (d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
     if (rc != SALAD_OK) return rc;
     return (d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
