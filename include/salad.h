@@ -210,6 +210,16 @@ int salad_proj_combine_fwd(const void* o_s, const void* o_l, const void* w, cons
                            int32_t* d_status, void* stream);
 
 /*
+ * salad_selftest_bounded_wait -- diagnostic (no counterpart in the paper).  Every wait inside the
+ * kernels is bounded: when one expires, the kernel records SALAD_ERR_TIMEOUT in the status word,
+ * lets copies in flight land, frees its tensor memory and returns, so the context stays usable.
+ * This entry point runs that mechanism on its own: a one-thread kernel waits 2 ms on a barrier
+ * that nothing arrives on and then writes SALAD_ERR_TIMEOUT (-6) to *d_status; *d_waited_ns
+ * (optional, device) receives the time it waited.  Nothing faults and nothing hangs.
+ */
+int salad_selftest_bounded_wait(int32_t* d_status, unsigned long long* d_waited_ns, void* stream);
+
+/*
  * salad_linear_attn_fwd_noalloc -- salad_linear_attn_fwd for callers that cannot provide
  * scratch memory (the paper has no counterpart; this is a deployment convenience).
  * Some hosts of this library may not call cudaMalloc at the point where attention runs: a

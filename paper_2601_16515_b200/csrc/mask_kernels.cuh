@@ -104,6 +104,24 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
 // start first and the short ones fill the tail.  Counting sort in shared memory; one CTA per
 // mask head.  The order among equal costs is arbitrary (it only affects scheduling).
 // It is the first kernel of a call, so it also clears the status words the later kernels test.
+// Diagnostic: one thread waits, with a 2 ms limit, on an mbarrier that nothing ever arrives on, and
+// reports the expiry the way the compute kernels do (status word = -6).  It exercises the bounded
+// wait and the status path without any fault: the kernel returns normally.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int32_t* __restrict__ status,
+                                                                   unsigned long long* __restrict__ waited_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+        const uint64_t t0 = global_timer_ns();
+        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, 2000000ull);
+        if (waited_ns) *waited_ns = global_timer_ns() - t0;
+        *status = ok ? 0 : -6;
+    }
+}
+
 // First kernel of a call that has no work-order kernel: clears the status words (and the work-item
 // counter next to the library's).  The kernel after it in the stream is launched so that it can be
 // set up and start its input loads meanwhile.

@@ -604,6 +604,15 @@ SALAD_EXPORT int salad_proj_combine_fwd(const void* o_s, const void* o_l, const 
     return check_launch();
 }
 
+SALAD_EXPORT int salad_selftest_bounded_wait(int32_t* d_status, unsigned long long* d_waited_ns, void* stream) {
+    if (!d_status) return SALAD_ERR_INVALID_ARG;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(d_status, d_waited_ns);
+    return check_launch();
+}
+
 SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* o_l,
                                                float* kv_out, float* z_out, int B, int H, int N, int d,
                                                float eps, int32_t* d_status, void* stream) {

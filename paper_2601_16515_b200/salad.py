@@ -27,7 +27,8 @@ SALAD_ERR_TIMEOUT = -6
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
-           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd")
+           "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
+           "salad_selftest_bounded_wait")
 
 
 class SaladError(RuntimeError):
@@ -69,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_permute_tokens.argtypes = [p, p] + [i32] * 7 + [p, i32, p]
     lib.salad_proj_combine_fwd.restype = i32
     lib.salad_proj_combine_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [p, p]
+    lib.salad_selftest_bounded_wait.restype = i32
+    lib.salad_selftest_bounded_wait.argtypes = [p, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -276,6 +279,14 @@ def salad_proj_combine_fwd(o_s, o_l, w, dyn_scale=None, bias=None, out=None, sta
         _check(_lib.salad_proj_combine_fwd(_ptr(o_s), _ptr(o_l), _ptr(w), _ptr(bias), _ptr(dyn_scale), _ptr(out),
                                            B, H, N, d, _ptr(status), _stream(stream)), "salad_proj_combine_fwd")
     return out
+
+
+def salad_selftest_bounded_wait(stream=None):
+    """Runs the bounded-wait self-test kernel; returns (status, waited_ns) device tensors."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(_lib.salad_selftest_bounded_wait(_ptr(status), _ptr(waited), _stream(stream)), "salad_selftest_bounded_wait")
+    return status, waited
 
 
 DYN_SCALE_WS_BYTES = 8192

@@ -642,3 +642,19 @@ def test_long_sequence_linear_and_sparse_band(salad):
                           np.array([0.5]), np.array([0.5]), sel=sel)
     got = f32(out.cpu()).reshape(-1, d)[sel]
     assert_close(got, ref, "long sequence")
+
+
+# ------------------------------------------------------------------------------ bounded waits
+
+def test_an_expired_wait_is_reported_and_the_context_stays_usable(salad):
+    # Nothing faults here: a one-thread kernel waits 2 ms on a barrier nobody arrives on, gives up and
+    # writes the time-out code, the way every wait inside the compute kernels does.
+    status, waited = salad.salad_selftest_bounded_wait()
+    torch.cuda.synchronize()
+    assert int(status.item()) == salad.SALAD_ERR_TIMEOUT
+    assert 2_000_000 <= int(waited.item()) < 50_000_000
+    # the context is fine: a compute call right after it runs and matches the oracle
+    wl = wlmod.C1
+    q, k, v = wlmod.make_qkv(wl)
+    out = salad.salad_linear_attn_fwd(q.cuda(), k.cuda(), v.cuda())
+    assert_close(f32(out.cpu()).reshape(-1, wl.d), orc.linear_attn(f32(q), f32(k), f32(v)), "after time-out")
