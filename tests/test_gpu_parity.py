@@ -658,3 +658,38 @@ def test_an_expired_wait_is_reported_and_the_context_stays_usable(salad):
     q, k, v = wlmod.make_qkv(wl)
     out = salad.salad_linear_attn_fwd(q.cuda(), k.cuda(), v.cuda())
     assert_close(f32(out.cpu()).reshape(-1, wl.d), orc.linear_attn(f32(q), f32(k), f32(v)), "after time-out")
+
+
+# ------------------------------------------------------------------------------ seeded random sweeps
+
+def test_mask_random_grids_bit_exact(salad):
+    rng = np.random.default_rng(2024)
+    for _ in range(25):
+        T, Hs, Ws = int(rng.integers(1, 7)), int(rng.integers(1, 10)), int(rng.integers(1, 12))
+        Bq = int(rng.choice([4, 8, 16, 32, 64, 128])); Bk = int(rng.choice([4, 8, 16, 32, 64]))
+        Hm = int(rng.integers(1, 4))
+        windows = [(int(rng.integers(0, T + 1)), int(rng.integers(0, Hs + 1)), int(rng.integers(0, Ws + 1)))
+                   for _ in range(Hm)]
+        rp, ci = salad.salad_mask_build(T, Hs, Ws, Bq, Bk, windows)
+        rp_ref, ci_ref = orc.mask_build(T, Hs, Ws, Bq, Bk, windows)
+        assert np.array_equal(rp.cpu().numpy(), rp_ref), (T, Hs, Ws, Bq, Bk, windows)
+        assert np.array_equal(ci.cpu().numpy()[:len(ci_ref)], ci_ref), (T, Hs, Ws, Bq, Bk, windows)
+
+
+def test_fused_random_shapes(salad):
+    rng = np.random.default_rng(4048)
+    for case in range(10):
+        B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
+        N = int(rng.integers(1, 1400)); d = int(rng.choice([64, 128])); Bq = int(rng.choice([64, 128]))
+        Hm = int(rng.choice([1, H, B * H]))
+        q, k, v = rand_qkv(B, H, N, d, 9000 + case)
+        nQb, nKb = -(-N // Bq), -(-N // 64)
+        rp, ci = random_csr(Hm * nQb, nKb, 77 + case, lo=0, hi=nKb)
+        rp_d, ci_d = dev_csr(rp, ci)
+        lam = rng.uniform(0, 1, H).astype(np.float32); s = rng.uniform(0, 1, B).astype(np.float32)
+        status = torch.ones(1, dtype=torch.int32, device="cuda")
+        out = salad.salad_fused_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, Hm, torch.from_numpy(lam).cuda(),
+                                    torch.from_numpy(s).cuda(), Bq=Bq, status=status)
+        status_ok(status)
+        ref = orc.salad_fused(f32(q), f32(k), f32(v), Bq, 64, rp, ci, Hm, lam.astype(np.float64), s.astype(np.float64))
+        assert_close(f32(out.cpu()).reshape(-1, d), ref, f"random case {case}: B{B} H{H} N{N} d{d} Bq{Bq} Hm{Hm}")
