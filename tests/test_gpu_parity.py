@@ -693,3 +693,24 @@ def test_fused_random_shapes(salad):
         status_ok(status)
         ref = orc.salad_fused(f32(q), f32(k), f32(v), Bq, 64, rp, ci, Hm, lam.astype(np.float64), s.astype(np.float64))
         assert_close(f32(out.cpu()).reshape(-1, d), ref, f"random case {case}: B{B} H{H} N{N} d{d} Bq{Bq} Hm{Hm}")
+
+
+def test_two_streams_with_their_own_workspaces(salad):
+    # calls that may overlap on the GPU need separate workspaces and status words; results must not change
+    B, H, N, d = 1, 4, 2048, 128
+    q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 808))
+    rp, ci = salad.salad_mask_build(4, 16, 32, 128, 64, [(1, 3, 8)])
+    lam = torch.rand(H, device="cuda"); s = torch.rand(B, device="cuda")
+    serial_f = salad.salad_fused_fwd(q, k, v, rp, ci, 1, lam, s)
+    serial_l = salad.salad_linear_attn_fwd(q, k, v)
+    torch.cuda.synchronize()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    ws_a = salad.alloc_workspace(B, H, N, d); ws_b = salad.alloc_workspace(B, H, N, d)
+    st_a = torch.ones(1, dtype=torch.int32, device="cuda"); st_b = torch.ones(1, dtype=torch.int32, device="cuda")
+    out_a = torch.empty_like(q); out_b = torch.empty_like(q)
+    for _ in range(10):
+        salad.salad_fused_fwd(q, k, v, rp, ci, 1, lam, s, out=out_a, workspace=ws_a, status=st_a, stream=sa)
+        salad.salad_linear_attn_fwd(q, k, v, out=out_b, workspace=ws_b, status=st_b, stream=sb)
+    torch.cuda.synchronize()
+    assert int(st_a.item()) == 0 and int(st_b.item()) == 0
+    assert torch.equal(out_a, serial_f) and torch.equal(out_b, serial_l)
