@@ -714,3 +714,27 @@ def test_two_streams_with_their_own_workspaces(salad):
     torch.cuda.synchronize()
     assert int(st_a.item()) == 0 and int(st_b.item()) == 0
     assert torch.equal(out_a, serial_f) and torch.equal(out_b, serial_l)
+
+
+def test_fused_call_in_a_cuda_graph(salad):
+    # the call allocates nothing and synchronises nothing: it can be captured and replayed
+    B, H, N, d = 1, 4, 2048, 128
+    q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 909))
+    rp, ci = salad.salad_mask_build(4, 16, 32, 128, 64, [(1, 3, 8)])
+    lam = torch.rand(H, device="cuda"); s = torch.rand(B, device="cuda")
+    ws = salad.alloc_workspace(B, H, N, d)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    eager = salad.salad_fused_fwd(q, k, v, rp, ci, 1, lam, s, workspace=ws, status=status)      # also the first-call set-up
+    torch.cuda.synchronize()
+    out = torch.zeros_like(q)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            salad.salad_fused_fwd(q, k, v, rp, ci, 1, lam, s, out=out, workspace=ws, status=status, stream=side)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(out, eager)
