@@ -1,41 +1,37 @@
 // Block-sparse softmax attention (Eq. 2) fused with the apply step of ReLU linear attention
 // (Eq. 3) and the scaled residual sum of Algorithm 1, for sm_100a.
 //
-// One CTA owns two consecutive query blocks of one (batch, head): two 128-row MMA tiles.
-//   warp 0        TMA producer of the Q tiles, the linear-state tile and the K ring
+// One CTA owns one query block of one (batch, head): a 128-row MMA tile.  Two CTAs share an SM
+// (each takes half of its shared memory, registers and tensor memory), so the set-up, the first
+// loads and the epilogue of one overlap the main loop of the other, and the two tiles of an SM run
+// independently of each other.
+//   warp 0        TMA producer of the Q tile, the K ring and (at the end) the linear-state tile
 //   warp 1        TMA producer of the V ring (independent of the K ring, so neither ring can
 //                 stall the other)
-//   warps 2, 3    tcgen05 issuers of S = Q K^T for tile 0 and tile 1 (one thread each); warp 2
-//                 owns the TMEM allocation
-//   warps 4, 5    tcgen05 issuers of O += P V (and of the linear numerator) for tile 0 and 1
-//   warps 8-15    softmax + epilogue warps of tile 0: a warp works on 16 query rows (TMEM lanes)
-//                 with the 16-lane load/store shapes, four threads share a row and each thread
-//                 serves two rows; row maxima and sums are combined with two shuffles
-//   warps 16-23   the same for tile 1
-// The kept lists of the two query blocks are walked as one sorted merge, so a key block that
-// both keep is fetched once and multiplied against both tiles.  Masked blocks are never
-// loaded.
+//   warp 2        tcgen05 issuer of S = Q K^T (one thread); owns the TMEM allocation
+//   warp 3        tcgen05 issuer of O += P V and of the linear numerator (one thread)
+//   warps 4-11    softmax + epilogue warps: a warp works on 16 query rows (TMEM lanes) with the
+//                 16-lane load/store shapes, four threads share a row and each thread serves two
+//                 rows; row maxima and sums are combined with two shuffles
+// Masked blocks are never loaded.
 //
-// Per tile, S = Q K^T (128x64xd, operands in shared memory) of block t lands in TMEM score
-// buffer t & 1; the softmax warps copy it to registers and write P = exp2(.), as bf16, over the
-// first half of the same buffer, which O += P V then reads.  The scores of block t + 1 go to the
-// other buffer as soon as the P V product of block t - 1 has read it, so both products of the
-// neighbouring blocks overlap the softmax of block t.  The running max lives in the log2 domain;
-// exponentials start against the max of the earlier blocks and the O accumulator is rescaled only
-// when the max grows by more than 2^8.
-// The two products of a tile have their own issuing threads: each walks the merged list,
-// waits only for what its next MMA series needs (so it reacts as soon as that arrives), and
-// releases the ring stages of the other tile's blocks, always after waiting for the stage to
-// be full so that a release can never run a phase ahead.
-// After the last block the warpgroup applies ReLU to its Q rows in shared memory, computes
-// the linear denominator with plain FMAs, the issuing thread multiplies ReLU(Q) with the bf16
-// linear state, and the epilogue writes
+// S = Q K^T (128x64xd, operands in shared memory) of block t lands in TMEM score buffer t & 1;
+// the softmax warps copy it to registers and write P = exp2(.), as bf16, over the first half of
+// the same buffer, which O += P V then reads.  The scores of block t + 1 go to the other buffer
+// as soon as the P V product of block t - 1 has read it, so both products of the neighbouring
+// blocks overlap the softmax of block t.  The running max lives in the log2 domain; exponentials
+// start against the max of the earlier blocks and the O accumulator is rescaled only when the max
+// grows by more than 2^8.  The two products have their own issuing threads: each waits only for
+// what its next MMA series needs, so it reacts as soon as that arrives.
+// After the last block the softmax warps apply ReLU to the Q rows in shared memory and compute the
+// linear denominator with plain FMAs; the linear state (bf16, transposed) is loaded over the K
+// ring, which is idle by then; the issuing thread multiplies ReLU(Q) with it, and the epilogue
+// writes
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
 //
-// TMEM columns (512 allocated), tile i at 256 i:  [0,64) and [64,128) two score buffers (block t
-// uses buffer t & 1; its probabilities, packed bf16, overwrite the first 32 columns of the same
-// buffer, so the scores of block t + 1 can be computed while block t is still in the softmax);
+// TMEM columns (256 allocated):  [0,64) and [64,128) two score buffers (block t uses buffer
+// t & 1; its probabilities, packed bf16, overwrite the first 32 columns of the same buffer);
 // [128,128+D) O.  The linear numerator reuses [0,D).
 #pragma once
 #include "ptx.cuh"
@@ -53,10 +49,10 @@ namespace salad {
 enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
 
 struct FusedParams {
-    int N, H, nQb, nKb, nPairs, Bq, Hm, mode;
+    int N, H, nQb, nKb, Bq, Hm, mode;
     const int32_t* row_ptr;
     const int32_t* col_idx;
-    const int32_t* order;        // [Hm][nPairs] launch order of the query-block pairs, or null (identity)
+    const int32_t* order;        // [Hm][nQb] launch order of the query blocks, or null (identity)
     int BH;                      // batch * heads
     const float* static_scale;   // [H] or null (=1)
     const float* dyn_scale;      // [B] or null (=1)
@@ -73,54 +69,34 @@ template <int D>
 struct FusedCfg {
     static constexpr int BK = 64;
     static constexpr int CH = D / 64;               // 128-byte chunks per row
-    static constexpr int Q_CHUNK = 128 * 128;       // bytes of one 64-column chunk of a Q tile
+    static constexpr int Q_CHUNK = 128 * 128;       // bytes of one 64-column chunk of the Q tile
     static constexpr int Q_BYTES = CH * Q_CHUNK;
     static constexpr int KV_CHUNK = BK * 128;
     static constexpr int KV_BYTES = CH * KV_CHUNK;  // one K or V tile
     static constexpr int ST_CHUNK = D * 128;
-    static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]
-    static constexpr int NK = 4, NV = 4;
+    static constexpr int ST_BYTES = CH * ST_CHUNK;  // linear state, bf16 [D][D]: as large as the K ring
+    static constexpr int NK = 2, NV = 2;
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_ST = 2 * Q_BYTES;
-    static constexpr int OFF_K = OFF_ST + ST_BYTES;
+    static constexpr int OFF_K = Q_BYTES;
+    static constexpr int OFF_ST = OFF_K;            // loaded over the K ring once every Q K^T has completed
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
-    static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack
-    static constexpr int THREADS = 768;
-    // TMEM columns within a tile's 256: two score buffers of 64 (P overwrites the first 32 columns
-    // of the buffer its scores came from), then the output accumulator
+    static constexpr int SMEM_BYTES = OFF_V + NV * KV_BYTES + 1024;   // + alignment slack: 97 KB at D = 128
+    static constexpr int THREADS = 384;
+    // TMEM columns: two score buffers of 64 (P overwrites the first 32 columns of the buffer its
+    // scores came from), then the output accumulator
     static constexpr uint32_t COL_SP = 0, SP_STRIDE = 64, COL_O = 128;
+    static constexpr uint32_t TMEM_COLS = 256;
 };
+static_assert(FusedCfg<128>::ST_BYTES == FusedCfg<128>::NK * FusedCfg<128>::KV_BYTES, "the state tile fills the K ring");
+static_assert(FusedCfg<64>::ST_BYTES <= FusedCfg<64>::NK * FusedCfg<64>::KV_BYTES, "the state tile fits in the K ring");
 
 struct FusedBarriers {
-    uint64_t q_full[2], st_full, k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2][2], p_ready[2][2], pv_done[2][2], o_final[2], lin_ready[2], lin_done[2], out_staged[2];
-};
-
-// Sorted merge of the two kept lists.  tag bit i set: tile i keeps this key block.
-// The heads of both lists are loaded one call ahead, so that the global-load latency of an
-// entry is spent while the caller works on the previous one (the kernel leaves almost no L1).
-struct MergeWalk {
-    const int32_t* col;
-    int e0, end0, e1, end1;
-    int c0, c1;
-    __device__ __forceinline__ MergeWalk(const int32_t* c, int s0, int n0, int s1, int n1)
-        : col(c), e0(s0), end0(n0), e1(s1), end1(n1) {
-        c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff;
-        c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff;
-    }
-    __device__ __forceinline__ bool next(int& c, int& tag) {
-        c = min(c0, c1);
-        if (c == 0x7fffffff) return false;
-        const bool a0 = (c0 == c), a1 = (c1 == c);
-        tag = (a0 ? 1 : 0) | (a1 ? 2 : 0);
-        if (a0) { ++e0; c0 = (e0 < end0) ? __ldg(col + e0) : 0x7fffffff; }
-        if (a1) { ++e1; c1 = (e1 < end1) ? __ldg(col + e1) : 0x7fffffff; }
-        return true;
-    }
+    uint64_t q_full, st_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
+    uint64_t s_full[2], p_ready[2], pv_done[2], o_final, lin_ready, lin_done, out_staged;
 };
 
 template <int D>
-__global__ void __launch_bounds__(768, 1)
+__global__ void __launch_bounds__(384, 2)
 salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                    const __grid_constant__ CUtensorMap map_st, const FusedParams p)
@@ -140,227 +116,203 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     // work item: head by head (K/V of one head stay hot in L2: ordering the cheapest items of all
     // heads last instead was measured to shorten the launch by 0.3 % and to raise its DRAM traffic by
-    // half), within a head the pairs of query blocks from the most to the least expensive, so that
-    // the kernel ends on short items
-    const int rank = blockIdx.x % p.nPairs, bh = blockIdx.x / p.nPairs;
+    // half), within a head the query blocks from the most to the least expensive, so that the
+    // kernel ends on short items
+    const int rank = blockIdx.x % p.nQb, bh = blockIdx.x / p.nQb;
     const int h = bh % p.H, b = bh / p.H;
     const int hm = (p.Hm == 1) ? 0 : (p.Hm == p.H ? h : bh);   // one mask, one per head, or one per (batch, head)
-    const int pair = p.order ? __ldg(p.order + size_t(hm) * p.nPairs + rank) : rank;
+    const int qb = p.order ? __ldg(p.order + size_t(hm) * p.nQb + rank) : rank;
     const bool sparse = (p.mode & MODE_SPARSE) != 0;
     // post-tuning branch dropping (Sec. 4.3): no linear work at all for a dropped batch item
     const bool linear = (p.mode & MODE_LINEAR) != 0 &&
                         !(p.dyn_scale != nullptr && __ldg(p.dyn_scale + b) < p.drop_tau);
-
-    // kept lists of the two tiles
-    int qb[2], ls[2], le[2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        qb[i] = 2 * pair + i;
-        ls[i] = le[i] = 0;
-        if (sparse && qb[i] < p.nQb) {
-            ls[i] = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb[i]);
-            le[i] = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb[i] + 1);
-        }
+    // kept list of the query block
+    int ls = 0, le = 0;
+    if (sparse) {
+        ls = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb);
+        le = __ldg(p.row_ptr + size_t(hm) * p.nQb + qb + 1);
     }
 
     // ------------------------------------------------------------------ set-up
     if (tid == 0) {
         TRACE_CTA(0);
         abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&bars.q_full[i]), 1);
-            mbar_init(smem_u32(&bars.o_final[i]), 1);
-            mbar_init(smem_u32(&bars.lin_ready[i]), 256);
-            mbar_init(smem_u32(&bars.lin_done[i]), 1);
-            mbar_init(smem_u32(&bars.out_staged[i]), 256);
-            for (int j = 0; j < 2; ++j) {
-                mbar_init(smem_u32(&bars.s_full[i][j]), 1);
-                mbar_init(smem_u32(&bars.p_ready[i][j]), 8);          // one arrival per softmax warp
-                mbar_init(smem_u32(&bars.pv_done[i][j]), 1);
-            }
-        }
+        mbar_init(smem_u32(&bars.q_full), 1);
         mbar_init(smem_u32(&bars.st_full), 1);
-        for (int s = 0; s < 4; ++s) {
-            mbar_init(smem_u32(&bars.k_full[s]), 1);
-            mbar_init(smem_u32(&bars.k_empty[s]), 2);     // released by both issuing threads
-            mbar_init(smem_u32(&bars.v_full[s]), 1);
-            mbar_init(smem_u32(&bars.v_empty[s]), 2);
+        mbar_init(smem_u32(&bars.o_final), 1);
+        mbar_init(smem_u32(&bars.lin_ready), 256);
+        mbar_init(smem_u32(&bars.lin_done), 1);
+        mbar_init(smem_u32(&bars.out_staged), 256);
+        for (int j = 0; j < 2; ++j) {
+            mbar_init(smem_u32(&bars.s_full[j]), 1);
+            mbar_init(smem_u32(&bars.p_ready[j]), 8);          // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.pv_done[j]), 1);
+            mbar_init(smem_u32(&bars.k_full[j]), 1);
+            mbar_init(smem_u32(&bars.k_empty[j]), 1);
+            mbar_init(smem_u32(&bars.v_full[j]), 1);
+            mbar_init(smem_u32(&bars.v_empty[j]), 1);
         }
         fence_mbar_init();
     }
     if (p.Bq < 128) {
-        // rows [Bq, 128) of the Q tiles are never written by TMA: zero them so the unused
+        // rows [Bq, 128) of the Q tile are never written by TMA: zero them so the unused
         // half of the MMA tile holds finite numbers
-        for (int i = tid; i < 2 * C::CH * (128 - p.Bq) * 8; i += C::THREADS) {
+        for (int i = tid; i < C::CH * (128 - p.Bq) * 8; i += C::THREADS) {
             const int chunk = i / ((128 - p.Bq) * 8), rest = i % ((128 - p.Bq) * 8);
             *reinterpret_cast<uint4*>(smem + C::OFF_Q + chunk * C::Q_CHUNK + p.Bq * 128 + rest * 16) =
                 make_uint4(0, 0, 0, 0);
         }
         fence_proxy_async_smem();
     }
-    if (warp == 2) { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
-    if (linear && tid >= 256 && tid < 256 + D) z_s[tid - 256] = __ldg(p.z + size_t(bh) * D + (tid - 256));
+    if (warp == 2) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
+    if (linear && tid >= 128 && tid < 128 + D) z_s[tid - 128] = __ldg(p.z + size_t(bh) * D + (tid - 128));
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_slot;
     volatile int* abortp = &abort_flag;
     if (tid == 0) TRACE_CTA(1);
+    const int len = le - ls;
 
     if (abort_flag == 0) {
-    if (warp == 0 || warp == 1) {
-        // ============================================================== TMA producers
+    if (warp == 0) {
+        // ============================================================== TMA producer: Q, the K ring, the state tile
         if (lane == 0) {
-            const bool is_k = (warp == 0);
-            if (is_k) {
-                prefetch_tmap(&map_q); prefetch_tmap(&map_k);
-                for (int i = 0; i < 2; ++i) {
-                    if (qb[i] >= p.nQb) continue;
-                    // A tile with no kept block and no linear branch never reads Q: its epilogue
-                    // stages zeros in the Q tile without waiting for q_full, so nothing may land there.
-                    if (le[i] == ls[i] && !linear) continue;
-                    const uint32_t bar = smem_u32(&bars.q_full[i]);
-                    mbar_arrive_expect_tx(bar, uint32_t(p.Bq) * D * 2);
-                    for (int ch = 0; ch < C::CH; ++ch)
-                        tma_load_3d(s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, &map_q, bar,
-                                    ch * 64, qb[i] * p.Bq, bh);
-                }
-                if (linear) {
+            prefetch_tmap(&map_q); prefetch_tmap(&map_k);
+            // A block with no kept key block and no linear branch never reads Q: its epilogue
+            // stages zeros in the Q tile without waiting for q_full, so nothing may land there.
+            if (len > 0 || linear) {
+                const uint32_t bar = smem_u32(&bars.q_full);
+                mbar_arrive_expect_tx(bar, uint32_t(p.Bq) * D * 2);
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_load_3d(s_base + C::OFF_Q + ch * C::Q_CHUNK, &map_q, bar, ch * 64, qb * p.Bq, bh);
+            }
+            bool ok = true;
+            for (int t = 0; t < len; ++t) {
+                const int s = t % C::NK;
+                ok = mbar_wait(smem_u32(&bars.k_empty[s]), ((t / C::NK) & 1) ^ 1, abortp);
+                if (!ok) break;
+                const int col = __ldg(p.col_idx + ls + t);
+                const uint32_t bar = smem_u32(&bars.k_full[s]);
+                mbar_arrive_expect_tx(bar, C::KV_BYTES);
+                for (int ch = 0; ch < C::CH; ++ch)
+                    tma_load_3d(s_base + C::OFF_K + s * C::KV_BYTES + ch * C::KV_CHUNK, &map_k, bar, ch * 64,
+                                col * C::BK, bh);
+            }
+            if (ok && linear) {
+                // the state tile goes over the K ring: every Q K^T must have read its K block.  The products
+                // complete in order, so the last one (signalled on its score buffer's barrier) covers all.
+                if (len > 0) ok = mbar_wait(smem_u32(&bars.s_full[(len - 1) & 1]), ((len - 1) >> 1) & 1, abortp);
+                if (ok) {
+                    prefetch_tmap(&map_st);
                     const uint32_t bar = smem_u32(&bars.st_full);
                     mbar_arrive_expect_tx(bar, C::ST_BYTES);
                     for (int ch = 0; ch < C::CH; ++ch)
                         tma_load_3d(s_base + C::OFF_ST + ch * C::ST_CHUNK, &map_st, bar, ch * 64, 0, bh);
                 }
-            } else {
-                prefetch_tmap(&map_v);
             }
-            const CUtensorMap* m = is_k ? &map_k : &map_v;
-            uint64_t* full = is_k ? bars.k_full : bars.v_full;
-            uint64_t* empty = is_k ? bars.k_empty : bars.v_empty;
-            const uint32_t ring = s_base + (is_k ? C::OFF_K : C::OFF_V);
-            constexpr int NS = 4;                          // NK == NV
-            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
-            int col, tag, g = 0;
-            while (wk.next(col, tag)) {
-                const int s = g % NS;
-                if (!mbar_wait(smem_u32(&empty[s]), ((g / NS) & 1) ^ 1, abortp)) break;
-                const uint32_t bar = smem_u32(&full[s]);
+        }
+    } else if (warp == 1) {
+        // ============================================================== TMA producer of the V ring
+        if (lane == 0) {
+            prefetch_tmap(&map_v);
+            for (int t = 0; t < len; ++t) {
+                const int s = t % C::NV;
+                if (!mbar_wait(smem_u32(&bars.v_empty[s]), ((t / C::NV) & 1) ^ 1, abortp)) break;
+                const int col = __ldg(p.col_idx + ls + t);
+                const uint32_t bar = smem_u32(&bars.v_full[s]);
                 mbar_arrive_expect_tx(bar, C::KV_BYTES);
                 for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(ring + s * C::KV_BYTES + ch * C::KV_CHUNK, m, bar, ch * 64, col * C::BK, bh);
-                ++g;
+                    tma_load_3d(s_base + C::OFF_V + s * C::KV_BYTES + ch * C::KV_CHUNK, &map_v, bar, ch * 64,
+                                col * C::BK, bh);
             }
         }
-    } else if (warp == 2 || warp == 3) {
-        // ============================================================== issuer of S = Q K^T, tile i
+    } else if (warp == 2) {
+        // ============================================================== issuer of S = Q K^T
         if (lane == 0) {
-            const int i = warp - 2;
             const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
             constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
-            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
+            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
             const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
-            const uint32_t t_tile = tmem + i * 256;
-            const int len = le[i] - ls[i];
             bool ok = true;
             if (len > 0) {
-                ok = mbar_wait(smem_u32(&bars.q_full[i]), 0, abortp);
+                ok = mbar_wait(smem_u32(&bars.q_full), 0, abortp);
                 tc_fence_after_sync();
             }
-            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
-            int col, tag, g = 0, t = 0;
-            while (ok && wk.next(col, tag)) {
-                const int s = g % C::NK;
-                ok = mbar_wait(smem_u32(&bars.k_full[s]), (g / C::NK) & 1, abortp);
+            for (int t = 0; t < len && ok; ++t) {
+                const int s = t % C::NK;
+                ok = mbar_wait(smem_u32(&bars.k_full[s]), (t / C::NK) & 1, abortp);
+                // score buffer t & 1 held P of block t - 2: its P V product must have read it
+                if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.pv_done[t & 1]), ((t >> 1) - 1) & 1, abortp);
                 if (!ok) break;
-                if ((tag >> i) & 1) {
-                    // score buffer t & 1 held P of block t - 2: its P V product must have read it
-                    if (t >= 2) ok = mbar_wait(smem_u32(&bars.pv_done[i][t & 1]), ((t >> 1) - 1) & 1, abortp);
-                    if (!ok) break;
-                    TRACE(2 + i, t, 0);
-                    tc_fence_after_sync();
-                    const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
+                TRACE(2, t, 0);
+                tc_fence_after_sync();
+                const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
-                        mma_ss_lohi(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
-                                    kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                    tc_commit(smem_u32(&bars.s_full[i][t & 1]));
-                    tc_commit(smem_u32(&bars.k_empty[s]));
-                    TRACE(2 + i, t, 3);
-                    ++t;
-                } else {
-                    mbar_arrive(smem_u32(&bars.k_empty[s]));      // a block of the other tile only
-                }
-                ++g;
+                for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
+                    mma_ss_lohi(tmem + C::COL_SP + (t & 1) * C::SP_STRIDE,
+                                q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
+                tc_commit(smem_u32(&bars.s_full[t & 1]));
+                tc_commit(smem_u32(&bars.k_empty[s]));
+                TRACE(2, t, 3);
             }
         }
-    } else if (warp == 4 || warp == 5) {
-        // ============================================================== issuer of O += P V, tile i
+    } else if (warp == 3) {
+        // ============================================================== issuer of O += P V and of the linear numerator
         if (lane == 0) {
-            const int i = warp - 4;
             const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
             const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
             constexpr uint32_t HI = sdesc_hi_sw128(1024);
-            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + i * C::Q_BYTES, 16);
+            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
             const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
-            const uint32_t t_tile = tmem + i * 256;
-            const int len = le[i] - ls[i];
             bool ok = true;
-            MergeWalk wk(p.col_idx, ls[0], le[0], ls[1], le[1]);
-            int col, tag, g = 0, t = 0;
-            while (ok && wk.next(col, tag)) {
-                const int s = g % C::NV;
-                ok = mbar_wait(smem_u32(&bars.v_full[s]), (g / C::NV) & 1, abortp);
+            for (int t = 0; t < len && ok; ++t) {
+                const int s = t % C::NV;
+                ok = mbar_wait(smem_u32(&bars.v_full[s]), (t / C::NV) & 1, abortp);
+                if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[t & 1]), (t >> 1) & 1, abortp);
                 if (!ok) break;
-                if ((tag >> i) & 1) {
-                    ok = mbar_wait(smem_u32(&bars.p_ready[i][t & 1]), (t >> 1) & 1, abortp);
-                    if (!ok) break;
-                    TRACE(2 + i, t, 1);
-                    tc_fence_after_sync();
-                    const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
-                    const uint32_t p_col = t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE;
+                TRACE(2, t, 1);
+                tc_fence_after_sync();
+                const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
+                const uint32_t p_col = tmem + C::COL_SP + (t & 1) * C::SP_STRIDE;
 #pragma unroll
-                    for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
-                        mma_ts_lohi(t_tile + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
-                                    (t > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&bars.v_empty[s]));
-                    tc_commit(smem_u32(&bars.pv_done[i][t & 1]));
-                    ++t;
-                    if (t == len) tc_commit(smem_u32(&bars.o_final[i]));
-                    TRACE(2 + i, t - 1, 2);
-                } else {
-                    mbar_arrive(smem_u32(&bars.v_empty[s]));
-                }
-                ++g;
+                for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
+                    mma_ts_lohi(tmem + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
+                                (t > 0 || k > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&bars.v_empty[s]));
+                tc_commit(smem_u32(&bars.pv_done[t & 1]));
+                if (t + 1 == len) tc_commit(smem_u32(&bars.o_final));
+                TRACE(2, t, 2);
             }
-            if (ok && linear && qb[i] < p.nQb) {
+            if (ok && linear) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
-                if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready[i]), 0, abortp);
+                if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready), 0, abortp);
                 if (ok) {
                     tc_fence_after_sync();
                     const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST, 16);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k)
-                        mma_ss_lohi(t_tile, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                        mma_ss_lohi(tmem, q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
                                     st_lo + (((k / 4) * C::ST_CHUNK + (k % 4) * 32) >> 4), HI, idesc_lin, k > 0);
-                    tc_commit(smem_u32(&bars.lin_done[i]));
+                    tc_commit(smem_u32(&bars.lin_done));
                 }
             }
         }
-    } else if (warp >= 8) {
+    } else {
         // ============================================================== softmax + epilogue
-        // Eight warps per tile.  A warp works on 16 TMEM lanes (query rows) with the 16-lane
+        // Eight warps.  A warp works on 16 TMEM lanes (query rows) with the 16-lane
         // load/store shapes: four threads share a row, each holding a quarter of its columns,
         // and every thread serves two rows (a and a + 8).  Row maxima and sums are combined
         // with two shuffles inside the group of four.
-        const int sw = warp - 8;
-        const int i = sw >> 3;                                  // tile
+        const int sw = warp - 4;
         const int q4 = lane & 3;                                // position in the group of four
-        const int lane0 = (warp & 3) * 32 + ((sw >> 2) & 1) * 16;          // first TMEM lane of this warp
+        const int lane0 = (warp & 3) * 32 + (sw >> 2) * 16;          // first TMEM lane of this warp
         const int ra = lane0 + (lane >> 2), rb = ra + 8;        // the thread's two query rows
-        const uint32_t t_tile = tmem + i * 256 + (uint32_t(lane0) << 16);
-        const bool tile_valid = qb[i] < p.nQb;
-        const int len = le[i] - ls[i];
-        uint8_t* qtile = smem + C::OFF_Q + i * C::Q_BYTES;
+        const uint32_t t_tile = tmem + (uint32_t(lane0) << 16);
+        const bool tile_valid = true;
+        const int len = le - ls;
+        uint8_t* qtile = smem + C::OFF_Q;
         float m_a = -INFINITY, m_b = -INFINITY;                 // running maxima (log2 domain)
         float l_a = 0.f, l_b = 0.f;                             // this thread's share of the row sums
         bool ok = true;
@@ -380,18 +332,18 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
         const bool ragged_keys = (p.N % C::BK) != 0;
         for (int t = 0; t < len && ok; ++t) {
-            if (ra == 0 && q4 == 0) TRACE(i, t, 0);
+            if (ra == 0 && q4 == 0) TRACE(0, t, 0);
             // only the last key block can be short; its id is needed only then
-            const int col = ragged_keys ? __ldg(p.col_idx + ls[i] + t) : 0;
-            ok = wait_uniform(&bars.s_full[i][t & 1], (t >> 1) & 1);
+            const int col = ragged_keys ? __ldg(p.col_idx + ls + t) : 0;
+            ok = wait_uniform(&bars.s_full[t & 1], (t >> 1) & 1);
             if (!ok) break;
-            if (ra == 0 && q4 == 0) TRACE(i, t, 1);
+            if (ra == 0 && q4 == 0) TRACE(0, t, 1);
             tc_fence_after_sync();
             // x[4n], x[4n+1] = S(row a, keys 8n + 2 q4, + 1);  x[4n+2], x[4n+3] = the same keys of row b
             uint32_t xr[32];
             tmem_ld_16x256b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, xr);
             tmem_wait_ld();
-            if (ra == 0 && q4 == 0) TRACE(i, t, 2);
+            if (ra == 0 && q4 == 0) TRACE(0, t, 2);
             float* x = reinterpret_cast<float*>(xr);
             const int valid = p.N - col * C::BK;              // keys of this block that exist
             if (ragged_keys && valid < C::BK) {
@@ -419,7 +371,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 m_a = quad_max(mxa) * p.scale_log2; m_b = quad_max(mxb) * p.scale_log2;
             } else if (__any_sync(0xffffffffu, mxa * p.scale_log2 > m_a + 8.0f || mxb * p.scale_log2 > m_b + 8.0f)) {
                 const float msa = quad_max(mxa) * p.scale_log2, msb = quad_max(mxb) * p.scale_log2;
-                ok = wait_uniform(&bars.pv_done[i][(t - 1) & 1], ((t - 1) >> 1) & 1);
+                ok = wait_uniform(&bars.pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const float na = fmaxf(m_a, msa), nb = fmaxf(m_b, msb);
@@ -442,7 +394,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 tmem_wait_st();
             }
-            if (ra == 0 && q4 == 0) TRACE(i, t, 3);
+            if (ra == 0 && q4 == 0) TRACE(0, t, 3);
             // P = exp2(x * scale - m), packed bf16: word 2n = row a, keys (8n + 2 q4, + 1) = packed
             // column 4n + q4 of the P tile, word 2n + 1 the same of row b -- the 16x128b layout
             uint32_t pk[16];
@@ -465,14 +417,14 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 unpack_f32x2(acc_a, s0, s1); l_a += s0 + s1;
                 unpack_f32x2(acc_b, s0, s1); l_b += s0 + s1;
             }
-            if (ra == 0 && q4 == 0) TRACE(i, t, 4);
+            if (ra == 0 && q4 == 0) TRACE(0, t, 4);
             // P goes over the scores it was computed from (this warp's own lanes, already in registers)
             tmem_st_16x128b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[i][t & 1]));   // one arrival per warp
-            if (ra == 0 && q4 == 0) TRACE(i, t, 5);
+            if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[t & 1]));   // one arrival per warp
+            if (ra == 0 && q4 == 0) TRACE(0, t, 5);
         }
         float coef_a = 0.f, coef_b = 0.f;
         if (ok && tile_valid && linear) {
@@ -480,7 +432,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // row take two 16-byte groups of every 64 channels each.  Every Q K^T of this tile has
             // completed (its scores were consumed above), so Q is no longer read; the last P V
             // product may still be running meanwhile.
-            ok = wait_uniform(&bars.q_full[i], 0);
+            ok = wait_uniform(&bars.q_full, 0);
             if (ok) {
                 float den_a = 0.f, den_b = 0.f;
 #pragma unroll
@@ -516,15 +468,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 coef_a = c_scale / (den_a + p.eps);
                 coef_b = c_scale / (den_b + p.eps);
                 fence_proxy_async_smem();
-                mbar_arrive(smem_u32(&bars.lin_ready[i]));
+                mbar_arrive(smem_u32(&bars.lin_ready));
             }
         }
         if (ok && len > 0) {
-            ok = wait_uniform(&bars.o_final[i], 0);
+            ok = wait_uniform(&bars.o_final, 0);
             tc_fence_after_sync();
         }
         if (ok && tile_valid && linear) {
-            ok = wait_uniform(&bars.lin_done[i], 0);
+            ok = wait_uniform(&bars.lin_done, 0);
             tc_fence_after_sync();
         }
 
@@ -558,11 +510,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
             fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&bars.out_staged[i]));
-            if (ra == 0 && q4 == 0 && mbar_wait(smem_u32(&bars.out_staged[i]), 0, abortp)) {
+            mbar_arrive(smem_u32(&bars.out_staged));
+            if (ra == 0 && q4 == 0 && mbar_wait(smem_u32(&bars.out_staged), 0, abortp)) {
                 for (int ch = 0; ch < C::CH; ++ch)
-                    tma_store_3d(&map_o, s_base + C::OFF_Q + i * C::Q_BYTES + ch * C::Q_CHUNK, ch * 64,
-                                 qb[i] * p.Bq, bh);
+                    tma_store_3d(&map_o, s_base + C::OFF_Q + ch * C::Q_CHUNK, ch * 64,
+                                 qb * p.Bq, bh);
                 tma_store_commit();
                 // only the shared-memory source must have been read before the CTA may exit; the
                 // writes are complete, like all of the kernel's, when the grid is
@@ -573,7 +525,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int e2 = 0; e2 < 2; ++e2) {
                     const int row = e2 ? rb : ra;
-                    const int n = qb[i] * p.Bq + row;
+                    const int n = qb * p.Bq + row;
                     if (row < p.Bq && n < p.N)
                         p.lse[size_t(bh) * p.N + n] =
                             (len > 0) ? ((e2 ? m_b : m_a) + log2f(e2 ? lt_b : lt_a)) * 0.6931471805599453f : -INFINITY;
@@ -597,7 +549,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
         __syncthreads();
     }
-    if (warp == 2) tmem_dealloc(tmem, 512);
+    if (warp == 2) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 }  // namespace salad

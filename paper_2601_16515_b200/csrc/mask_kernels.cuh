@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(32) status_clear_kernel(int32_t* __restrict__ 
 }
 
 __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
-                                                          int nPairs, int32_t* __restrict__ order,
+                                                          int32_t* __restrict__ order,
                                                           int32_t* __restrict__ ws_status,
                                                           int32_t* __restrict__ user_status) {
     grid_launch_dependents();         // the next kernel of the call may be placed now; it waits for this one
@@ -148,11 +148,8 @@ __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restr
     __shared__ int hist[BINS];
     const int hm = blockIdx.x, tid = threadIdx.x;
     const int32_t* rp = row_ptr + size_t(hm) * nQb;
-    auto cost_of = [&](int pr) {
-        const int a = rp[2 * pr + 1] - rp[2 * pr];
-        const int b = (2 * pr + 1 < nQb) ? rp[2 * pr + 2] - rp[2 * pr + 1] : 0;
-        return min(BINS - 1, max(a, b));
-    };
+    const int nPairs = nQb;           // one work item per query block
+    auto cost_of = [&](int pr) { return min(BINS - 1, rp[pr + 1] - rp[pr]); };
     for (int i = tid; i < BINS; i += blockDim.x) hist[i] = 0;
     __syncthreads();
     for (int pr = tid; pr < nPairs; pr += blockDim.x) atomicAdd(&hist[cost_of(pr)], 1);

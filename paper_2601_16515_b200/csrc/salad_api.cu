@@ -44,7 +44,7 @@ struct Workspace {
 Workspace carve(int B, int H, int N, int d, int Bq) {
     Workspace w;
     const size_t BH = size_t(B) * H;
-    const size_t nPairs = (size_t(N + Bq - 1) / Bq + 1) / 2;
+    const size_t nItems = size_t(N + Bq - 1) / Bq;                 // work items of the attention kernel: query blocks
     w.slots = int(BH > size_t(kPartialSlots) ? BH : size_t(kPartialSlots));
     w.off_status = 0;
     w.off_kvt = kAlign;
@@ -52,7 +52,7 @@ Workspace carve(int B, int H, int N, int d, int Bq) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = w.off_zp + align_up(size_t(w.slots) * d * 4);
-    w.total = w.off_order + align_up(BH * nPairs * 4);              // launch order, per mask (at most B*H)
+    w.total = w.off_order + align_up(BH * nItems * 4);              // launch order, per mask (at most B*H)
     return w;
 }
 
@@ -89,6 +89,12 @@ int prepare_device(DeviceInfo* info) {
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      FusedCfg<64>::SMEM_BYTES);
+        if (e == cudaSuccess)      // two CTAs of the attention kernel share an SM: ask for the largest shared-memory carve-out
+            e = cudaFuncSetAttribute(salad_fused_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_fused_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_linear_state_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      StateCfg<128>::SMEM_BYTES);
@@ -211,7 +217,6 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.N = P.N; fp.H = P.H; fp.Bq = P.Bq; fp.Hm = P.Hm; fp.mode = P.mode;
     fp.nQb = (P.N + P.Bq - 1) / P.Bq;
     fp.nKb = (P.N + 63) / 64;
-    fp.nPairs = (fp.nQb + 1) / 2;
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
     fp.BH = BH;
     fp.order = nullptr;
@@ -225,7 +230,7 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.drop_tau = P.drop_tau;
     fp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     fp.user_status = P.d_status;
-    const int64_t grid = int64_t(fp.nPairs) * BH;
+    const int64_t grid = int64_t(fp.nQb) * BH;
     if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
     record_profile(2, P.stream);
     launch_dependent(salad_fused_kernel<D>, dim3(unsigned(grid)), dim3(FusedCfg<D>::THREADS),
@@ -272,7 +277,7 @@ int run(const Problem& P) {
         // first kernel of the call: longest work items first (the mask is an input of every call,
         // so is its order); it also clears the status words
         const int nQb = (P.N + P.Bq - 1) / P.Bq;
-        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb, (nQb + 1) / 2,
+        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb,
                                                       reinterpret_cast<int32_t*>(ws + w.off_order),
                                                       reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
         if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
