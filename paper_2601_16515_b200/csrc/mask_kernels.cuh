@@ -99,11 +99,6 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
     }
 }
 
-// Launch order of the attention kernel's work items: for every mask head, the pairs of query
-// blocks sorted by decreasing cost (the longer of the two kept lists), so that the long items
-// start first and the short ones fill the tail.  Counting sort in shared memory; one CTA per
-// mask head.  The order among equal costs is arbitrary (it only affects scheduling).
-// It is the first kernel of a call, so it also clears the status words the later kernels test.
 // Diagnostic: one thread waits, with a 2 ms limit, on an mbarrier that nothing ever arrives on, and
 // reports the expiry the way the compute kernels do (status word = -6).  It exercises the bounded
 // wait and the status path without any fault: the kernel returns normally.
@@ -135,6 +130,11 @@ __global__ void __launch_bounds__(32) status_clear_kernel(int32_t* __restrict__ 
     }
 }
 
+// Launch order of the attention kernel's work items: for every mask head, the query blocks
+// sorted by decreasing length of their kept list, so that the long items start first and the
+// short ones fill the tail.  Counting sort in shared memory; one CTA per mask head.  The order
+// among equal costs is arbitrary (it only affects scheduling).
+// It is the first kernel of a call, so it also clears the status words the later kernels test.
 __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
                                                           int32_t* __restrict__ order,
                                                           int32_t* __restrict__ ws_status,
@@ -148,11 +148,10 @@ __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restr
     __shared__ int hist[BINS];
     const int hm = blockIdx.x, tid = threadIdx.x;
     const int32_t* rp = row_ptr + size_t(hm) * nQb;
-    const int nPairs = nQb;           // one work item per query block
-    auto cost_of = [&](int pr) { return min(BINS - 1, rp[pr + 1] - rp[pr]); };
+    auto cost_of = [&](int qb) { return min(BINS - 1, rp[qb + 1] - rp[qb]); };
     for (int i = tid; i < BINS; i += blockDim.x) hist[i] = 0;
     __syncthreads();
-    for (int pr = tid; pr < nPairs; pr += blockDim.x) atomicAdd(&hist[cost_of(pr)], 1);
+    for (int qb = tid; qb < nQb; qb += blockDim.x) atomicAdd(&hist[cost_of(qb)], 1);
     __syncthreads();
     // start position of every cost, largest cost first: an exclusive suffix sum over the bins,
     // two bins per thread, Hillis-Steele over the per-thread totals
@@ -170,8 +169,8 @@ __global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restr
     hist[2 * tid + 1] = above;
     hist[2 * tid] = above + h1;
     __syncthreads();
-    for (int pr = tid; pr < nPairs; pr += blockDim.x)
-        order[size_t(hm) * nPairs + atomicAdd(&hist[cost_of(pr)], 1)] = pr;
+    for (int qb = tid; qb < nQb; qb += blockDim.x)
+        order[size_t(hm) * nQb + atomicAdd(&hist[cost_of(qb)], 1)] = qb;
 }
 
 }  // namespace salad
