@@ -29,6 +29,9 @@
 // writes
 //     O = O_acc / l + (s_b lambda_h / (den + eps)) * num
 // once, as bf16, through a TMA store.
+// The kernels that make the linear state come before this one in the stream and run beside it: this
+// kernel is launched to start early and waits for them only in warp 0, just before the state tile and
+// the normaliser Z are fetched, so the softmax attention of the first tiles hides the state pass.
 //
 // TMEM columns (256 allocated):  [0,64) and [64,128) two score buffers (block t uses buffer
 // t & 1; its probabilities, packed bf16, overwrite the first 32 columns of the same buffer);
@@ -92,7 +95,7 @@ static_assert(FusedCfg<64>::ST_BYTES <= FusedCfg<64>::NK * FusedCfg<64>::KV_BYTE
 
 struct FusedBarriers {
     uint64_t q_full, st_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
-    uint64_t s_full[2], p_ready[2], pv_done[2], o_final, lin_ready, lin_done, out_staged;
+    uint64_t s_full[2], p_ready[2], pv_done[2], o_final, lin_ready, lin_done, out_staged, z_full;
 };
 
 template <int D>
@@ -111,7 +114,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    grid_dependency_wait();           // the order and the linear state come from the kernels before
+    // The work order comes from the first kernel of the call.  Without a linear branch that is the kernel
+    // before this one.  With one, the state kernels lie between, and this kernel does not wait for them
+    // here: it runs beside them (each of their CTAs has passed its own wait for the first kernel before
+    // a CTA of this one is placed) and waits only where it first touches the state, in the epilogue.
+    if ((p.mode & MODE_LINEAR) == 0) grid_dependency_wait();
     grid_launch_dependents();
 
     // work item: head by head (K/V of one head stay hot in L2: ordering the cheapest items of all
@@ -143,6 +150,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(smem_u32(&bars.lin_ready), 256);
         mbar_init(smem_u32(&bars.lin_done), 1);
         mbar_init(smem_u32(&bars.out_staged), 256);
+        mbar_init(smem_u32(&bars.z_full), 32);
         for (int j = 0; j < 2; ++j) {
             mbar_init(smem_u32(&bars.s_full[j]), 1);
             mbar_init(smem_u32(&bars.p_ready[j]), 8);          // one arrival per softmax warp
@@ -165,7 +173,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         fence_proxy_async_smem();
     }
     if (warp == 2) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
-    if (linear && tid >= 128 && tid < 128 + D) z_s[tid - 128] = __ldg(p.z + size_t(bh) * D + (tid - 128));
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -177,6 +184,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (abort_flag == 0) {
     if (warp == 0) {
         // ============================================================== TMA producer: Q, the K ring, the state tile
+        bool ok = true;
         if (lane == 0) {
             prefetch_tmap(&map_q); prefetch_tmap(&map_k);
             // A block with no kept key block and no linear branch never reads Q: its epilogue
@@ -187,7 +195,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 for (int ch = 0; ch < C::CH; ++ch)
                     tma_load_3d(s_base + C::OFF_Q + ch * C::Q_CHUNK, &map_q, bar, ch * 64, qb * p.Bq, bh);
             }
-            bool ok = true;
             for (int t = 0; t < len; ++t) {
                 const int s = t % C::NK;
                 ok = mbar_wait(smem_u32(&bars.k_empty[s]), ((t / C::NK) & 1) ^ 1, abortp);
@@ -199,7 +206,16 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tma_load_3d(s_base + C::OFF_K + s * C::KV_BYTES + ch * C::KV_CHUNK, &map_k, bar, ch * 64,
                                 col * C::BK, bh);
             }
-            if (ok && linear) {
+        }
+        if (linear) {
+            // From here on the linear state is needed: wait for the kernels that make it (whole warp: the
+            // other lanes fetch the normaliser Z of this head for the softmax warps meanwhile).
+            __syncwarp();
+            grid_dependency_wait();
+            if (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) *abortp = 1;     // the state kernel gave up
+            for (int a = lane; a < D; a += 32) z_s[a] = __ldcg(p.z + size_t(bh) * D + a);
+            mbar_arrive(smem_u32(&bars.z_full));
+            if (lane == 0 && ok) {
                 // the state tile goes over the K ring: every Q K^T must have read its K block.  The products
                 // complete in order, so the last one (signalled on its score buffer's barrier) covers all.
                 if (len > 0) ok = mbar_wait(smem_u32(&bars.s_full[(len - 1) & 1]), ((len - 1) >> 1) & 1, abortp);
@@ -433,6 +449,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // completed (its scores were consumed above), so Q is no longer read; the last P V
             // product may still be running meanwhile.
             ok = wait_uniform(&bars.q_full, 0);
+            if (ok) ok = wait_uniform(&bars.z_full, 0);
             if (ok) {
                 float den_a = 0.f, den_b = 0.f;
 #pragma unroll

@@ -2,7 +2,8 @@
 //
 // HBM-bound: K and V are read exactly once.  The token axis of every (batch, head) is cut
 // into `chunks` contiguous ranges of key blocks (64 tokens); one CTA per SM streams one range
-// through a six-stage ring (192 KB in flight per SM):
+// through a ring of stages (linear-only calls: six, 192 KB in flight per SM; fused calls: three,
+// so that a CTA of the attention kernel fits on the SM beside it and starts meanwhile):
 //   warp 0      TMA producer, K and V tiles through a ring of stages
 //   warp 1      tcgen05 MMA issuer; per 16 tokens one MMA  D[d x d] += ReLU(K)^T V with both
 //               operands token-major in shared memory (MN-major descriptors), plus one
@@ -22,14 +23,14 @@
 
 namespace salad {
 
-template <int D>
+template <int D, bool OVERLAP>
 struct StateCfg {
     static constexpr int BK = 64;
     static constexpr int CH = D / 64;
     static constexpr int T_CHUNK = BK * 128;           // bytes of one 64-column chunk of a tile
     static constexpr int T_BYTES = CH * T_CHUNK;       // one K or V tile
     static constexpr int STAGE_BYTES = 2 * T_BYTES;    // K then V
-    static constexpr int STAGES = (D == 128) ? 6 : 8;
+    static constexpr int STAGES = OVERLAP ? 3 : ((D == 128) ? 6 : 8);
     static constexpr int OFF_ONES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = OFF_ONES + 2048 + 1024;
     static constexpr int THREADS = 192;
@@ -53,12 +54,12 @@ __device__ __forceinline__ bool branch_dropped(const float* dyn_scale, float tau
     return dyn_scale != nullptr && __ldg(dyn_scale + b) < tau;
 }
 
-template <int D>
+template <int D, bool OVERLAP>
 __global__ void __launch_bounds__(192)
 salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                           const StateParams p)
 {
-    using C = StateCfg<D>;
+    using C = StateCfg<D, OVERLAP>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full[C::STAGES], relu_done[C::STAGES], empty[C::STAGES], acc_done;
     __shared__ uint32_t tmem_base_slot;
@@ -68,7 +69,10 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x, bh = blockIdx.y;
-    if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) return;     // whole CTA, before any allocation
+    if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) {           // whole CTA, before any allocation
+        grid_dependency_wait();        // an exit releases the kernels after this one: not before the kernel before it is done
+        return;
+    }
     const int kb0 = chunk * p.blocks_per_chunk;
     const int kb1 = min(p.nKb, kb0 + p.blocks_per_chunk);
     const int nblk = max(0, kb1 - kb0);
@@ -214,23 +218,27 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 //   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
 //           num = ReLU(Q) KV in the fused kernel.
 template <int D>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(256)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
                              __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
-    grid_dependency_wait();
+    // The kernel after this one may be placed at once (it waits for this one before it touches the
+    // state); this one is small, 256 threads and few registers, so that while it waits for the state
+    // kernel it does not keep a CTA of the attention kernel off its SM.
     grid_launch_dependents();
+    grid_dependency_wait();
     if (branch_dropped(dyn_scale, drop_tau, blockIdx.z / H)) return;
-    // grid (D/32, D/32, BH), block (32, 32): one 32 x 32 tile of KV per block, one element per
+    // grid (D/32, D/32, BH), block (32, 8): one 32 x 32 tile of KV per block, four elements per
     // thread, transposed through shared memory so that both the partial reads and the bf16
     // writes are coalesced
     __shared__ float tile[32][33];
     const int bh = blockIdx.z;
     const int a0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
     const int tx = threadIdx.x, ty = threadIdx.y;
-    {
-        const int a = a0 + ty;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int a = a0 + ty + 8 * r;
         const float* src = kv_part + size_t(bh) * chunks * D * D + size_t(a) * D + c0 + tx;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
         int ch = 0;
@@ -243,12 +251,14 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
         for (; ch < chunks; ++ch) s0 += src[size_t(ch) * D * D];
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
-        tile[ty][tx] = s;
+        tile[ty + 8 * r][tx] = s;
     }
     __syncthreads();
-    kvt[size_t(bh) * D * D + size_t(c0 + ty) * D + a0 + tx] = __float2bfloat16(tile[tx][ty]);
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+        kvt[size_t(bh) * D * D + size_t(c0 + ty + 8 * r) * D + a0 + tx] = __float2bfloat16(tile[tx][ty + 8 * r]);
     if (blockIdx.x == 0 && blockIdx.y == 0) {
-        for (int a = ty * 32 + tx; a < D; a += 1024) {
+        for (int a = ty * 32 + tx; a < D; a += 256) {
             const float* src = z_part + size_t(bh) * chunks * D + a;
             float s = 0.f;
             for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];

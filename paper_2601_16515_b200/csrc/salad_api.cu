@@ -96,11 +96,23 @@ int prepare_device(DeviceInfo* info) {
             e = cudaFuncSetAttribute(salad_fused_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<128>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128, false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<64>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64, false>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128, true>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64, true>::SMEM_BYTES);
+        if (e == cudaSuccess)      // beside a CTA of the attention kernel
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_linear_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      ApplyCfg<128>::SMEM_BYTES);
@@ -194,10 +206,15 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.user_status = P.d_status;
     sp.dyn_scale = P.dyn_scale; sp.drop_tau = P.drop_tau; sp.H = P.H;
     record_profile(0, P.stream);
-    launch_dependent(salad_linear_state_kernel<D>, dim3(chunks, BH), dim3(StateCfg<D>::THREADS),
-                     StateCfg<D>::SMEM_BYTES, P.stream, mk, mv, sp);
+    // fused calls: the short-ring variant, which shares its SM with a CTA of the attention kernel
+    if (P.mode & MODE_SPARSE)
+        launch_dependent(salad_linear_state_kernel<D, true>, dim3(chunks, BH), dim3(StateCfg<D, true>::THREADS),
+                         StateCfg<D, true>::SMEM_BYTES, P.stream, mk, mv, sp);
+    else
+        launch_dependent(salad_linear_state_kernel<D, false>, dim3(chunks, BH), dim3(StateCfg<D, false>::THREADS),
+                         StateCfg<D, false>::SMEM_BYTES, P.stream, mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    launch_dependent(salad_linear_finalize_kernel<D>, dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream,
+    launch_dependent(salad_linear_finalize_kernel<D>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
                      sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
                      reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt), P.dyn_scale, P.drop_tau, P.H);
     record_profile(1, P.stream);
