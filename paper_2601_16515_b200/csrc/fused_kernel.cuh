@@ -211,7 +211,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // From here on the linear state is needed: wait for the kernels that make it (whole warp: the
             // other lanes fetch the normaliser Z of this head for the softmax warps meanwhile).
             __syncwarp();
+            if (lane == 0) TRACE_CTA(2);
             grid_dependency_wait();
+            if (lane == 0) TRACE_CTA(3);
             if (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) *abortp = 1;     // the state kernel gave up
             for (int a = lane; a < D; a += 32) z_s[a] = __ldcg(p.z + size_t(bh) * D + a);
             mbar_arrive(smem_u32(&bars.z_full));
@@ -566,6 +568,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
         __syncthreads();
     }
+    if (tid == 0) TRACE_CTA(5);
     if (warp == 2) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

@@ -217,19 +217,20 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 //   kv_out  fp32 [BH][D][D]  (optional)      z fp32 [BH][D]  (+ optional user copy)
 //   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
 //           num = ReLU(Q) KV in the fused kernel.
-template <int D>
-__global__ void __launch_bounds__(256)
+template <int D, int ROWS>
+__global__ void __launch_bounds__(32 * ROWS)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
                              float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
                              __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
     // The kernel after this one may be placed at once (it waits for this one before it touches the
-    // state); this one is small, 256 threads and few registers, so that while it waits for the state
-    // kernel it does not keep a CTA of the attention kernel off its SM.
+    // state).  In fused calls ROWS = 8: a block is small, 256 threads and few registers, so that while it
+    // waits for the state kernel it does not keep a CTA of the attention kernel off its SM.  In linear-only
+    // calls, where this kernel's latency counts, ROWS = 32: one element per thread.
     grid_launch_dependents();
     grid_dependency_wait();
     if (branch_dropped(dyn_scale, drop_tau, blockIdx.z / H)) return;
-    // grid (D/32, D/32, BH), block (32, 8): one 32 x 32 tile of KV per block, four elements per
+    // grid (D/32, D/32, BH), block (32, ROWS): one 32 x 32 tile of KV per block, 32 / ROWS elements per
     // thread, transposed through shared memory so that both the partial reads and the bf16
     // writes are coalesced
     __shared__ float tile[32][33];
@@ -237,8 +238,8 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
     const int a0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
     const int tx = threadIdx.x, ty = threadIdx.y;
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const int a = a0 + ty + 8 * r;
+    for (int r = 0; r < 32 / ROWS; ++r) {
+        const int a = a0 + ty + ROWS * r;
         const float* src = kv_part + size_t(bh) * chunks * D * D + size_t(a) * D + c0 + tx;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
         int ch = 0;
@@ -251,14 +252,14 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
         for (; ch < chunks; ++ch) s0 += src[size_t(ch) * D * D];
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
-        tile[ty + 8 * r][tx] = s;
+        tile[ty + ROWS * r][tx] = s;
     }
     __syncthreads();
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-        kvt[size_t(bh) * D * D + size_t(c0 + ty + 8 * r) * D + a0 + tx] = __float2bfloat16(tile[tx][ty + 8 * r]);
+    for (int r = 0; r < 32 / ROWS; ++r)
+        kvt[size_t(bh) * D * D + size_t(c0 + ty + ROWS * r) * D + a0 + tx] = __float2bfloat16(tile[tx][ty + ROWS * r]);
     if (blockIdx.x == 0 && blockIdx.y == 0) {
-        for (int a = ty * 32 + tx; a < D; a += 256) {
+        for (int a = ty * 32 + tx; a < D; a += 32 * ROWS) {
             const float* src = z_part + size_t(bh) * chunks * D + a;
             float s = 0.f;
             for (int ch = 0; ch < chunks; ++ch) s += src[size_t(ch) * D];

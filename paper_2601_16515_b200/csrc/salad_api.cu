@@ -214,12 +214,21 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
         launch_dependent(salad_linear_state_kernel<D, false>, dim3(chunks, BH), dim3(StateCfg<D, false>::THREADS),
                          StateCfg<D, false>::SMEM_BYTES, P.stream, mk, mv, sp);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    launch_dependent(salad_linear_finalize_kernel<D>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
-                     sp.kv_part, sp.z_part, chunks, P.kv_out, reinterpret_cast<float*>(ws + w.off_z), P.z_out,
-                     reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt), P.dyn_scale, P.drop_tau, P.H);
+    float* z_ws = reinterpret_cast<float*>(ws + w.off_z);
+    __nv_bfloat16* kvt = reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt);
+    if (P.mode & MODE_SPARSE)
+        launch_dependent(salad_linear_finalize_kernel<D, 8>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+    else
+        launch_dependent(salad_linear_finalize_kernel<D, 32>, dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream,
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
     record_profile(1, P.stream);
     return check_launch();
 }
+
+#ifdef SALAD_TRACE
+float* g_trace_buffer = nullptr;
+#endif
 
 template <int D>
 int launch_fused(const Problem& P, const Workspace& w) {
@@ -241,6 +250,9 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.static_scale = P.static_scale; fp.dyn_scale = P.dyn_scale;
     fp.z = reinterpret_cast<const float*>(ws + w.off_z);
     fp.lse = P.lse;
+#ifdef SALAD_TRACE
+    if (!fp.lse) fp.lse = g_trace_buffer;      // trace builds only: time stamps go where the LSE would
+#endif
     const float sc = (P.softmax_scale > 0.f) ? P.softmax_scale : 1.0f / sqrtf(float(D));
     fp.scale_log2 = sc * 1.4426950408889634f;
     fp.eps = P.eps;
@@ -668,3 +680,7 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     if (rc != SALAD_OK) return rc;
     return (d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
 }
+
+#ifdef SALAD_TRACE
+extern "C" __attribute__((visibility("default"))) void salad_trace_set_buffer(float* d_buf) { g_trace_buffer = d_buf; }
+#endif
