@@ -21,11 +21,14 @@
  *
  * Pins (see tests): dense masked softmax written as an N x N matrix (Eq. 2 literally),
  * the library routine torch SDPA, the un-reordered N x N form of Eq. 3, closed forms
- * (constant V, zero K, homogeneity in K), hand-counted window masks.
+ * (constant V, zero K, homogeneity in K), hand-counted window masks; for the rotary linear branch a
+ * two-token example worked by hand, the N x N form with explicit rotation matrices, zero angles
+ * (plain Eq. 3), invariance under a common shift of all positions.
  *
  * Parity unpinned: nothing ties these functions to the authors' own implementation (the
  * paper prints no worked numeric example); the 3-D window reading of the ST-SWA mask and
- * the per-head scalar reading of the static projection are this build's readings.
+ * the per-head scalar reading of the static projection are this build's readings, and so is the
+ * place of the rotary embedding in the linear branch (numerator only), for which the paper has no formula.
  */
 #include <math.h>
 #include <stdint.h>
@@ -385,4 +388,115 @@ ORACLE_API void oracle_proj_combine(const float* o_s, const float* o_l, const fl
             }
         }
     }
+}
+
+/*
+ * Linear branch with rotary position embedding.  Sec. 4.1 states that the linear branch carries a
+ * 3-D rotary embedding and gives no formula; the form taken here is the one the rotary-embedding
+ * paper it cites defines for linear attention: the rotation enters the numerator only,
+ *     O_l[n] = sum_j < R_n ReLU(Q_n), R_j ReLU(K_j) > V_j  /  ( sum_j < ReLU(Q_n), ReLU(K_j) > + eps ),
+ * so that the normaliser keeps its sign.  R_n rotates the channel pair (2i, 2i+1) of token n by an
+ * angle given through its cosine and sine, rope[n][i][0] and rope[n][i][1] (fp32, an input: for a 3-D
+ * embedding the pairs are shared out among the t, h and w axes of the latent grid).
+ *
+ * rotate_pairs:  y[2i] = c x[2i] - s x[2i+1],   y[2i+1] = s x[2i] + c x[2i+1].
+ */
+static void rotate_pairs(const double* x, const float* cs, int d, double* y)
+{
+    for (int i = 0; i < d / 2; ++i) {
+        double c = (double)cs[2 * i], s = (double)cs[2 * i + 1];
+        y[2 * i] = c * x[2 * i] - s * x[2 * i + 1];
+        y[2 * i + 1] = s * x[2 * i] + c * x[2 * i + 1];
+    }
+}
+
+/*
+ * oracle_linear_state_rope: the two reductions of Eq. 3 with rotated keys in the first,
+ *     KV[b,h] = sum_j (R_j ReLU(K_j))^T V_j,     Z[b,h] = sum_j ReLU(K_j)   (not rotated).
+ */
+ORACLE_API void oracle_linear_state_rope(const float* k, const float* v, const float* rope,
+                                         int B, int H, int N, int d, double* kv, double* z)
+{
+    int64_t BH = (int64_t)B * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < BH; ++bh) {
+        const float* kb = k + bh * (int64_t)N * d;
+        const float* vb = v + bh * (int64_t)N * d;
+        double* kvb = kv + bh * (int64_t)d * d;
+        double* zb = z + bh * (int64_t)d;
+        double* f = (double*)malloc(sizeof(double) * (size_t)d);
+        double* fr = (double*)malloc(sizeof(double) * (size_t)d);
+        for (int64_t i = 0; i < (int64_t)d * d; ++i) kvb[i] = 0.0;
+        for (int a = 0; a < d; ++a) zb[a] = 0.0;
+        for (int j = 0; j < N; ++j) {
+            for (int a = 0; a < d; ++a) f[a] = relu((double)kb[(int64_t)j * d + a]);
+            rotate_pairs(f, rope + (int64_t)j * d, d, fr);
+            const float* vj = vb + (int64_t)j * d;
+            for (int a = 0; a < d; ++a) {
+                zb[a] += f[a];
+                for (int c = 0; c < d; ++c) kvb[(int64_t)a * d + c] += fr[a] * (double)vj[c];
+            }
+        }
+        free(f); free(fr);
+    }
+}
+
+/*
+ * oracle_linear_attn_rope: for selected rows, from that state,
+ *     O_l[n] = (R_n ReLU(Q_n)) KV / (ReLU(Q_n) . Z + eps).
+ */
+ORACLE_API void oracle_linear_attn_rope(const float* q, const float* rope, const double* kv, const double* z,
+                                        int B, int H, int N, int d, double eps,
+                                        const int64_t* sel, int64_t nsel, double* o_l)
+{
+    if (!sel) nsel = (int64_t)B * H * N;
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsel; ++s) {
+        int64_t bh; int n;
+        decode_row(sel, s, N, &bh, &n);
+        const float* qn = q + (bh * N + n) * (int64_t)d;
+        const double* kvb = kv + bh * (int64_t)d * d;
+        const double* zb = z + bh * (int64_t)d;
+        double* f = (double*)malloc(sizeof(double) * (size_t)d);
+        double* fr = (double*)malloc(sizeof(double) * (size_t)d);
+        double den = 0.0;
+        for (int a = 0; a < d; ++a) { f[a] = relu((double)qn[a]); den += f[a] * zb[a]; }
+        rotate_pairs(f, rope + (int64_t)n * d, d, fr);
+        double* on = o_l + s * (int64_t)d;
+        for (int c = 0; c < d; ++c) {
+            double num = 0.0;
+            for (int a = 0; a < d; ++a) num += fr[a] * kvb[(int64_t)a * d + c];
+            on[c] = num / (den + eps);
+        }
+        free(f); free(fr);
+    }
+}
+
+/*
+ * oracle_salad_fused_rope: Algorithm 1 with that linear branch and the drop threshold of Sec. 4.3,
+ *     O[b,h,n] = O_s[b,h,n] + [s[b] >= tau] * s[b] * lambda[h] * O_l[b,h,n]      (tau = -inf: never dropped).
+ */
+ORACLE_API void oracle_salad_fused_rope(const float* q, const float* k, const float* v, const float* rope,
+                                        int B, int H, int N, int d, int Bq, int Bk,
+                                        const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                        const double* lambda_h, const double* s_b, double tau,
+                                        double scale, double eps,
+                                        const int64_t* sel, int64_t nsel, double* o)
+{
+    if (!sel) nsel = (int64_t)B * H * N;
+    int64_t BH = (int64_t)B * H;
+    double* kv = (double*)malloc(sizeof(double) * (size_t)(BH * d * d));
+    double* z = (double*)malloc(sizeof(double) * (size_t)(BH * d));
+    double* ol = (double*)malloc(sizeof(double) * (size_t)(nsel * d));
+    oracle_sparse_attn(q, k, v, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, scale, sel, nsel, o, NULL);
+    oracle_linear_state_rope(k, v, rope, B, H, N, d, kv, z);
+    oracle_linear_attn_rope(q, rope, kv, z, B, H, N, d, eps, sel, nsel, ol);
+    for (int64_t s = 0; s < nsel; ++s) {
+        int64_t bh; int n;
+        decode_row(sel, s, N, &bh, &n);
+        double sb = s_b[bh / H];
+        double c = (sb >= tau) ? sb * lambda_h[bh % H] : 0.0;
+        for (int a = 0; a < d; ++a) o[s * d + a] += c * ol[s * d + a];
+    }
+    free(kv); free(z); free(ol);
 }

@@ -57,6 +57,13 @@ def _load():
         lib.oracle_proj_combine.argtypes = [p, p, p, p, p, i32, i32, i32, i32, p]
         lib.oracle_topk_mask.restype = None
         lib.oracle_topk_mask.argtypes = [p, p] + [i32] * 7 + [p, p]
+        lib.oracle_linear_state_rope.restype = None
+        lib.oracle_linear_state_rope.argtypes = [p, p, p] + [i32] * 4 + [p, p]
+        lib.oracle_linear_attn_rope.restype = None
+        lib.oracle_linear_attn_rope.argtypes = [p, p, p, p] + [i32] * 4 + [f64, p, i64, p]
+        lib.oracle_salad_fused_rope.restype = None
+        lib.oracle_salad_fused_rope.argtypes = ([p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
+                                                                            p, i64, p])
         _lib = lib
     return _lib
 
@@ -256,3 +263,58 @@ def proj_combine(o_s, o_l, w, s_b, bias=None):
     out = np.empty((B, H, N, d), dtype=np.float64)
     lib.oracle_proj_combine(sp, lp, wp, bp, sb.ctypes.data, B, H, N, d, out.ctypes.data)
     return out
+
+
+def _rope(rope, N, d):
+    r = np.ascontiguousarray(rope, dtype=np.float32)
+    assert r.shape == (N, d // 2, 2), "rope is [N, d/2, 2]: cosine and sine of the angle of every token and channel pair"
+    return r, r.ctypes.data
+
+
+def linear_state_rope(k, v, rope):
+    """Linear state with rotated keys: KV = sum_j (R_j ReLU(K_j))^T V_j, Z = sum_j ReLU(K_j).
+    Returns (KV [B,H,d,d], Z [B,H,d]) float64."""
+    lib = _load()
+    k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = k.shape
+    r, rp = _rope(rope, N, d)
+    kv = np.empty((B, H, d, d), dtype=np.float64)
+    z = np.empty((B, H, d), dtype=np.float64)
+    lib.oracle_linear_state_rope(kp, vp, rp, B, H, N, d, kv.ctypes.data, z.ctypes.data)
+    return kv, z
+
+
+def linear_attn_rope(q, k, v, rope, eps=1e-6, sel=None, state=None):
+    """Eq. 3 with the rotary embedding in the numerator.  Returns O_l [rows, d] float64."""
+    lib = _load()
+    q, qp = _f32(q)
+    B, H, N, d = q.shape
+    r, rp = _rope(rope, N, d)
+    kv, z = state if state is not None else linear_state_rope(k, v, rope)
+    kv = np.ascontiguousarray(kv, dtype=np.float64); z = np.ascontiguousarray(z, dtype=np.float64)
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    lib.oracle_linear_attn_rope(qp, rp, kv.ctypes.data, z.ctypes.data, B, H, N, d, float(eps),
+                                sp, nsel, o.ctypes.data)
+    return o
+
+
+def salad_fused_rope(q, k, v, rope, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, tau=-np.inf, scale=None,
+                     eps=1e-6, sel=None):
+    """Algorithm 1 with the rotary linear branch (and the drop threshold tau).  [rows, d] float64."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = q.shape
+    r, rop = _rope(rope, N, d)
+    rp, rpp = _i32(row_ptr); ci, cip = _i32(col_idx if len(col_idx) else np.zeros(1, np.int32))
+    lam = np.ascontiguousarray(lambda_h, dtype=np.float64); sb = np.ascontiguousarray(s_b, dtype=np.float64)
+    assert lam.size == H and sb.size == B
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    lib.oracle_salad_fused_rope(qp, kp, vp, rop, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
+                                sb.ctypes.data, float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
+    return o

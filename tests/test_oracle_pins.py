@@ -518,3 +518,133 @@ def test_proj_combine_block_diagonal_is_the_fused_path():
     # o_s and o_l pass through fp32 in the wrapper: compare at that precision
     ref = orc.salad_fused(q, k, v, 16, 16, rp, ci, 1, lam, s).reshape(B, H, N, d)
     np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
+
+
+# ----------------------------------------------------------------------------------------
+# Linear branch with the rotary embedding (Sec. 4.1: the linear branch carries a 3-D rotary
+# embedding; rotation in the numerator only, the normaliser un-rotated)
+
+def _rotation_matrix(cs):
+    """Dense d x d block-diagonal rotation of one token from its [d/2, 2] cosine/sine rows."""
+    d = 2 * cs.shape[0]
+    R = np.zeros((d, d))
+    for i, (c, s) in enumerate(cs.astype(np.float64)):
+        R[2 * i, 2 * i] = c;  R[2 * i, 2 * i + 1] = -s
+        R[2 * i + 1, 2 * i] = s;  R[2 * i + 1, 2 * i + 1] = c
+    return R
+
+
+def _angles_table(ang):
+    return np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)
+
+
+def test_rope_linear_hand_example():
+    # d = 2 (one pair), two tokens with angles 0 and pi/2, eps = 0.
+    #   keys   k0 = (1, 0), k1 = (0, 1); rotated: (1, 0) and R(pi/2)(0, 1) = (-1, 0)
+    #   values v0 = (2, 3), v1 = (5, 7)
+    #   query 0 = (1, 0), angle 0:    weights <(1,0),(1,0)> = 1 and <(1,0),(-1,0)> = -1, normaliser 1 + 0
+    #                                 -> O_l = v0 - v1 = (-3, -4)
+    #   query 1 = (0, 1), angle pi/2: rotated (-1, 0): weights -1 and 1, normaliser 0 + 1 -> v1 - v0 = (3, 4)
+    q = np.array([[1.0, 0.0], [0.0, 1.0]], dtype=np.float32).reshape(1, 1, 2, 2)
+    k = np.array([[1.0, 0.0], [0.0, 1.0]], dtype=np.float32).reshape(1, 1, 2, 2)
+    v = np.array([[2.0, 3.0], [5.0, 7.0]], dtype=np.float32).reshape(1, 1, 2, 2)
+    rope = np.array([[[1.0, 0.0]], [[0.0, 1.0]]], dtype=np.float32)      # cos, sin of 0 and pi/2
+    o = orc.linear_attn_rope(q, k, v, rope, eps=0.0)
+    np.testing.assert_allclose(o, [[-3.0, -4.0], [3.0, 4.0]], atol=1e-12)
+    kv, z = orc.linear_state_rope(k, v, rope)
+    np.testing.assert_allclose(kv[0, 0], [[2.0 - 5.0, 3.0 - 7.0], [0.0, 0.0]], atol=1e-12)
+    np.testing.assert_allclose(z[0, 0], [1.0, 1.0], atol=1e-12)
+
+
+def test_rope_linear_vs_explicit_quadratic_form():
+    B, H, N, d = 1, 2, 37, 8
+    q, k, v = rand_qkv(B, H, N, d, 41)
+    rng = np.random.default_rng(5)
+    rope = _angles_table(rng.uniform(-np.pi, np.pi, size=(N, d // 2)))
+    eps = 1e-6
+    got = orc.linear_attn_rope(q, k, v, rope, eps=eps).reshape(B, H, N, d)
+    R = [_rotation_matrix(rope[n]) for n in range(N)]
+    for h in range(H):
+        fq = np.maximum(q[0, h].astype(np.float64), 0.0)
+        fk = np.maximum(k[0, h].astype(np.float64), 0.0)
+        qr = np.stack([R[n] @ fq[n] for n in range(N)])
+        kr = np.stack([R[n] @ fk[n] for n in range(N)])
+        w = qr @ kr.T                                   # [N, N] rotated similarities
+        den = (fq @ fk.T).sum(axis=1) + eps             # un-rotated normaliser
+        want = (w @ v[0, h].astype(np.float64)) / den[:, None]
+        np.testing.assert_allclose(got[0, h], want, rtol=1e-10, atol=1e-12)
+
+
+def test_rope_linear_special_cases():
+    B, H, N, d = 2, 2, 50, 16
+    q, k, v = rand_qkv(B, H, N, d, 43)
+    # zero angles: the plain linear attention of Eq. 3
+    ident = _angles_table(np.zeros((N, d // 2)))
+    np.testing.assert_allclose(orc.linear_attn_rope(q, k, v, ident), orc.linear_attn(q, k, v), rtol=1e-12, atol=1e-14)
+    kv0, z0 = orc.linear_state(k, v)
+    kv1, z1 = orc.linear_state_rope(k, v, ident)
+    np.testing.assert_allclose(kv1, kv0, rtol=1e-12); np.testing.assert_allclose(z1, z0, rtol=1e-12)
+    # relative positions only: angle = position * frequency; moving every token by the same offset
+    # changes nothing
+    freq = 10000.0 ** (-np.arange(d // 2) / (d // 2))
+    pos = np.arange(N, dtype=np.float64)
+    a = orc.linear_attn_rope(q, k, v, _angles_table(pos[:, None] * freq[None, :]))
+    b = orc.linear_attn_rope(q, k, v, _angles_table((pos[:, None] + 17.0) * freq[None, :]))
+    np.testing.assert_allclose(a, b, rtol=1e-5, atol=1e-6)          # the tables are fp32
+    assert np.abs(a - orc.linear_attn(q, k, v)).max() > 1e-2          # and the rotation does something
+    # the normaliser ignores the rotation: the state's Z is the plain one for any table
+    rng = np.random.default_rng(9)
+    rope = _angles_table(rng.uniform(-np.pi, np.pi, size=(N, d // 2)))
+    _, z2 = orc.linear_state_rope(k, v, rope)
+    np.testing.assert_allclose(z2, z0, rtol=1e-12)
+    # a rotation by pi flips the sign of the rotated keys and queries alike: numerator unchanged
+    flip = _angles_table(np.full((N, d // 2), np.pi))
+    np.testing.assert_allclose(orc.linear_attn_rope(q, k, v, flip), orc.linear_attn(q, k, v), rtol=1e-5, atol=1e-6)
+    # row selection gives the same rows
+    sel = np.array([0, 7, N * 3 + 11, B * H * N - 1], dtype=np.int64)
+    full = orc.linear_attn_rope(q, k, v, rope)
+    np.testing.assert_allclose(orc.linear_attn_rope(q, k, v, rope, sel=sel), full[sel], rtol=1e-12)
+
+
+def test_rope_fused_pins():
+    wl = wlmod.C1
+    q, k, v = (t.float().numpy() for t in wlmod.make_qkv(wl))
+    T, Hs, Ws = wl.grid
+    rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    lam, s = wlmod.make_scales(wl)
+    sel = wlmod.sample_rows(wl, 64, seed=3)
+    rope = wlmod.rope_table(wl.grid, wl.d)
+    # zero angles: Algorithm 1 as before
+    ident = _angles_table(np.zeros((wl.N, wl.d // 2)))
+    a = orc.salad_fused_rope(q, k, v, ident, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s, sel=sel)
+    b = orc.salad_fused(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s, sel=sel)
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-14)
+    # the sum of its parts
+    o_s, _ = orc.sparse_attn(q, k, v, wl.Bq, wl.Bk, rp, ci, wl.Hm, sel=sel)
+    o_l = orc.linear_attn_rope(q, k, v, rope, sel=sel)
+    heads = (sel // wl.N) % wl.H
+    want = o_s + (np.float64(s[0]) * lam.astype(np.float64)[heads])[:, None] * o_l
+    got = orc.salad_fused_rope(q, k, v, rope, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s, sel=sel)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-14)
+    # dropped branch: the sparse output alone
+    dropped = orc.salad_fused_rope(q, k, v, rope, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s, tau=2.0, sel=sel)
+    np.testing.assert_allclose(dropped, o_s, rtol=0, atol=0)
+
+
+def test_rope_table_generator():
+    grid, d = (3, 4, 5), 32
+    r = wlmod.rope_table(grid, d).astype(np.float64)
+    N = 3 * 4 * 5
+    assert r.shape == (N, d // 2, 2)
+    np.testing.assert_allclose((r ** 2).sum(-1), 1.0, atol=1e-6)
+    np.testing.assert_allclose(r[0, :, 0], 1.0); np.testing.assert_allclose(r[0, :, 1], 0.0)   # origin: no rotation
+    p_hw = (d // 2) // 3; p_t = d // 2 - 2 * p_hw
+    n = lambda t, h, w: (t * 4 + h) * 5 + w
+    # a step along w changes only the w pairs, by the pair's frequency
+    np.testing.assert_allclose(r[n(1, 2, 3), :p_t + p_hw], r[n(1, 2, 4), :p_t + p_hw])
+    ang = np.arctan2(r[n(0, 0, 1), p_t + p_hw:, 1], r[n(0, 0, 1), p_t + p_hw:, 0])
+    np.testing.assert_allclose(ang, 10000.0 ** (-np.arange(p_hw) / p_hw), rtol=1e-5)
+    # along t only the first p_t pairs change
+    np.testing.assert_allclose(r[n(0, 2, 3), p_t:], r[n(2, 2, 3), p_t:])
+    ang_t = np.arctan2(r[n(1, 0, 0), :p_t, 1], r[n(1, 0, 0), :p_t, 0])
+    np.testing.assert_allclose(ang_t, 10000.0 ** (-np.arange(p_t) / p_t), rtol=1e-5)
