@@ -142,6 +142,35 @@ int salad_fused_drop_fwd(const void* q, const void* k, const void* v, void* o,
                          int32_t* d_status, void* stream);
 
 /*
+ * salad_fused_rope_fwd / salad_linear_attn_rope_fwd -- the same two calls with a rotary position
+ * embedding in the linear branch (Sec. 4.1 states that the linear branch carries a 3-D rotary embedding
+ * and gives no formula; the rotation enters the numerator only, as the rotary-embedding paper it cites
+ * defines for linear attention, so the normaliser keeps its sign):
+ *     O_l[n] = sum_j < R_n ReLU(Q_n), R_j ReLU(K_j) > V_j / ( sum_j < ReLU(Q_n), ReLU(K_j) > + eps ),
+ * R_n rotating the channel pair (2i, 2i+1) of token n:  y[2i] = c x[2i] - s x[2i+1],  y[2i+1] = s x[2i] + c x[2i+1].
+ *   d_rope  device fp16 (IEEE half) [N, d/2, 2], 16-byte aligned: (c, s) = cosine and sine of the angle of
+ *           token n and pair i; shared by every batch item and head; read-only; a 3-D embedding shares the
+ *           pairs out among the t, h, w axes of the latent grid (the caller's table decides).  Half precision
+ *           (11 significant bits for values in [-1, 1]) halves the traffic of the table, which every tile
+ *           of every head re-reads from L2; it is finer than the bf16 activations it multiplies.
+ * The rotation is applied in fp32 to the bf16 ReLU values and rounded to bf16 for the tensor cores; the
+ * state KV = sum_j (R_j ReLU(K_j))^T V_j is what kv_out receives, Z stays the plain sum.
+ * salad_fused_rope_fwd takes drop_tau like salad_fused_drop_fwd (-INFINITY: no branch is dropped).
+ * Errors as for the calls without the table; a null d_rope is SALAD_ERR_INVALID_ARG.
+ */
+int salad_fused_rope_fwd(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int N, int d, int Bq, int Bk,
+                         const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                         const float* d_static_scale, const float* d_dyn_scale, const void* d_rope,
+                         float drop_tau, float softmax_scale, float eps, void* workspace,
+                         size_t workspace_bytes, int32_t* d_status, void* stream);
+
+int salad_linear_attn_rope_fwd(const void* q, const void* k, const void* v, void* o_l,
+                               float* kv_out, float* z_out, int B, int H, int N, int d,
+                               const void* d_rope, float eps, void* workspace, size_t workspace_bytes,
+                               int32_t* d_status, void* stream);
+
+/*
  * salad_dynamic_scale -- the input- and timestep-aware scaling factor of Algorithm 1, Level 2
  * (Sec. 4.2): a D -> 1 linear layer on the modulated hidden states, a sigmoid, a token average:
  *     s[b] = (1/N) sum_n sigmoid( <x[b,n,:], w> + bias ),   s in (0, 1).

@@ -266,6 +266,7 @@ def proj_combine(o_s, o_l, w, s_b, bias=None):
 
 
 def _rope(rope, N, d):
+    # any float dtype (the GPU library takes fp16): widened exactly to fp32 for the C routine
     r = np.ascontiguousarray(rope, dtype=np.float32)
     assert r.shape == (N, d // 2, 2), "rope is [N, d/2, 2]: cosine and sine of the angle of every token and channel pair"
     return r, r.ctypes.data

@@ -64,6 +64,7 @@ struct FusedParams {
     float scale_log2;            // softmax_scale * log2(e)
     float eps;
     float drop_tau;              // linear branch of batch item b skipped when dyn_scale[b] < drop_tau
+    const __half* rope;          // [N][D] fp16: (cos, sin) per token and channel pair of the rotary linear branch, or null
     int32_t* ws_status;          // library status word (never null)
     int32_t* user_status;        // optional
 };
@@ -450,35 +451,53 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // row take two 16-byte groups of every 64 channels each.  Every Q K^T of this tile has
             // completed (its scores were consumed above), so Q is no longer read; the last P V
             // product may still be running meanwhile.
+            // Rotary variant (Sec. 4.1): the numerator takes ReLU(Q) rotated pair by pair, the denominator
+            // the un-rotated values.  A thread meets CH * 4 vectors of 8 channels; the (cos, sin) values of
+            // each (16 bytes of the table, from L2) are fetched two vectors ahead, the first before the waits.
+            constexpr int NIT = C::CH * 4;
+            const bool rotary = p.rope != nullptr;
+            auto rot_ptr = [&](int it) {
+                const int row = (it & 1) ? rb : ra;
+                const int tok = min(qb * p.Bq + row, p.N - 1);           // rows past the block or N hold zeros
+                return reinterpret_cast<const uint4*>(p.rope + size_t(tok) * D + (it >> 2) * 64 +
+                                                      (q4 + 4 * ((it >> 1) & 1)) * 8);
+            };
+            uint4 tw[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                tw[u] = make_uint4(0, 0, 0, 0);
+                if (rotary) tw[u] = __ldg(rot_ptr(u));
+            }
             ok = wait_uniform(&bars.q_full, 0);
             if (ok) ok = wait_uniform(&bars.z_full, 0);
             if (ok) {
                 float den_a = 0.f, den_b = 0.f;
 #pragma unroll
-                for (int ch = 0; ch < C::CH; ++ch) {
+                for (int it = 0; it < NIT; ++it) {
+                    const int ch = it >> 2, c16 = q4 + 4 * ((it >> 1) & 1), e2 = it & 1;
+                    const int row = e2 ? rb : ra;
+                    uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
+                                                          ((c16 ^ (row & 7)) << 4));
+                    uint4 v = *ptr;
+                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+                    const uint4 tv = tw[it & 1];
+                    if (rotary && it + 2 < NIT) tw[it & 1] = __ldg(rot_ptr(it + 2));
+                    const __half2* th = reinterpret_cast<const __half2*>(&tv);      // (cos, sin) of four pairs
+                    float den = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int c16 = q4 + 4 * j;
-#pragma unroll
-                        for (int e2 = 0; e2 < 2; ++e2) {
-                            const int row = e2 ? rb : ra;
-                            uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 +
-                                                                  ((c16 ^ (row & 7)) << 4));
-                            uint4 v = *ptr;
-                            __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
-                            float den = 0.f;
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
-                                const float2 f = __bfloat1622float2(hv[e]);
-                                const int a = ch * 64 + c16 * 8 + e * 2;
-                                den = fmaf(f.x, z_s[a], den);
-                                den = fmaf(f.y, z_s[a + 1], den);
-                            }
-                            *ptr = v;
-                            if (e2) den_b += den; else den_a += den;
+                    for (int e = 0; e < 4; ++e) {
+                        hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
+                        const float2 f = __bfloat1622float2(hv[e]);
+                        const int a = ch * 64 + c16 * 8 + e * 2;
+                        den = fmaf(f.x, z_s[a], den);
+                        den = fmaf(f.y, z_s[a + 1], den);
+                        if (rotary) {
+                            const float2 cs = __half22float2(th[e]);
+                            hv[e] = __floats2bfloat162_rn(cs.x * f.x - cs.y * f.y, cs.y * f.x + cs.x * f.y);
                         }
                     }
+                    *ptr = v;
+                    if (e2) den_b += den; else den_a += den;
                 }
                 den_a = quad_sum(den_a); den_b = quad_sum(den_b);
                 float c_scale = 1.f;

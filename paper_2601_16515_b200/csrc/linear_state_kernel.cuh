@@ -15,6 +15,12 @@
 // emits the fp32 state plus the bf16, transposed copy that the fused attention kernel
 // multiplies with ReLU(Q).
 //
+// ROPE variant (linear branch with a rotary position embedding, Sec. 4.1): the ReLU warps rotate the
+// channel pairs of ReLU(K) before the MMA reads them, with the fp16 rotation rows (cosine, sine per
+// channel pair) of the tile's tokens, which they fetch from global memory (L2: the table is shared by all
+// heads) one tile ahead into registers; Z, which takes the un-rotated values, they form in registers (a
+// thread always meets the same 8 channels of a 64-channel chunk) and sum in a fixed order.
+//
 // For d = 64 the MMA still uses M = 128: the "rows 64..127" of the MN-major A operand are
 // addressed through the leading-byte-offset, which is pointed at the V tile that follows
 // the K tile in the stage; those accumulator rows are ignored.
@@ -23,7 +29,7 @@
 
 namespace salad {
 
-template <int D, bool OVERLAP>
+template <int D, bool OVERLAP, bool ROPE = false>
 struct StateCfg {
     static constexpr int BK = 64;
     static constexpr int CH = D / 64;
@@ -43,6 +49,7 @@ struct StateParams {
     float* z_part;        // [BH][chunks][D]
     int32_t* ws_status;
     int32_t* user_status;
+    const __half* rope;       // ROPE variant: fp16 [N][D], (cosine, sine) per token and channel pair
     const float* dyn_scale;   // [B] or null: with drop_tau, batch items whose scale is below it are skipped
     float drop_tau;
     int H;
@@ -54,14 +61,14 @@ __device__ __forceinline__ bool branch_dropped(const float* dyn_scale, float tau
     return dyn_scale != nullptr && __ldg(dyn_scale + b) < tau;
 }
 
-template <int D, bool OVERLAP>
+template <int D, bool OVERLAP, bool ROPE>
 __global__ void __launch_bounds__(192)
 salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                           const StateParams p)
 {
-    using C = StateCfg<D, OVERLAP>;
+    using C = StateCfg<D, OVERLAP, ROPE>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full[C::STAGES], relu_done[C::STAGES], empty[C::STAGES], acc_done;
+    __shared__ uint64_t full[C::STAGES], relu_done[C::STAGES], empty[C::STAGES], acc_done, z_staged;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -97,6 +104,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             mbar_init(smem_u32(&empty[s]), 1);
         }
         mbar_init(smem_u32(&acc_done), 1);
+        mbar_init(smem_u32(&z_staged), 128);
         fence_mbar_init();
         prefetch_tmap(&map_k); prefetch_tmap(&map_v);
         for (int g = 0; g < min(nblk, C::STAGES); ++g) load_stage(g);
@@ -143,7 +151,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                     const uint64_t db = make_sdesc_sw128(va + k * 2048, C::T_CHUNK, 1024);
                     const uint32_t acc = (g > 0 || k > 0) ? 1u : 0u;
                     mma_ss(tmem, da, db, idesc_kv, acc);
-                    mma_ss(tmem + D, da, ones, idesc_z, acc);
+                    if (!ROPE) mma_ss(tmem + D, da, ones, idesc_z, acc);
                 }
                 tc_commit(smem_u32(&empty[s]));
             }
@@ -152,8 +160,29 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     } else {
         const int wt = tid - 64;                       // 0..127 within the ReLU/epilogue group
         bool ok = true;
+        float zacc[C::CH][8];                          // ROPE: this thread's share of Z
+#pragma unroll
+        for (int ch = 0; ch < C::CH; ++ch)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) zacc[ch][e] = 0.f;
+        // Vector i*128 + wt of a tile: 64-channel chunk i / 4, token row (i % 4) * 16 + wt / 8, 16-byte group
+        // wt % 8 of the swizzled row = channels 8 * (group ^ (row & 7)) .. + 7.  ROPE: its rotation values
+        // ((cos, sin) of four channel pairs, 16 bytes) are fetched one tile ahead.
+        constexpr int NV = C::T_BYTES / 16 / 128;
+        uint4 rot[NV], nxt[NV];
+        auto fetch_rot = [&](int g, uint4 (&dst)[NV]) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int c64 = i / 4, row = (i % 4) * 16 + (wt >> 3);
+                const int grp = (wt & 7) ^ (row & 7);
+                const int tok = min((kb0 + g) * C::BK + row, p.N - 1);      // rows past N hold zero keys
+                dst[i] = __ldg(reinterpret_cast<const uint4*>(p.rope + size_t(tok) * D + c64 * 64 + grp * 8));
+            }
+        };
+        if (ROPE && nblk > 0) fetch_rot(0, rot);
         for (int g = 0; g < nblk && ok; ++g) {
             const int s = g % C::STAGES;
+            if (ROPE && g + 1 < nblk) fetch_rot(g + 1, nxt);      // in flight while this tile is awaited and processed
             ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&full[s]), (g / C::STAGES) & 1, abortp));
             if (!ok) break;
             uint4* kt = reinterpret_cast<uint4*>(smem + s * C::STAGE_BYTES);
@@ -164,10 +193,24 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
                 hv[0] = __hmax2(hv[0], zero); hv[1] = __hmax2(hv[1], zero);
                 hv[2] = __hmax2(hv[2], zero); hv[3] = __hmax2(hv[3], zero);
+                if (ROPE) {
+                    const __half2* th = reinterpret_cast<const __half2*>(&rot[i]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 x = __bfloat1622float2(hv[e]);
+                        zacc[i / 4][2 * e] += x.x; zacc[i / 4][2 * e + 1] += x.y;
+                        const float2 cs = __half22float2(th[e]);
+                        hv[e] = __floats2bfloat162_rn(cs.x * x.x - cs.y * x.y, cs.y * x.x + cs.x * x.y);
+                    }
+                }
                 kt[i * 128 + wt] = v;
             }
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&relu_done[s]));
+            if (ROPE) {
+#pragma unroll
+                for (int i = 0; i < NV; ++i) rot[i] = nxt[i];
+            }
         }
         // accumulator -> this chunk's partial.  TMEM lane = key channel a; columns [0,D) = KV
         // row a, column D = Z[a].
@@ -191,10 +234,31 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                     }
                 }
             }
-            uint32_t zr[32];
-            if (nblk > 0) { tmem_ld32(t_row + D, zr); tmem_wait_ld(); }   // reads 32 columns, uses the first
-            if (a < D)
-                p.z_part[(size_t(bh) * p.chunks + chunk) * D + a] = nblk > 0 ? __uint_as_float(zr[0]) : 0.f;
+            if (!ROPE) {
+                uint32_t zr[32];
+                if (nblk > 0) { tmem_ld32(t_row + D, zr); tmem_wait_ld(); }   // reads 32 columns, uses the first
+                if (a < D)
+                    p.z_part[(size_t(bh) * p.chunks + chunk) * D + a] = nblk > 0 ? __uint_as_float(zr[0]) : 0.f;
+            }
+        }
+        if (ROPE && ok) {
+            // Z of this chunk: the 128 threads' register sums, staged in the (now idle) first stage and
+            // added per channel over the 16 threads that met it, in a fixed order
+            float* zs = reinterpret_cast<float*>(smem);
+#pragma unroll
+            for (int ch = 0; ch < C::CH; ++ch)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) zs[wt * (C::CH * 8) + ch * 8 + e] = zacc[ch][e];
+            mbar_arrive(smem_u32(&z_staged));
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&z_staged), 0, abortp));
+            if (ok && wt < D) {
+                const int ch = wt / 64, grp = (wt % 64) / 8, e = wt % 8;
+                float sum = 0.f;
+#pragma unroll
+                for (int r8 = 0; r8 < 16; ++r8)
+                    sum += zs[(r8 * 8 + (grp ^ (r8 & 7))) * (C::CH * 8) + ch * 8 + e];
+                p.z_part[(size_t(bh) * p.chunks + chunk) * D + wt] = sum;
+            }
         }
     }
     }

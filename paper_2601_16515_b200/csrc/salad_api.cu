@@ -96,22 +96,28 @@ int prepare_device(DeviceInfo* info) {
             e = cudaFuncSetAttribute(salad_fused_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<128, false>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128, false, false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<64, false>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64, false, false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<128, true>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128, true, false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     StateCfg<64, true>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64, true, false>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<128, false, true>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     StateCfg<64, false, true>::SMEM_BYTES);
         if (e == cudaSuccess)      // beside a CTA of the attention kernel
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<128, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+            e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_linear_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -161,6 +167,7 @@ struct Problem {
     const float *static_scale, *dyn_scale;
     float softmax_scale, eps, drop_tau;
     float *kv_out, *z_out;
+    const void* rope;             // fp16 [N, d/2, 2] cosine and sine per token and channel pair, or null
     void* ws; size_t ws_bytes; int32_t* d_status; cudaStream_t stream;
 };
 
@@ -177,6 +184,7 @@ int validate(const Problem& P) {
     }
     if (P.mode & MODE_LINEAR) {
         if (!(P.eps >= 0.f) || !isfinite(P.eps)) return SALAD_ERR_INVALID_ARG;
+        if (P.rope && !aligned16(P.rope)) return SALAD_ERR_INVALID_ARG;
     }
     if (P.mode == MODE_FUSED && (!P.static_scale || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
     const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
@@ -199,6 +207,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     if (!make_tmap_bf16_3d(&mk, P.k, D, P.N, BH, 64) || !make_tmap_bf16_3d(&mv, P.v, D, P.N, BH, 64))
         return SALAD_ERR_CUDA;
     StateParams sp;
+    sp.rope = static_cast<const __half*>(P.rope);
     sp.N = P.N; sp.nKb = nKb; sp.chunks = chunks; sp.blocks_per_chunk = bpc;
     sp.kv_part = reinterpret_cast<float*>(ws + w.off_kvp);
     sp.z_part = reinterpret_cast<float*>(ws + w.off_zp);
@@ -206,17 +215,22 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.user_status = P.d_status;
     sp.dyn_scale = P.dyn_scale; sp.drop_tau = P.drop_tau; sp.H = P.H;
     record_profile(0, P.stream);
-    // fused calls: the short-ring variant, which shares its SM with a CTA of the attention kernel
-    if (P.mode & MODE_SPARSE)
-        launch_dependent(salad_linear_state_kernel<D, true>, dim3(chunks, BH), dim3(StateCfg<D, true>::THREADS),
-                         StateCfg<D, true>::SMEM_BYTES, P.stream, mk, mv, sp);
+    // Fused calls: the short-ring variant, which shares its SM with a CTA of the attention kernel.  With a
+    // rotation table the state pass keeps the SM to itself (full ring): beside the warps of the attention
+    // kernel its ReLU warps, which then also rotate the keys, fall behind, and the call was measured slower.
+    auto launch = [&](auto kernel, int smem) {
+        launch_dependent(kernel, dim3(chunks, BH), dim3(192), size_t(smem), P.stream, mk, mv, sp);
+    };
+    if (P.rope)
+        launch(salad_linear_state_kernel<D, false, true>, StateCfg<D, false, true>::SMEM_BYTES);
+    else if (P.mode & MODE_SPARSE)
+        launch(salad_linear_state_kernel<D, true, false>, StateCfg<D, true, false>::SMEM_BYTES);
     else
-        launch_dependent(salad_linear_state_kernel<D, false>, dim3(chunks, BH), dim3(StateCfg<D, false>::THREADS),
-                         StateCfg<D, false>::SMEM_BYTES, P.stream, mk, mv, sp);
+        launch(salad_linear_state_kernel<D, false, false>, StateCfg<D, false, false>::SMEM_BYTES);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     float* z_ws = reinterpret_cast<float*>(ws + w.off_z);
     __nv_bfloat16* kvt = reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt);
-    if (P.mode & MODE_SPARSE)
+    if ((P.mode & MODE_SPARSE) && !P.rope)
         launch_dependent(salad_linear_finalize_kernel<D, 8>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
                          sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
     else
@@ -257,6 +271,7 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.scale_log2 = sc * 1.4426950408889634f;
     fp.eps = P.eps;
     fp.drop_tau = P.drop_tau;
+    fp.rope = static_cast<const __half*>(P.rope);
     fp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     fp.user_status = P.d_status;
     const int64_t grid = int64_t(fp.nQb) * BH;
@@ -318,7 +333,10 @@ int run(const Problem& P) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
         if (rc != SALAD_OK) return rc;
     }
-    if (P.mode == MODE_LINEAR) return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
+    // linear-only calls: the stand-alone apply kernel; with a rotation table the attention kernel's epilogue
+    // does the apply step (every query block has an empty kept list)
+    if (P.mode == MODE_LINEAR && !P.rope)
+        return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
     return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }
 
@@ -499,6 +517,41 @@ SALAD_EXPORT int salad_fused_fwd(const void* q, const void* k, const void* v, vo
     // no threshold: every branch is kept, whatever the value of its scale
     return salad_fused_drop_fwd(q, k, v, o, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, d_static_scale, d_dyn_scale,
                                 -INFINITY, softmax_scale, eps, workspace, workspace_bytes, d_status, stream);
+}
+
+SALAD_EXPORT int salad_fused_rope_fwd(const void* q, const void* k, const void* v, void* o,
+                                      int B, int H, int N, int d, int Bq, int Bk,
+                                      const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                      const float* d_static_scale, const float* d_dyn_scale, const void* d_rope,
+                                      float drop_tau, float softmax_scale, float eps, void* workspace,
+                                      size_t workspace_bytes, int32_t* d_status, void* stream) {
+    if (isnan(drop_tau) || !d_rope) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
+    P.rope = d_rope;
+    P.softmax_scale = softmax_scale; P.eps = eps;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_linear_attn_rope_fwd(const void* q, const void* k, const void* v, void* o_l,
+                                            float* kv_out, float* z_out, int B, int H, int N, int d,
+                                            const void* d_rope, float eps, void* workspace,
+                                            size_t workspace_bytes, int32_t* d_status, void* stream) {
+    if (!d_rope) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.drop_tau = -INFINITY;
+    P.q = q; P.k = k; P.v = v; P.o = o_l;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
+    P.rope = d_rope;
+    P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
 }
 
 SALAD_EXPORT int salad_dynamic_scale(const void* x, const float* w, float bias, int B, int N, int D,

@@ -28,7 +28,7 @@ EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
            "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
-           "salad_selftest_bounded_wait")
+           "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd")
 
 
 class SaladError(RuntimeError):
@@ -72,6 +72,10 @@ def _load() -> ctypes.CDLL:
     lib.salad_proj_combine_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [p, p]
     lib.salad_selftest_bounded_wait.restype = i32
     lib.salad_selftest_bounded_wait.argtypes = [p, p, p]
+    lib.salad_fused_rope_fwd.restype = i32
+    lib.salad_fused_rope_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, p, f32, f32, f32, p, sz, p, p]
+    lib.salad_linear_attn_rope_fwd.restype = i32
+    lib.salad_linear_attn_rope_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [p, f32, p, sz, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -190,6 +194,51 @@ def salad_linear_attn_fwd(q, k, v, eps: float = 1e-6, out=None, kv_out=None, z_o
         _check(_lib.salad_linear_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_out), _ptr(z_out),
                                           B, H, N, d, float(eps), _ptr(workspace), workspace.numel(),
                                           _ptr(status), _stream(stream)), "salad_linear_attn_fwd")
+    return out
+
+
+def _rope_table(rope, N, d):
+    if (rope.dtype != torch.float16 or not rope.is_cuda or not rope.is_contiguous()
+            or tuple(rope.shape) != (N, d // 2, 2)):
+        raise ValueError(f"rope must be a contiguous CUDA fp16 tensor of shape [{N}, {d // 2}, 2] (cosine, sine)")
+    return rope
+
+
+def salad_linear_attn_rope_fwd(q, k, v, rope, eps: float = 1e-6, out=None, kv_out=None, z_out=None,
+                               workspace=None, status=None, stream=None):
+    """ReLU linear attention with a rotary position embedding in the numerator.  `rope` is the fp16
+    table [N, d/2, 2] of cosines and sines per token and channel pair."""
+    B, H, N, d, workspace = _common(q, k, v, 128, 64, workspace)
+    _rope_table(rope, N, d)
+    if out is None:
+        out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_linear_attn_rope_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kv_out), _ptr(z_out),
+                                               B, H, N, d, _ptr(rope), float(eps), _ptr(workspace),
+                                               workspace.numel(), _ptr(status), _stream(stream)),
+               "salad_linear_attn_rope_fwd")
+    return out
+
+
+def salad_fused_rope_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_scale, rope, Bq: int = 128,
+                         Bk: int = 64, softmax_scale: float = 0.0, eps: float = 1e-6, out=None,
+                         workspace=None, status=None, stream=None, drop_tau: Optional[float] = None):
+    """salad_fused_fwd with the rotary linear branch (and, with `drop_tau`, branch dropping)."""
+    B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    _rope_table(rope, N, d)
+    for name, t, n in (("static_scale", static_scale, H), ("dyn_scale", dyn_scale, B)):
+        if t.dtype != torch.float32 or not t.is_cuda or t.numel() != n or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor with {n} elements")
+    if out is None:
+        out = torch.empty_like(q)
+    tau = float("-inf") if drop_tau is None else float(drop_tau)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_fused_rope_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                         _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale),
+                                         _ptr(rope), tau, float(softmax_scale), float(eps), _ptr(workspace),
+                                         workspace.numel(), _ptr(status), _stream(stream)),
+               "salad_fused_rope_fwd")
     return out
 
 

@@ -123,7 +123,8 @@ def make_scales(wl: Workload):
 
 def rope_table(grid, d: int, base: float = 10000.0) -> np.ndarray:
     """Rotation table of a 3-D rotary position embedding, an INPUT of the rotary linear branch:
-    float32 [N, d/2, 2] holding the cosine and sine of the angle of every token and channel pair.
+    float16 [N, d/2, 2] (the dtype of the library's table argument; the oracle widens the same values)
+    holding the cosine and sine of the angle of every token and channel pair.
     The d/2 channel pairs are shared out among the t, h and w axes of the latent grid (the last two
     get floor(d/6) pairs each, t the rest, as video DiTs of the Wan family do); pair j of an axis with
     P pairs turns by position * base**(-j / P) for a token at that position along the axis.  Tokens are
@@ -138,7 +139,7 @@ def rope_table(grid, d: int, base: float = 10000.0) -> np.ndarray:
         freq = base ** (-np.arange(P, dtype=np.float64) / max(P, 1))
         parts.append(pos.reshape(-1, 1).astype(np.float64) * freq[None, :])
     ang = np.concatenate(parts, axis=1)                      # [N, d/2]
-    return np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)
+    return np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float16)
 
 
 def irregular_csr(wl: Workload, lo_frac: float = 0.05, hi_frac: float = 0.15):

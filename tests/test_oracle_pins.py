@@ -633,18 +633,20 @@ def test_rope_fused_pins():
 
 def test_rope_table_generator():
     grid, d = (3, 4, 5), 32
-    r = wlmod.rope_table(grid, d).astype(np.float64)
+    r = wlmod.rope_table(grid, d)
+    assert r.dtype == np.float16                  # the library's table dtype; 2^-11 relative rounding
+    r = r.astype(np.float64)
     N = 3 * 4 * 5
     assert r.shape == (N, d // 2, 2)
-    np.testing.assert_allclose((r ** 2).sum(-1), 1.0, atol=1e-6)
+    np.testing.assert_allclose((r ** 2).sum(-1), 1.0, atol=2e-3)
     np.testing.assert_allclose(r[0, :, 0], 1.0); np.testing.assert_allclose(r[0, :, 1], 0.0)   # origin: no rotation
     p_hw = (d // 2) // 3; p_t = d // 2 - 2 * p_hw
     n = lambda t, h, w: (t * 4 + h) * 5 + w
     # a step along w changes only the w pairs, by the pair's frequency
     np.testing.assert_allclose(r[n(1, 2, 3), :p_t + p_hw], r[n(1, 2, 4), :p_t + p_hw])
     ang = np.arctan2(r[n(0, 0, 1), p_t + p_hw:, 1], r[n(0, 0, 1), p_t + p_hw:, 0])
-    np.testing.assert_allclose(ang, 10000.0 ** (-np.arange(p_hw) / p_hw), rtol=1e-5)
+    np.testing.assert_allclose(ang, 10000.0 ** (-np.arange(p_hw) / p_hw), rtol=2e-2, atol=1e-3)
     # along t only the first p_t pairs change
     np.testing.assert_allclose(r[n(0, 2, 3), p_t:], r[n(2, 2, 3), p_t:])
     ang_t = np.arctan2(r[n(1, 0, 0), :p_t, 1], r[n(1, 0, 0), :p_t, 0])
-    np.testing.assert_allclose(ang_t, 10000.0 ** (-np.arange(p_t) / p_t), rtol=1e-5)
+    np.testing.assert_allclose(ang_t, 10000.0 ** (-np.arange(p_t) / p_t), rtol=2e-2, atol=1e-3)
