@@ -461,7 +461,7 @@ def main():
                          "unit": "TFLOP/s", "frac": achieved / peak, "peak_source": peaks["source"] + " (burst)",
                          # DRAM bytes of one launch from the ncu capture of this workload
                          # (profiles/salad_fused_kernel_wan1.3b-90.md); algorithmic bytes are 402.6 MB
-                         "traffic": 393.4e6 if wl.name == "wan1.3b-90" else None,
+                         "traffic": 393.7e6 if wl.name == "wan1.3b-90" else None,
                          "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, see profiles/",
                          "kernel_ms": attn_ms, "state_kernels_ms": state_ms,
                          "timed_how": "CUDA events around the launch, %d steps directly before the timed region" % KP},
