@@ -39,7 +39,8 @@ struct StateCfg {
     static constexpr int STAGES = OVERLAP ? 3 : ((D == 128) ? 6 : 8);
     static constexpr int OFF_ONES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = OFF_ONES + 2048 + 1024;
-    static constexpr int THREADS = 192;
+    static constexpr int RELU_THREADS = ROPE ? 256 : 128;   // the rotation doubles the work per element
+    static constexpr int THREADS = 64 + RELU_THREADS;
     static constexpr int TMEM_COLS = 256;
 };
 
@@ -62,7 +63,7 @@ __device__ __forceinline__ bool branch_dropped(const float* dyn_scale, float tau
 }
 
 template <int D, bool OVERLAP, bool ROPE>
-__global__ void __launch_bounds__(192)
+__global__ void __launch_bounds__(64 + (ROPE ? 256 : 128))
 salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                           const StateParams p)
 {
@@ -100,11 +101,11 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&relu_done[s]), 128);
+            mbar_init(smem_u32(&relu_done[s]), C::RELU_THREADS);
             mbar_init(smem_u32(&empty[s]), 1);
         }
         mbar_init(smem_u32(&acc_done), 1);
-        mbar_init(smem_u32(&z_staged), 128);
+        mbar_init(smem_u32(&z_staged), C::RELU_THREADS);
         fence_mbar_init();
         prefetch_tmap(&map_k); prefetch_tmap(&map_v);
         for (int g = 0; g < min(nblk, C::STAGES); ++g) load_stage(g);
@@ -158,22 +159,23 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             if (ok) tc_commit(smem_u32(&acc_done));
         }
     } else {
-        const int wt = tid - 64;                       // 0..127 within the ReLU/epilogue group
+        constexpr int RW = C::RELU_THREADS;
+        const int wt = tid - 64;                       // 0..RW-1 within the ReLU/epilogue group
         bool ok = true;
         float zacc[C::CH][8];                          // ROPE: this thread's share of Z
 #pragma unroll
         for (int ch = 0; ch < C::CH; ++ch)
 #pragma unroll
             for (int e = 0; e < 8; ++e) zacc[ch][e] = 0.f;
-        // Vector i*128 + wt of a tile: 64-channel chunk i / 4, token row (i % 4) * 16 + wt / 8, 16-byte group
-        // wt % 8 of the swizzled row = channels 8 * (group ^ (row & 7)) .. + 7.  ROPE: its rotation values
+        // Vector i*RW + wt of a tile (512 vectors per 64-channel chunk): chunk i*RW / 512, token row
+        // (i*RW % 512) / 8 + wt / 8, 16-byte group wt % 8 of the swizzled row = channels 8 * (group ^ (row & 7)) .. + 7.  ROPE: its rotation values
         // ((cos, sin) of four channel pairs, 16 bytes) are fetched one tile ahead.
-        constexpr int NV = C::T_BYTES / 16 / 128;
+        constexpr int NV = C::T_BYTES / 16 / RW;
         uint4 rot[NV], nxt[NV];
         auto fetch_rot = [&](int g, uint4 (&dst)[NV]) {
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
-                const int c64 = i / 4, row = (i % 4) * 16 + (wt >> 3);
+                const int c64 = (i * RW) / 512, row = ((i * RW) % 512) / 8 + (wt >> 3);
                 const int grp = (wt & 7) ^ (row & 7);
                 const int tok = min((kb0 + g) * C::BK + row, p.N - 1);      // rows past N hold zero keys
                 dst[i] = __ldg(reinterpret_cast<const uint4*>(p.rope + size_t(tok) * D + c64 * 64 + grp * 8));
@@ -188,8 +190,8 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             uint4* kt = reinterpret_cast<uint4*>(smem + s * C::STAGE_BYTES);
             const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
 #pragma unroll
-            for (int i = 0; i < C::T_BYTES / 16 / 128; ++i) {
-                uint4 v = kt[i * 128 + wt];
+            for (int i = 0; i < NV; ++i) {
+                uint4 v = kt[i * RW + wt];
                 __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
                 hv[0] = __hmax2(hv[0], zero); hv[1] = __hmax2(hv[1], zero);
                 hv[2] = __hmax2(hv[2], zero); hv[3] = __hmax2(hv[3], zero);
@@ -198,12 +200,12 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 x = __bfloat1622float2(hv[e]);
-                        zacc[i / 4][2 * e] += x.x; zacc[i / 4][2 * e + 1] += x.y;
+                        zacc[(i * RW) / 512][2 * e] += x.x; zacc[(i * RW) / 512][2 * e + 1] += x.y;
                         const float2 cs = __half22float2(th[e]);
                         hv[e] = __floats2bfloat162_rn(cs.x * x.x - cs.y * x.y, cs.y * x.x + cs.x * x.y);
                     }
                 }
-                kt[i * 128 + wt] = v;
+                kt[i * RW + wt] = v;
             }
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&relu_done[s]));
@@ -220,8 +222,11 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             const int a = (warp & 3) * 32 + lane;       // lanes this warp may access
             const uint32_t t_row = tmem + (uint32_t((warp & 3) * 32) << 16);
             float* kv_row = p.kv_part + ((size_t(bh) * p.chunks + chunk) * D + a) * D;
+            // (ROPE: eight warps, two per group of 32 lanes: each takes half of the columns)
+            constexpr int NCC = (D / 32) / (RW / 128);
+            const int cc0 = ((warp - 2) / 4) * NCC;
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
+            for (int cc = cc0; cc < cc0 + NCC; ++cc) {
                 uint32_t r[32];
                 if (nblk > 0) { tmem_ld32(t_row + cc * 32, r); tmem_wait_ld(); }
                 if (a < D) {
@@ -242,8 +247,8 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             }
         }
         if (ROPE && ok) {
-            // Z of this chunk: the 128 threads' register sums, staged in the (now idle) first stage and
-            // added per channel over the 16 threads that met it, in a fixed order
+            // Z of this chunk: the threads' register sums, staged in the (now idle) first stage and added
+            // per channel over the RW / 8 threads that met it, in a fixed order
             float* zs = reinterpret_cast<float*>(smem);
 #pragma unroll
             for (int ch = 0; ch < C::CH; ++ch)
@@ -255,7 +260,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 const int ch = wt / 64, grp = (wt % 64) / 8, e = wt % 8;
                 float sum = 0.f;
 #pragma unroll
-                for (int r8 = 0; r8 < 16; ++r8)
+                for (int r8 = 0; r8 < RW / 8; ++r8)
                     sum += zs[(r8 * 8 + (grp ^ (r8 & 7))) * (C::CH * 8) + ch * 8 + e];
                 p.z_part[(size_t(bh) * p.chunks + chunk) * D + wt] = sum;
             }

@@ -216,17 +216,20 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     sp.dyn_scale = P.dyn_scale; sp.drop_tau = P.drop_tau; sp.H = P.H;
     record_profile(0, P.stream);
     // Fused calls: the short-ring variant, which shares its SM with a CTA of the attention kernel.  With a
-    // rotation table the state pass keeps the SM to itself (full ring): beside the warps of the attention
-    // kernel its ReLU warps, which then also rotate the keys, fall behind, and the call was measured slower.
-    auto launch = [&](auto kernel, int smem) {
-        launch_dependent(kernel, dim3(chunks, BH), dim3(192), size_t(smem), P.stream, mk, mv, sp);
+    // rotation table the state pass keeps the SM to itself (full ring, eight ReLU warps): sharing the SM with
+    // the attention kernel was measured no faster.
+    auto launch = [&](auto kernel, int threads, int smem) {
+        launch_dependent(kernel, dim3(chunks, BH), dim3(threads), size_t(smem), P.stream, mk, mv, sp);
     };
     if (P.rope)
-        launch(salad_linear_state_kernel<D, false, true>, StateCfg<D, false, true>::SMEM_BYTES);
+        launch(salad_linear_state_kernel<D, false, true>, StateCfg<D, false, true>::THREADS,
+               StateCfg<D, false, true>::SMEM_BYTES);
     else if (P.mode & MODE_SPARSE)
-        launch(salad_linear_state_kernel<D, true, false>, StateCfg<D, true, false>::SMEM_BYTES);
+        launch(salad_linear_state_kernel<D, true, false>, StateCfg<D, true, false>::THREADS,
+               StateCfg<D, true, false>::SMEM_BYTES);
     else
-        launch(salad_linear_state_kernel<D, false, false>, StateCfg<D, false, false>::SMEM_BYTES);
+        launch(salad_linear_state_kernel<D, false, false>, StateCfg<D, false, false>::THREADS,
+               StateCfg<D, false, false>::SMEM_BYTES);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     float* z_ws = reinterpret_cast<float*>(ws + w.off_z);
     __nv_bfloat16* kvt = reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt);

@@ -129,3 +129,50 @@ def test_rope_argument_checks(salad):
         salad.salad_linear_attn_rope_fwd(q, k, v, good.float())
     with pytest.raises(ValueError):
         salad.salad_linear_attn_rope_fwd(q, k, v, good.cpu())
+
+
+def test_fused_rope_drops_per_batch_item(salad):
+    # two batch items, one scale below the threshold: its linear branch is skipped on the device
+    B, H, N, d, Bq = 2, 2, 1100, 128, 128
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), Bq, 64, (), 1)
+    q, k, v = rand_qkv(B, H, N, d, 4242)
+    rope = random_table(N, d, 8)
+    rp, ci = random_csr(wl.nQb, wl.nKb, 31, lo=1, hi=6)
+    lam = np.array([0.9, 0.4], np.float32); s = np.array([0.2, 0.8], np.float32)
+    rp_d, ci_d = dev_csr(rp, ci)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_rope_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, torch.from_numpy(lam).cuda(),
+                                     torch.from_numpy(s).cuda(), torch.from_numpy(rope).cuda(), Bq=Bq, status=status,
+                                     drop_tau=0.5)
+    status_ok(status)
+    ref = orc.salad_fused_rope(f32(q), f32(k), f32(v), rope, Bq, 64, rp, ci, 1, lam, s, tau=0.5)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "fused rope drop")
+    sparse = salad.salad_sparse_attn_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, 1, Bq=Bq)
+    assert torch.equal(out[0], sparse[0]) and not torch.equal(out[1], sparse[1])
+
+
+def test_fused_rope_call_in_a_cuda_graph_and_repeatable(salad):
+    B, H, N, d = 1, 4, 2048, 128
+    q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 911))
+    rope = torch.from_numpy(wlmod.rope_table((4, 16, 32), d)).cuda()
+    rp, ci = salad.salad_mask_build(4, 16, 32, 128, 64, [(1, 3, 8)])
+    lam = torch.rand(H, device="cuda"); s = torch.rand(B, device="cuda")
+    ws = salad.alloc_workspace(B, H, N, d)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    eager = salad.salad_fused_rope_fwd(q, k, v, rp, ci, 1, lam, s, rope, workspace=ws, status=status)
+    again = salad.salad_fused_rope_fwd(q, k, v, rp, ci, 1, lam, s, rope, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    assert torch.equal(eager, again)             # fixed summation orders: bit-identical from call to call
+    out = torch.zeros_like(q)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            salad.salad_fused_rope_fwd(q, k, v, rp, ci, 1, lam, s, rope, out=out, workspace=ws, status=status,
+                                       stream=side)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(out, eager)
