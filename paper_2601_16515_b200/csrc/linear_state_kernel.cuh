@@ -17,9 +17,10 @@
 //
 // ROPE variant (linear branch with a rotary position embedding, Sec. 4.1): the ReLU warps rotate the
 // channel pairs of ReLU(K) before the MMA reads them, with the fp16 rotation rows (cosine, sine per
-// channel pair) of the tile's tokens, which they fetch from global memory (L2: the table is shared by all
-// heads) one tile ahead into registers; Z, which takes the un-rotated values, they form in registers (a
-// thread always meets the same 8 channels of a 64-channel chunk) and sum in a fixed order.
+// channel pair) of the tile's tokens, which ride in the stage behind K and V (a third TMA load; fetching
+// them from L2 with plain loads one tile ahead left the L2 latency exposed on every tile); Z, which takes
+// the un-rotated values, they form in registers (a thread always meets the same 8 channels of a 64-channel
+// chunk) and sum in a fixed order.  The rotation doubles the work per element: eight ReLU warps.
 //
 // For d = 64 the MMA still uses M = 128: the "rows 64..127" of the MN-major A operand are
 // addressed through the leading-byte-offset, which is pointed at the V tile that follows
@@ -35,8 +36,9 @@ struct StateCfg {
     static constexpr int CH = D / 64;
     static constexpr int T_CHUNK = BK * 128;           // bytes of one 64-column chunk of a tile
     static constexpr int T_BYTES = CH * T_CHUNK;       // one K or V tile
-    static constexpr int STAGE_BYTES = 2 * T_BYTES;    // K then V
-    static constexpr int STAGES = OVERLAP ? 3 : ((D == 128) ? 6 : 8);
+    static constexpr int R_BYTES = ROPE ? BK * D * 2 : 0;          // fp16 rotation rows of the tile's tokens
+    static constexpr int STAGE_BYTES = 2 * T_BYTES + R_BYTES;      // K, V, then the rotation rows
+    static constexpr int STAGES = ROPE ? ((D == 128) ? 4 : 8) : (OVERLAP ? 3 : ((D == 128) ? 6 : 8));
     static constexpr int OFF_ONES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = OFF_ONES + 2048 + 1024;
     static constexpr int RELU_THREADS = ROPE ? 256 : 128;   // the rotation doubles the work per element
@@ -50,7 +52,6 @@ struct StateParams {
     float* z_part;        // [BH][chunks][D]
     int32_t* ws_status;
     int32_t* user_status;
-    const __half* rope;       // ROPE variant: fp16 [N][D], (cosine, sine) per token and channel pair
     const float* dyn_scale;   // [B] or null: with drop_tau, batch items whose scale is below it are skipped
     float drop_tau;
     int H;
@@ -65,7 +66,7 @@ __device__ __forceinline__ bool branch_dropped(const float* dyn_scale, float tau
 template <int D, bool OVERLAP, bool ROPE>
 __global__ void __launch_bounds__(64 + (ROPE ? 256 : 128))
 salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                          const StateParams p)
+                          const __grid_constant__ CUtensorMap map_r, const StateParams p)
 {
     using C = StateCfg<D, OVERLAP, ROPE>;
     extern __shared__ uint8_t smem_raw[];
@@ -97,6 +98,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             tma_load_3d(dst + ch * C::T_CHUNK, &map_k, bar, ch * 64, (kb0 + g) * C::BK, bh);
             tma_load_3d(dst + C::T_BYTES + ch * C::T_CHUNK, &map_v, bar, ch * 64, (kb0 + g) * C::BK, bh);
         }
+        if (ROPE) tma_load_3d(dst + 2 * C::T_BYTES, &map_r, bar, 0, (kb0 + g) * C::BK, 0);   // [BK tokens][D halves]
     };
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -108,6 +110,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         mbar_init(smem_u32(&z_staged), C::RELU_THREADS);
         fence_mbar_init();
         prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+        if (ROPE) prefetch_tmap(&map_r);
         for (int g = 0; g < min(nblk, C::STAGES); ++g) load_stage(g);
     }
     // all-ones bf16 tile (0x3F80 = 1.0)
@@ -168,23 +171,12 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 #pragma unroll
             for (int e = 0; e < 8; ++e) zacc[ch][e] = 0.f;
         // Vector i*RW + wt of a tile (512 vectors per 64-channel chunk): chunk i*RW / 512, token row
-        // (i*RW % 512) / 8 + wt / 8, 16-byte group wt % 8 of the swizzled row = channels 8 * (group ^ (row & 7)) .. + 7.  ROPE: its rotation values
-        // ((cos, sin) of four channel pairs, 16 bytes) are fetched one tile ahead.
+        // (i*RW % 512) / 8 + wt / 8, 16-byte group wt % 8 of the swizzled row = channels 8 * (group ^ (row & 7))
+        // .. + 7.  ROPE: its rotation values ((cos, sin) of four channel pairs) are 16 bytes of the stage's
+        // rotation rows.
         constexpr int NV = C::T_BYTES / 16 / RW;
-        uint4 rot[NV], nxt[NV];
-        auto fetch_rot = [&](int g, uint4 (&dst)[NV]) {
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const int c64 = (i * RW) / 512, row = ((i * RW) % 512) / 8 + (wt >> 3);
-                const int grp = (wt & 7) ^ (row & 7);
-                const int tok = min((kb0 + g) * C::BK + row, p.N - 1);      // rows past N hold zero keys
-                dst[i] = __ldg(reinterpret_cast<const uint4*>(p.rope + size_t(tok) * D + c64 * 64 + grp * 8));
-            }
-        };
-        if (ROPE && nblk > 0) fetch_rot(0, rot);
         for (int g = 0; g < nblk && ok; ++g) {
             const int s = g % C::STAGES;
-            if (ROPE && g + 1 < nblk) fetch_rot(g + 1, nxt);      // in flight while this tile is awaited and processed
             ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&full[s]), (g / C::STAGES) & 1, abortp));
             if (!ok) break;
             uint4* kt = reinterpret_cast<uint4*>(smem + s * C::STAGE_BYTES);
@@ -196,7 +188,11 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 hv[0] = __hmax2(hv[0], zero); hv[1] = __hmax2(hv[1], zero);
                 hv[2] = __hmax2(hv[2], zero); hv[3] = __hmax2(hv[3], zero);
                 if (ROPE) {
-                    const __half2* th = reinterpret_cast<const __half2*>(&rot[i]);
+                    const int row = ((i * RW) % 512) / 8 + (wt >> 3);
+                    const int grp = (wt & 7) ^ (row & 7);
+                    const uint4 tv = *reinterpret_cast<const uint4*>(
+                        smem + s * C::STAGE_BYTES + 2 * C::T_BYTES + (row * D + ((i * RW) / 512) * 64 + grp * 8) * 2);
+                    const __half2* th = reinterpret_cast<const __half2*>(&tv);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 x = __bfloat1622float2(hv[e]);
@@ -209,10 +205,6 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             }
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&relu_done[s]));
-            if (ROPE) {
-#pragma unroll
-                for (int i = 0; i < NV; ++i) rot[i] = nxt[i];
-            }
         }
         // accumulator -> this chunk's partial.  TMEM lane = key channel a; columns [0,D) = KV
         // row a, column D = Z[a].

@@ -206,8 +206,9 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     CUtensorMap mk, mv;
     if (!make_tmap_bf16_3d(&mk, P.k, D, P.N, BH, 64) || !make_tmap_bf16_3d(&mv, P.v, D, P.N, BH, 64))
         return SALAD_ERR_CUDA;
+    CUtensorMap mr = mk;          // unused without a rotation table
+    if (P.rope && !make_tmap_f16_rows(&mr, P.rope, D, P.N, 64)) return SALAD_ERR_CUDA;
     StateParams sp;
-    sp.rope = static_cast<const __half*>(P.rope);
     sp.N = P.N; sp.nKb = nKb; sp.chunks = chunks; sp.blocks_per_chunk = bpc;
     sp.kv_part = reinterpret_cast<float*>(ws + w.off_kvp);
     sp.z_part = reinterpret_cast<float*>(ws + w.off_zp);
@@ -219,7 +220,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     // rotation table the state pass keeps the SM to itself (full ring, eight ReLU warps): sharing the SM with
     // the attention kernel was measured no faster.
     auto launch = [&](auto kernel, int threads, int smem) {
-        launch_dependent(kernel, dim3(chunks, BH), dim3(threads), size_t(smem), P.stream, mk, mv, sp);
+        launch_dependent(kernel, dim3(chunks, BH), dim3(threads), size_t(smem), P.stream, mk, mv, mr, sp);
     };
     if (P.rope)
         launch(salad_linear_state_kernel<D, false, true>, StateCfg<D, false, true>::THREADS,

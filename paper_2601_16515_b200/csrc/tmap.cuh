@@ -43,4 +43,20 @@ inline bool make_tmap_bf16_3d(CUtensorMap* out, const void* base, int d, int64_t
     return r == CUDA_SUCCESS;
 }
 
+// Map over an fp16 matrix [rows, cols] (cols fastest, contiguous; cols <= 256).  One box is
+// [box_rows, cols], written to shared memory row after row without swizzle.  Rows past `rows`
+// read as zero.
+inline bool make_tmap_f16_rows(CUtensorMap* out, const void* base, int cols, int64_t rows, int box_rows) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), 1};
+    cuuint64_t strides[2] = {cuuint64_t(cols) * 2, cuuint64_t(cols) * 2 * cuuint64_t(rows)};
+    cuuint32_t box[3] = {cuuint32_t(cols), cuuint32_t(box_rows), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 }  // namespace salad
