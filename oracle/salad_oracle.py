@@ -319,3 +319,30 @@ def salad_fused_rope(q, k, v, rope, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b,
     lib.oracle_salad_fused_rope(qp, kp, vp, rop, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
                                 sb.ctypes.data, float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
     return o
+
+
+def rope3d_table(grid, d, base=10000.0, tokens=None):
+    """Rotation table of a 3-D rotary position embedding for the tokens of a T x Hs x Ws latent grid
+    (Sec. 4.1 says "3D"; the paper gives no layout, this one follows video DiTs of the Wan family):
+    the d/2 channel pairs are shared out among the axes, floor(d/6) pairs each for h and w (in that order,
+    after the t pairs) and the rest for t; pair j of an axis with P pairs turns by
+        angle = position * base**(-j / P)
+    for a token at that position along the axis; tokens are numbered with time slowest,
+    n = (t*Hs + h)*Ws + w.  Angles, cosines and sines in float64, rounded once to float16 (the dtype of
+    the GPU library's table).  Returns float16 [N, d/2, 2] = (cos, sin), or the rows of `tokens` only."""
+    T, Hs, Ws = grid
+    pairs = d // 2
+    p_hw = pairs // 3
+    p_t = pairs - 2 * p_hw
+    tokens = range(T * Hs * Ws) if tokens is None else [int(n) for n in tokens]
+    table = np.empty((len(tokens), pairs, 2), dtype=np.float16)
+    for row, n in enumerate(tokens):
+        pos = (n // (Hs * Ws), (n // Ws) % Hs, n % Ws)
+        i = 0
+        for axis, P in enumerate((p_t, p_hw, p_hw)):
+            for j in range(P):
+                angle = float(pos[axis]) * float(base) ** (-float(j) / P)
+                table[row, i, 0] = np.float16(np.cos(angle))
+                table[row, i, 1] = np.float16(np.sin(angle))
+                i += 1
+    return table

@@ -122,7 +122,9 @@ def make_scales(wl: Workload):
 
 
 def rope_table(grid, d: int, base: float = 10000.0) -> np.ndarray:
-    """Rotation table of a 3-D rotary position embedding, an INPUT of the rotary linear branch:
+    """Rotation table of a 3-D rotary position embedding, an INPUT of the rotary linear branch (the
+    vectorised twin of the oracle's token-by-token definition, bit-identical to it, so that full-size
+    tables need no minutes of Python loops; the library's own producer is checked against the oracle):
     float16 [N, d/2, 2] (the dtype of the library's table argument; the oracle widens the same values)
     holding the cosine and sine of the angle of every token and channel pair.
     The d/2 channel pairs are shared out among the t, h and w axes of the latent grid (the last two

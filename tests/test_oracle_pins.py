@@ -631,22 +631,36 @@ def test_rope_fused_pins():
     np.testing.assert_allclose(dropped, o_s, rtol=0, atol=0)
 
 
-def test_rope_table_generator():
+def test_rope3d_table_pins():
     grid, d = (3, 4, 5), 32
-    r = wlmod.rope_table(grid, d)
-    assert r.dtype == np.float16                  # the library's table dtype; 2^-11 relative rounding
-    r = r.astype(np.float64)
+    r16 = orc.rope3d_table(grid, d)
+    assert r16.dtype == np.float16                # the library's table dtype; 2^-11 relative rounding
+    r = r16.astype(np.float64)
     N = 3 * 4 * 5
     assert r.shape == (N, d // 2, 2)
     np.testing.assert_allclose((r ** 2).sum(-1), 1.0, atol=2e-3)
     np.testing.assert_allclose(r[0, :, 0], 1.0); np.testing.assert_allclose(r[0, :, 1], 0.0)   # origin: no rotation
     p_hw = (d // 2) // 3; p_t = d // 2 - 2 * p_hw
+    assert (p_t, p_hw) == (6, 5)
     n = lambda t, h, w: (t * 4 + h) * 5 + w
     # a step along w changes only the w pairs, by the pair's frequency
     np.testing.assert_allclose(r[n(1, 2, 3), :p_t + p_hw], r[n(1, 2, 4), :p_t + p_hw])
     ang = np.arctan2(r[n(0, 0, 1), p_t + p_hw:, 1], r[n(0, 0, 1), p_t + p_hw:, 0])
     np.testing.assert_allclose(ang, 10000.0 ** (-np.arange(p_hw) / p_hw), rtol=2e-2, atol=1e-3)
-    # along t only the first p_t pairs change
+    # along h only the middle pairs, along t only the first p_t pairs
+    np.testing.assert_allclose(r[n(1, 0, 3), :p_t], r[n(1, 3, 3), :p_t])
+    np.testing.assert_allclose(r[n(1, 0, 3), p_t + p_hw:], r[n(1, 3, 3), p_t + p_hw:])
     np.testing.assert_allclose(r[n(0, 2, 3), p_t:], r[n(2, 2, 3), p_t:])
     ang_t = np.arctan2(r[n(1, 0, 0), :p_t, 1], r[n(1, 0, 0), :p_t, 0])
     np.testing.assert_allclose(ang_t, 10000.0 ** (-np.arange(p_t) / p_t), rtol=2e-2, atol=1e-3)
+    # the first pair of every axis turns by one radian per position (frequency base**0 = 1)
+    np.testing.assert_allclose(r[n(2, 3, 4), [0, p_t, p_t + p_hw], 0], np.cos([2.0, 3.0, 4.0]), atol=5e-4)
+    np.testing.assert_allclose(r[n(2, 3, 4), [0, p_t, p_t + p_hw], 1], np.sin([2.0, 3.0, 4.0]), atol=5e-4)
+    # rows on request, and the vectorised input generator the tests feed to both sides is the same table
+    sel = [0, 7, 33, N - 1]
+    assert np.array_equal(orc.rope3d_table(grid, d, tokens=sel).view(np.uint16), r16[sel].view(np.uint16))
+    assert np.array_equal(wlmod.rope_table(grid, d).view(np.uint16), r16.view(np.uint16))
+    big = wlmod.C2.grid
+    tok = np.random.default_rng(3).integers(0, wlmod.C2.N, size=200)
+    assert np.array_equal(wlmod.rope_table(big, 128)[tok].view(np.uint16),
+                          orc.rope3d_table(big, 128, tokens=tok).view(np.uint16))
