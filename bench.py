@@ -429,7 +429,7 @@ def main():
 
         # rotary variant of the linear branch (Sec. 4.1): the same fused call with the 3-D rotation table of
         # the workload's latent grid (fp16, 8.4 MB at this shape, shared by all heads)
-        rope_d = torch.from_numpy(wlmod.rope_table(wl.grid, wl.d)).to(dev)
+        rope_d = salad.salad_rope3d_table_build(*wl.grid, wl.d, device=dev)
         rope_ms = timed(lambda: salad.salad_fused_rope_fwd(q, k, v, rp, ci, Hm, lam_d, s_d, rope_d, Bq=wl.Bq, Bk=wl.Bk,
                                                            out=out, workspace=ws), 20)
         extras["rope_linear_branch"] = {"fused_ms": rope_ms, "fused_tflops": flops / (rope_ms * 1e-3) / 1e12,

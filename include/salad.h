@@ -171,6 +171,20 @@ int salad_linear_attn_rope_fwd(const void* q, const void* k, const void* v, void
                                int32_t* d_status, void* stream);
 
 /*
+ * salad_rope3d_table_build -- the rotation table of a 3-D rotary position embedding for the tokens of a
+ * T x Hs x Ws latent grid, n = (t*Hs + h)*Ws + w (Sec. 4.1 says the embedding is 3-D and gives no layout;
+ * this one follows video DiTs of the Wan family).  The d/2 channel pairs are shared out among the axes:
+ * floor(d/6) pairs each for h and w (in that order, after the t pairs), the rest for t; pair j of an axis
+ * with P pairs turns by  position * base^(-j / P).
+ *   d_rope  out, device fp16 [T*Hs*Ws, d/2, 2] = (cos, sin), 16-byte aligned, caller-owned; the table
+ *           argument of the two calls above.  Built once per grid; angles in double precision, so every
+ *           entry is the correctly rounded fp16 value.
+ * base > 1 (10000 is customary); d even.  Errors: SALAD_ERR_INVALID_ARG, SALAD_ERR_UNSUPPORTED (more
+ * than 2^31 - 1 tokens), SALAD_ERR_CUDA.  Asynchronous on `stream`.
+ */
+int salad_rope3d_table_build(int T, int Hs, int Ws, int d, float base, void* d_rope, void* stream);
+
+/*
  * salad_dynamic_scale -- the input- and timestep-aware scaling factor of Algorithm 1, Level 2
  * (Sec. 4.2): a D -> 1 linear layer on the modulated hidden states, a sigmoid, a token average:
  *     s[b] = (1/N) sum_n sigmoid( <x[b,n,:], w> + bias ),   s in (0, 1).

@@ -17,6 +17,7 @@ LIB = os.path.join(HERE, "libsalad.so")
 SOURCES = ["salad_api.cu"]
 HEADERS = ["ptx.cuh", "tmap.cuh", "mask_kernels.cuh", "linear_state_kernel.cuh", "fused_kernel.cuh",
            "dynamic_scale_kernel.cuh", "linear_apply_kernel.cuh", "topk_mask_kernels.cuh", "permute_kernel.cuh", "proj_gemm_kernel.cuh",
+           "rope_table_kernel.cuh",
            os.path.join("..", "..", "include", "salad.h")]
 
 

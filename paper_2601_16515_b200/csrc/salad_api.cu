@@ -15,6 +15,7 @@
 #include "mask_kernels.cuh"
 #include "permute_kernel.cuh"
 #include "proj_gemm_kernel.cuh"
+#include "rope_table_kernel.cuh"
 #include "tmap.cuh"
 #include "topk_mask_kernels.cuh"
 
@@ -661,6 +662,26 @@ SALAD_EXPORT int salad_permute_tokens(const void* x, void* y, int B, int H, int 
         if (h_head_flags[h]) pp.flag_bits[h >> 5] |= 1u << (h & 31);
     permute_tokens_kernel<<<dim3(unsigned((N + kPermuteRows - 1) / kPermuteRows), unsigned(B * H)), kPermuteThreads, 0,
                             static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(x), static_cast<uint4*>(y), pp);
+    return check_launch();
+}
+
+SALAD_EXPORT int salad_rope3d_table_build(int T, int Hs, int Ws, int d, float base, void* d_rope, void* stream) {
+    if (!d_rope || T <= 0 || Hs <= 0 || Ws <= 0 || d <= 0 || (d & 1) || !(base > 1.f) || !isfinite(base))
+        return SALAD_ERR_INVALID_ARG;
+    if (!aligned16(d_rope)) return SALAD_ERR_INVALID_ARG;
+    const int64_t N = int64_t(T) * Hs * Ws;
+    if (N > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    RopeGeom g{};
+    g.T = T; g.Hs = Hs; g.Ws = Ws; g.pairs = d / 2;
+    g.p_hw = g.pairs / 3; g.p_t = g.pairs - 2 * g.p_hw;
+    g.entries = N * g.pairs;
+    g.log2_base = log2(double(base));
+    const long long blocks = (g.entries + 255) / 256;
+    if (blocks > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
+    rope3d_table_kernel<<<unsigned(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(g, static_cast<__half2*>(d_rope));
     return check_launch();
 }
 

@@ -28,7 +28,8 @@ EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
            "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
-           "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd")
+           "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd",
+           "salad_rope3d_table_build")
 
 
 class SaladError(RuntimeError):
@@ -76,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.salad_fused_rope_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, p, f32, f32, f32, p, sz, p, p]
     lib.salad_linear_attn_rope_fwd.restype = i32
     lib.salad_linear_attn_rope_fwd.argtypes = [p, p, p, p, p, p] + [i32] * 4 + [p, f32, p, sz, p, p]
+    lib.salad_rope3d_table_build.restype = i32
+    lib.salad_rope3d_table_build.argtypes = [i32, i32, i32, i32, f32, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
     return lib
@@ -202,6 +205,18 @@ def _rope_table(rope, N, d):
             or tuple(rope.shape) != (N, d // 2, 2)):
         raise ValueError(f"rope must be a contiguous CUDA fp16 tensor of shape [{N}, {d // 2}, 2] (cosine, sine)")
     return rope
+
+
+def salad_rope3d_table_build(T: int, Hs: int, Ws: int, d: int, base: float = 10000.0, out=None, device=None,
+                             stream=None):
+    """fp16 rotation table [T*Hs*Ws, d/2, 2] of the 3-D rotary embedding of a latent grid, on the device."""
+    if out is None:
+        out = torch.empty((T * Hs * Ws, d // 2, 2), dtype=torch.float16, device=device or "cuda")
+    _rope_table(out, T * Hs * Ws, d)
+    with torch.cuda.device(out.device):
+        _check(_lib.salad_rope3d_table_build(T, Hs, Ws, d, float(base), _ptr(out), _stream(stream)),
+               "salad_rope3d_table_build")
+    return out
 
 
 def salad_linear_attn_rope_fwd(q, k, v, rope, eps: float = 1e-6, out=None, kv_out=None, z_out=None,

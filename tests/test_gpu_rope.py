@@ -176,3 +176,29 @@ def test_fused_rope_call_in_a_cuda_graph_and_repeatable(salad):
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert torch.equal(out, eager)
+
+
+@pytest.mark.parametrize("grid,d", [((3, 4, 5), 32), ((4, 16, 16), 64), ((2, 7, 9), 128)])
+def test_rope3d_table_bit_exact(salad, grid, d):
+    got = salad.salad_rope3d_table_build(*grid, d).cpu().numpy()
+    ref = orc.rope3d_table(grid, d)
+    assert got.dtype == np.float16 and got.shape == ref.shape
+    assert np.array_equal(got.view(np.uint16), ref.view(np.uint16))
+
+
+def test_rope3d_table_wan13b_shape_sampled_and_feeds_the_fused_call(salad):
+    wl = wlmod.C2
+    table = salad.salad_rope3d_table_build(*wl.grid, wl.d)
+    tok = np.random.default_rng(11).integers(0, wl.N, size=400)
+    ref = orc.rope3d_table(wl.grid, wl.d, tokens=tok)
+    assert np.array_equal(table.cpu().numpy()[tok].view(np.uint16), ref.view(np.uint16))
+    # other bases and the argument checks
+    t2 = salad.salad_rope3d_table_build(2, 3, 4, 64, base=500.0).cpu().numpy()
+    assert np.array_equal(t2.view(np.uint16), orc.rope3d_table((2, 3, 4), 64, base=500.0).view(np.uint16))
+    with pytest.raises(salad.SaladError):
+        salad.salad_rope3d_table_build(2, 3, 4, 64, base=1.0)
+    # the device-built table is the one the rotary calls take
+    q, k, v = (t.cuda() for t in wlmod.make_qkv(wl, heads=[0, 1]))
+    a = salad.salad_linear_attn_rope_fwd(q, k, v, table)
+    b = salad.salad_linear_attn_rope_fwd(q, k, v, torch.from_numpy(wlmod.rope_table(wl.grid, wl.d)).cuda())
+    assert torch.equal(a, b)
