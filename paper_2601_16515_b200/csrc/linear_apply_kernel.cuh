@@ -15,22 +15,30 @@
 //               swizzled staging tile, TMA store (the tile is free again as soon as the store
 //               has read it, long before the next accumulator is ready)
 // Every hand-over is an mbarrier with a bounded wait.
+//
+// ROPE variant (rotary position embedding in the linear branch, Sec. 4.1): a Q stage also holds the fp16
+// rotation rows (cos, sin per channel pair) of the tile's 128 tokens, laid out like the Q tile itself (same
+// 128-byte swizzle), so a row thread reads the four (cos, sin) values of a 16-byte Q vector from the same
+// offset; the denominator takes the un-rotated ReLU values, the MMA the rotated ones.  The ring is two
+// stages of 64 KB then, and the state has one buffer (a CTA meets a second head at most once or twice).
 #pragma once
 #include "ptx.cuh"
 
 namespace salad {
 
-template <int D>
+template <int D, bool ROPE = false>
 struct ApplyCfg {
     static constexpr int CH = D / 64;                  // 128-byte chunks per row
     static constexpr int Q_CHUNK = 128 * 128;          // bytes of one 64-column chunk of a 128-row tile
     static constexpr int Q_BYTES = CH * Q_CHUNK;
     static constexpr int ST_CHUNK = D * 128;
     static constexpr int ST_BYTES = CH * ST_CHUNK;     // bf16 state [d][d], transposed
-    static constexpr int NQ = 3;                       // Q stages
+    static constexpr int NQ = ROPE ? 2 : 3;            // Q stages
+    static constexpr int STAGE_BYTES = ROPE ? 2 * Q_BYTES : Q_BYTES;   // Q tile, then its rotation rows
+    static constexpr int NST = ROPE ? 1 : 2;           // state buffers
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_ST = NQ * Q_BYTES;
-    static constexpr int OFF_O = OFF_ST + 2 * ST_BYTES;
+    static constexpr int OFF_ST = NQ * STAGE_BYTES;
+    static constexpr int OFF_O = OFF_ST + NST * ST_BYTES;
     static constexpr int SMEM_BYTES = OFF_O + Q_BYTES + 1024;       // + alignment slack
     static constexpr int THREADS = 320;
     static constexpr int TMEM_COLS = 2 * D;            // 256 or 128: a power of two
@@ -54,12 +62,13 @@ struct ApplyBarriers {
     uint64_t acc_full[2], acc_free[2], out_staged, out_free;
 };
 
-template <int D>
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(320)
 salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_st,
-                          const __grid_constant__ CUtensorMap map_o, const ApplyParams p)
+                          const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_r,
+                          const ApplyParams p)
 {
-    using C = ApplyCfg<D>;
+    using C = ApplyCfg<D, ROPE>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ ApplyBarriers bars;
     __shared__ float z_s[2][D];
@@ -105,12 +114,13 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         // ============================================================== TMA producer
         if (lane == 0) {
             prefetch_tmap(&map_q); prefetch_tmap(&map_st); prefetch_tmap(&map_o);
+            if (ROPE) prefetch_tmap(&map_r);
             int prev_bh = -1, n_st = 0, j = 0;
             for (long long t = t0; t < t1; ++t, ++j) {
                 const int bh = int(t / p.nQb), qb = int(t % p.nQb);
                 if (bh != prev_bh) {
-                    const int sb = n_st & 1;
-                    if (!mbar_wait(smem_u32(&bars.st_empty[sb]), ((n_st >> 1) & 1) ^ 1, abortp)) break;
+                    const int sb = n_st % C::NST;
+                    if (!mbar_wait(smem_u32(&bars.st_empty[sb]), ((n_st / C::NST) & 1) ^ 1, abortp)) break;
                     const uint32_t bar = smem_u32(&bars.st_full[sb]);
                     mbar_arrive_expect_tx(bar, C::ST_BYTES);
                     for (int ch = 0; ch < C::CH; ++ch)
@@ -121,10 +131,14 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 const int s = j % C::NQ;
                 if (!mbar_wait(smem_u32(&bars.q_empty[s]), ((j / C::NQ) & 1) ^ 1, abortp)) break;
                 const uint32_t bar = smem_u32(&bars.q_full[s]);
-                mbar_arrive_expect_tx(bar, C::Q_BYTES);
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(s_base + C::OFF_Q + s * C::Q_BYTES + ch * C::Q_CHUNK, &map_q, bar,
+                mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    tma_load_3d(s_base + C::OFF_Q + s * C::STAGE_BYTES + ch * C::Q_CHUNK, &map_q, bar,
                                 ch * 64, qb * 128, bh);
+                    if (ROPE)
+                        tma_load_3d(s_base + C::OFF_Q + s * C::STAGE_BYTES + C::Q_BYTES + ch * C::Q_CHUNK, &map_r, bar,
+                                    ch * 64, qb * 128, 0);
+                }
             }
         }
     } else if (warp == 1) {
@@ -139,8 +153,8 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 if (bh != prev_bh) {
                     // the MMAs that read the previous state buffer are all issued: hand it back
                     if (prev_bh >= 0) tc_commit(smem_u32(&bars.st_empty[sb]));
-                    sb = n_st & 1;
-                    ok = mbar_wait(smem_u32(&bars.st_full[sb]), (n_st >> 1) & 1, abortp);
+                    sb = n_st % C::NST;
+                    ok = mbar_wait(smem_u32(&bars.st_full[sb]), (n_st / C::NST) & 1, abortp);
                     if (!ok) break;
                     ++n_st; prev_bh = bh;
                 }
@@ -149,7 +163,7 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 if (ok) ok = mbar_wait(smem_u32(&bars.acc_free[ab]), ((j >> 1) & 1) ^ 1, abortp);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + s * C::Q_BYTES, 16);
+                const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q + s * C::STAGE_BYTES, 16);
                 const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST + sb * C::ST_BYTES, 16);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
@@ -183,7 +197,7 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             const int s = j % C::NQ;
             ok = mbar_wait(smem_u32(&bars.q_full[s]), (j / C::NQ) & 1, abortp);
             if (!ok) break;
-            uint8_t* qtile = smem + C::OFF_Q + s * C::Q_BYTES;
+            uint8_t* qtile = smem + C::OFF_Q + s * C::STAGE_BYTES;
             const float* zz = z_s[zb];
             float den = 0.f;
 #pragma unroll
@@ -193,6 +207,9 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                     uint4* ptr = reinterpret_cast<uint4*>(qtile + ch * C::Q_CHUNK + row * 128 + ((c16 ^ (row & 7)) << 4));
                     uint4 v = *ptr;
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&v);
+                    uint4 tv = make_uint4(0, 0, 0, 0);
+                    if (ROPE) tv = *reinterpret_cast<const uint4*>(reinterpret_cast<uint8_t*>(ptr) + C::Q_BYTES);
+                    const __half2* th = reinterpret_cast<const __half2*>(&tv);      // (cos, sin) of four pairs
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         hv[e] = __hmax2(hv[e], __float2bfloat162_rn(0.f));
@@ -200,6 +217,10 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                         const int a = ch * 64 + c16 * 8 + e * 2;
                         den = fmaf(f.x, zz[a], den);
                         den = fmaf(f.y, zz[a + 1], den);
+                        if (ROPE) {
+                            const float2 cs = __half22float2(th[e]);
+                            hv[e] = __floats2bfloat162_rn(cs.x * f.x - cs.y * f.y, cs.y * f.x + cs.x * f.y);
+                        }
                     }
                     *ptr = v;
                 }

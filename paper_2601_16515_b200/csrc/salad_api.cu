@@ -121,11 +121,17 @@ int prepare_device(DeviceInfo* info) {
             e = cudaFuncSetAttribute(salad_linear_state_kernel<64, true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     ApplyCfg<128>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<128, false>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(salad_linear_apply_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     ApplyCfg<64>::SMEM_BYTES);
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<64, false>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<128, true>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_linear_apply_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ApplyCfg<64, true>::SMEM_BYTES);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(topk_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      128 * (kScoreRows + kScoreTile) * 4);
@@ -293,10 +299,13 @@ template <int D>
 int launch_apply(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     const int BH = P.B * P.H;
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
-    CUtensorMap mq, mo, ms;
+    CUtensorMap mq, mo, ms, mr;
     if (!make_tmap_bf16_3d(&mq, P.q, D, P.N, BH, 128) || !make_tmap_bf16_3d(&mo, P.o, D, P.N, BH, 128) ||
         !make_tmap_bf16_3d(&ms, ws + w.off_kvt, D, D, BH, D))
         return SALAD_ERR_CUDA;
+    mr = mq;                      // unused without a rotation table
+    // the fp16 table [N, D] is tiled exactly like a Q tile of one (batch, head): 16-bit elements, 128-byte swizzle
+    if (P.rope && !make_tmap_bf16_3d(&mr, P.rope, D, P.N, 1, 128)) return SALAD_ERR_CUDA;
     ApplyParams ap;
     ap.N = P.N; ap.H = P.H;
     ap.nQb = (P.N + 127) / 128;
@@ -308,8 +317,12 @@ int launch_apply(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     ap.user_status = P.d_status;
     const unsigned grid = unsigned(ap.tiles < dev.sms ? ap.tiles : dev.sms);
     record_profile(2, P.stream);
-    launch_dependent(salad_linear_apply_kernel<D>, dim3(grid), dim3(ApplyCfg<D>::THREADS), ApplyCfg<D>::SMEM_BYTES,
-                     P.stream, mq, ms, mo, ap);
+    if (P.rope)
+        launch_dependent(salad_linear_apply_kernel<D, true>, dim3(grid), dim3(ApplyCfg<D, true>::THREADS),
+                         ApplyCfg<D, true>::SMEM_BYTES, P.stream, mq, ms, mo, mr, ap);
+    else
+        launch_dependent(salad_linear_apply_kernel<D, false>, dim3(grid), dim3(ApplyCfg<D, false>::THREADS),
+                         ApplyCfg<D, false>::SMEM_BYTES, P.stream, mq, ms, mo, mr, ap);
     record_profile(3, P.stream);
     return check_launch();
 }
@@ -338,9 +351,8 @@ int run(const Problem& P) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
         if (rc != SALAD_OK) return rc;
     }
-    // linear-only calls: the stand-alone apply kernel; with a rotation table the attention kernel's epilogue
-    // does the apply step (every query block has an empty kept list)
-    if (P.mode == MODE_LINEAR && !P.rope)
+    // linear-only calls: the stand-alone apply kernel
+    if (P.mode == MODE_LINEAR)
         return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
     return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
 }
