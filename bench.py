@@ -432,8 +432,10 @@ def main():
         rope_d = salad.salad_rope3d_table_build(*wl.grid, wl.d, device=dev)
         rope_ms = timed(lambda: salad.salad_fused_rope_fwd(q, k, v, rp, ci, Hm, lam_d, s_d, rope_d, Bq=wl.Bq, Bk=wl.Bk,
                                                            out=out, workspace=ws), 20)
+        rope_lin_ms = timed(lambda: salad.salad_linear_attn_rope_fwd(q, k, v, rope_d, out=out, workspace=ws), 20)
         extras["rope_linear_branch"] = {"fused_ms": rope_ms, "fused_tflops": flops / (rope_ms * 1e-3) / 1e12,
-                                        "extra_ms_over_plain_call": rope_ms - ms_per_step}
+                                        "extra_ms_over_plain_call": rope_ms - ms_per_step,
+                                        "linear_only_ms": rope_lin_ms}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
