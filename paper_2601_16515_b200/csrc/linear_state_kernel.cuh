@@ -302,15 +302,20 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
     for (int r = 0; r < 32 / ROWS; ++r) {
         const int a = a0 + ty + ROWS * r;
         const float* src = kv_part + size_t(bh) * chunks * D * D + size_t(a) * D + c0 + tx;
+        // fixed order: ((p0+p4+..)+(p1+p5+..))+((p2+..)+(p3+..)), the chunks % 4 last partials into the first
+        // sum; sixteen loads are issued before the first add (the kernel is a chain of L2 round trips otherwise)
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int ch = 0;
-        for (; ch + 4 <= chunks; ch += 4) {           // fixed order: ((p0+p4+..)+(p1+p5+..))+...
-            s0 += src[size_t(ch) * D * D];
-            s1 += src[size_t(ch + 1) * D * D];
-            s2 += src[size_t(ch + 2) * D * D];
-            s3 += src[size_t(ch + 3) * D * D];
+        const int full = chunks & ~3;
+        for (int ch0 = 0; ch0 < chunks; ch0 += 16) {
+            float v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) v[u] = (ch0 + u < chunks) ? src[size_t(ch0 + u) * D * D] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 16; u += 4) {
+                if (ch0 + u + 4 <= full) { s0 += v[u]; s1 += v[u + 1]; s2 += v[u + 2]; s3 += v[u + 3]; }
+                else if (ch0 + u < chunks) { s0 += v[u]; s0 += v[u + 1]; s0 += v[u + 2]; }    // absent ones are zero
+            }
         }
-        for (; ch < chunks; ++ch) s0 += src[size_t(ch) * D * D];
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
         tile[ty + ROWS * r][tx] = s;
