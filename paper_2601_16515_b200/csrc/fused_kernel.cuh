@@ -329,7 +329,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int lane0 = (warp & 3) * 32 + (sw >> 2) * 16;          // first TMEM lane of this warp
         const int ra = lane0 + (lane >> 2), rb = ra + 8;        // the thread's two query rows
         const uint32_t t_tile = tmem + (uint32_t(lane0) << 16);
-        const bool tile_valid = true;
         const int len = le - ls;
         uint8_t* qtile = smem + C::OFF_Q;
         float m_a = -INFINITY, m_b = -INFINITY;                 // running maxima (log2 domain)
@@ -446,7 +445,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (ra == 0 && q4 == 0) TRACE(0, t, 5);
         }
         float coef_a = 0.f, coef_b = 0.f;
-        if (ok && tile_valid && linear) {
+        if (ok && linear) {
             // ReLU of the Q rows in place, and the denominators ReLU(Q_n) . Z: the four threads of a
             // row take two 16-byte groups of every 64 channels each.  Every Q K^T of this tile has
             // completed (its scores were consumed above), so Q is no longer read; the last P V
@@ -513,12 +512,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             ok = wait_uniform(&bars.o_final, 0);
             tc_fence_after_sync();
         }
-        if (ok && tile_valid && linear) {
+        if (ok && linear) {
             ok = wait_uniform(&bars.lin_done, 0);
             tc_fence_after_sync();
         }
 
-        if (ok && tile_valid) {
+        if (ok) {
             // O = O_acc / l + coef * num, rounded once to bf16, staged in the Q tile
             const float lt_a = quad_sum(l_a), lt_b = quad_sum(l_b);
             const float inv_a = (len > 0) ? 1.0f / lt_a : 0.f, inv_b = (len > 0) ? 1.0f / lt_b : 0.f;
