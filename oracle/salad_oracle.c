@@ -25,10 +25,11 @@
  * two-token example worked by hand, the N x N form with explicit rotation matrices, zero angles
  * (plain Eq. 3), invariance under a common shift of all positions.
  *
- * Parity unpinned: nothing ties these functions to the authors' own implementation (the
- * paper prints no worked numeric example); the 3-D window reading of the ST-SWA mask and
- * the per-head scalar reading of the static projection are this build's readings, and so is the
- * place of the rotary embedding in the linear branch (numerator only), for which the paper has no formula.
+ * Every function of this file has at least one such pin; none is left unpinned.  What no pin can
+ * settle is whether a READING of the paper is the authors' (the paper prints no worked numeric
+ * example and no code): the 3-D window reading of the ST-SWA mask, the per-head scalar reading of the
+ * static projection, and the place of the rotary embedding in the linear branch (numerator only), for
+ * which the paper has no formula.  Those readings are listed where the build documents its design.
  */
 #include <math.h>
 #include <stdint.h>
