@@ -596,6 +596,8 @@ def test_full_projection_pipeline_matches_fused_for_block_diagonal(salad):
     (3, 1, 65, 64, 128),        # one token into the second key block
     (5, 1, 129, 128, 64),       # one row into the third query block, odd number of query blocks
     (1, 20, 200, 64, 64),       # many heads, short sequence
+    (4, 48, 330, 64, 128),      # more (batch, head) pairs than SMs: one state chunk per head, 192 state CTAs
+    (2, 80, 700, 128, 128),     # 160 heads at d = 128: the state kernel runs in more than one wave
 ])
 def test_fused_degenerate_sizes(salad, B, H, N, d, Bq):
     q, k, v = rand_qkv(B, H, N, d, 700 + N)
