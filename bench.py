@@ -109,16 +109,19 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def oracle_sample(wl, steps, warmup, rank):
-    """CPU oracle on a bounded sample: the first `heads` heads of batch item 0, every query
-    row; those heads' linear states are computed in full inside the timed call."""
+def oracle_sample(wl, steps, warmup, rank, heads=None, rows=None):
+    """CPU oracle on a bounded sample: the first `heads` heads of batch item 0 and the first `rows` query
+    rows of each (default: 8 heads, every row); those heads' linear states are computed in full inside the
+    timed call."""
     from oracle import salad_oracle as orc
-    nh = min(wl.H, int(os.environ.get("SALAD_ORACLE_HEADS", "8")))
+    orc.use_all_cores()          # a multi-process launcher sets OMP_NUM_THREADS=1; the other ranks do no CPU work here
+    nh = min(wl.H, heads if heads else int(os.environ.get("SALAD_ORACLE_HEADS", "8")))
+    nr = wl.N if not rows else max(1, min(wl.N, int(rows)))
     q, k, v = (t.float().numpy() for t in wlmod.make_qkv(wl, heads=list(range(nh))))
     T, Hs, Ws = wl.grid
     rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
     lam, s = wlmod.make_scales(wl)
-    sel = np.arange(nh * wl.N, dtype=np.int64)
+    sel = (np.arange(nh, dtype=np.int64)[:, None] * wl.N + np.arange(nr, dtype=np.int64)[None, :]).reshape(-1)
     nQb = wl.nQb
     vk = np.minimum(wl.Bk, wl.N - np.arange(wl.nKb) * wl.Bk).astype(np.float64)
     keys_per_qb = np.array([vk[ci[rp[i]:rp[i + 1]]].sum() for i in range(nQb)])
@@ -132,17 +135,25 @@ def oracle_sample(wl, steps, warmup, rank):
             times.append(dt)
     sec = float(np.mean(times))
     return {"value": flops / sec / 1e12, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
-            "sample": f"{nh} of {wl.B * wl.H} heads, all {wl.N} query rows each (kept-block flops of "
-                      f"those rows), those heads' linear states included in the time; "
+            "sample": f"{nh} of {wl.B * wl.H} heads, the first {nr} of {wl.N} query rows each (kept-block flops "
+                      f"of those rows), those heads' linear states included in the time; "
                       f"{sec:.2f} s per pass"}, sec
 
 
 def run_reference(args, wl, rank, world):
+    """The oracle as the reference arm: exactly --steps timed passes after --warmup untimed ones, each pass a
+    sample of the workload sized (from one calibration pass over a single head) so that the whole run takes
+    about two to three minutes."""
     if rank != 0:
         return
-    steps = max(1, min(args.steps, 3))
-    warm = min(args.warmup, 1)
-    base, sec = oracle_sample(wl, steps, warm, rank)
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    _, t_head = oracle_sample(wl, 1, 0, rank, heads=1)                 # calibration: one head, every row
+    budget = min(20.0, 150.0 / (steps + warm))                         # seconds per pass
+    if t_head <= budget:
+        heads, rows = max(1, min(8, wl.H, int(budget / t_head))), None
+    else:                                                              # less than a head: a prefix of its rows
+        heads, rows = 1, max(wl.Bq, int(wl.N * budget / t_head) // wl.Bq * wl.Bq)
+    base, sec = oracle_sample(wl, steps, warm, rank, heads=heads, rows=rows)
     line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

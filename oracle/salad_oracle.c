@@ -38,6 +38,29 @@
 
 #define ORACLE_API __attribute__((visibility("default")))
 
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Threads of the parallel-for loops below: a launcher may have set OMP_NUM_THREADS=1 for the process. */
+ORACLE_API void oracle_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+ORACLE_API int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
 static int iabs(int x) { return x < 0 ? -x : x; }
 
 /* Does any (query token in block i, key token in block j) pair lie inside the 3-D window?

@@ -64,6 +64,10 @@ def _load():
         lib.oracle_salad_fused_rope.restype = None
         lib.oracle_salad_fused_rope.argtypes = ([p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
                                                                             p, i64, p])
+        lib.oracle_set_threads.restype = None
+        lib.oracle_set_threads.argtypes = [i32]
+        lib.oracle_max_threads.restype = i32
+        lib.oracle_max_threads.argtypes = []
         _lib = lib
     return _lib
 
@@ -86,14 +90,19 @@ def _sel(sel):
 
 
 def num_threads() -> int:
-    """Threads the OpenMP runtime will use (OMP_NUM_THREADS or all visible cores)."""
-    env = os.environ.get("OMP_NUM_THREADS")
-    if env:
-        return int(env.split(",")[0])
+    """Threads the oracle's parallel loops will use."""
+    return int(_load().oracle_max_threads())
+
+
+def use_all_cores() -> int:
+    """Let the parallel loops use every core this process may run on, whatever OMP_NUM_THREADS says
+    (launchers of multi-process jobs set it to 1).  Returns the thread count."""
     try:
-        return len(os.sched_getaffinity(0))
+        n = len(os.sched_getaffinity(0))
     except AttributeError:
-        return os.cpu_count() or 1
+        n = os.cpu_count() or 1
+    _load().oracle_set_threads(n)
+    return num_threads()
 
 
 def mask_build(T, Hs, Ws, Bq, Bk, windows):
