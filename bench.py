@@ -148,11 +148,11 @@ def run_reference(args, wl, rank, world):
         return
     steps, warm = max(1, args.steps), max(0, args.warmup)
     _, t_head = oracle_sample(wl, 1, 0, rank, heads=1)                 # calibration: one head, every row
-    budget = min(20.0, 150.0 / (steps + warm))                         # seconds per pass
-    if t_head <= budget:
-        heads, rows = max(1, min(8, wl.H, int(budget / t_head))), None
+    per_pass_s = min(20.0, 150.0 / (steps + warm))                         # seconds per pass
+    if t_head <= per_pass_s:
+        heads, rows = max(1, min(8, wl.H, int(per_pass_s / t_head))), None
     else:                                                              # less than a head: a prefix of its rows
-        heads, rows = 1, max(wl.Bq, int(wl.N * budget / t_head) // wl.Bq * wl.Bq)
+        heads, rows = 1, max(wl.Bq, int(wl.N * per_pass_s / t_head) // wl.Bq * wl.Bq)
     base, sec = oracle_sample(wl, steps, warm, rank, heads=heads, rows=rows)
     line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": sec * 1e3, "higher_is_better": True,
