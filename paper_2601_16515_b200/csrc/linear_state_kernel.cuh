@@ -52,6 +52,7 @@ struct StateParams {
     float* z_part;        // [BH][chunks][D]
     int32_t* ws_status;
     int32_t* user_status;
+    int clear_status;         // 1: this kernel is the first of its call and clears the status words itself
     const float* dyn_scale;   // [B] or null: with drop_tau, batch items whose scale is below it are skipped
     float drop_tau;
     int H;
@@ -78,6 +79,14 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t s_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x, bh = blockIdx.y;
+    // First kernel of a linear-only call (an ordinary launch, so everything before it in the stream is done):
+    // its first CTA, which is in the first wave, clears the status words at once; a CTA sets them only after
+    // a bounded wait of a second has run out.  No CTA of this kernel reads them (there is no earlier kernel of
+    // the call whose failure it would have to honour).
+    if (p.clear_status && chunk == 0 && bh == 0 && tid == 0) {
+        p.ws_status[0] = 0; p.ws_status[1] = 0;
+        if (p.user_status) *p.user_status = 0;
+    }
     if (branch_dropped(p.dyn_scale, p.drop_tau, bh / p.H)) {           // whole CTA, before any allocation
         grid_dependency_wait();        // an exit releases the kernels after this one: not before the kernel before it is done
         return;
@@ -120,7 +129,7 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
     grid_dependency_wait();            // the status word is cleared by the kernel before
     grid_launch_dependents();
-    if (tid == 0) abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+    if (tid == 0) abort_flag = (!p.clear_status && *reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();

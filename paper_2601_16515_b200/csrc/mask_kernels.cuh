@@ -117,19 +117,6 @@ __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int32_t* __re
     }
 }
 
-// First kernel of a call that has no work-order kernel: clears the status words (and the work-item
-// counter next to the library's).  The kernel after it in the stream is launched so that it can be
-// set up and start its input loads meanwhile.
-__global__ void __launch_bounds__(32) status_clear_kernel(int32_t* __restrict__ ws_status,
-                                                          int32_t* __restrict__ user_status) {
-    grid_launch_dependents();
-    if (threadIdx.x == 0) {
-        ws_status[0] = 0;
-        ws_status[1] = 0;
-        if (user_status) *user_status = 0;
-    }
-}
-
 // Launch order of the attention kernel's work items: for every mask head, the query blocks
 // sorted by decreasing length of their kept list, so that the long items start first and the
 // short ones fill the tail.  Counting sort in shared memory; one CTA per mask head.  The order

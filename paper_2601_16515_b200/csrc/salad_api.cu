@@ -226,8 +226,14 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     // Fused calls: the short-ring variant, which shares its SM with a CTA of the attention kernel.  With a
     // rotation table the state pass keeps the SM to itself (full ring, eight ReLU warps): sharing the SM with
     // the attention kernel was measured no faster.
+    // In a linear-only call this is the first kernel: an ordinary launch (it must not start before the call
+    // before it has ended), which clears the status words itself.
+    sp.clear_status = (P.mode & MODE_SPARSE) ? 0 : 1;
     auto launch = [&](auto kernel, int threads, int smem) {
-        launch_dependent(kernel, dim3(chunks, BH), dim3(threads), size_t(smem), P.stream, mk, mv, mr, sp);
+        if (sp.clear_status)
+            kernel<<<dim3(chunks, BH), dim3(threads), size_t(smem), P.stream>>>(mk, mv, mr, sp);
+        else
+            launch_dependent(kernel, dim3(chunks, BH), dim3(threads), size_t(smem), P.stream, mk, mv, mr, sp);
     };
     if (P.rope)
         launch(salad_linear_state_kernel<D, false, true>, StateCfg<D, false, true>::THREADS,
@@ -342,9 +348,6 @@ int run(const Problem& P) {
         work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb,
                                                       reinterpret_cast<int32_t*>(ws + w.off_order),
                                                       reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
-        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    } else {
-        status_clear_kernel<<<1, 32, 0, P.stream>>>(reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
         if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     }
     if (P.mode & MODE_LINEAR) {
@@ -762,10 +765,7 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     P.eps = eps; P.kv_out = kv_out; P.z_out = z_out;
     P.ws = scratch; P.ws_bytes = kNoAllocBytes; P.d_status = d_status;
     P.stream = static_cast<cudaStream_t>(stream);
-    // the array keeps the last call's contents: the status word must start at zero
-    uint8_t* ws = static_cast<uint8_t*>(scratch);
-    status_clear_kernel<<<1, 32, 0, P.stream>>>(reinterpret_cast<int32_t*>(ws + w.off_status), d_status);
-    if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+    // (the array keeps the last call's contents: the state kernel, first of the call, clears the status words)
     rc = (d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
     if (rc != SALAD_OK) return rc;
     return (d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);

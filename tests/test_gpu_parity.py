@@ -740,3 +740,22 @@ def test_fused_call_in_a_cuda_graph(salad):
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert torch.equal(out, eager)
+
+
+def test_calls_do_not_depend_on_the_workspace_contents(salad):
+    # the first kernel of every call clears the status words; nothing else is read before it is written
+    B, H, N, d = 1, 3, 1500, 128
+    q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 321))
+    rp, ci = random_csr(-(-N // 128), -(-N // 64), 5, lo=1, hi=8)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = torch.rand(H, device="cuda"); s = torch.rand(B, device="cuda")
+    clean = salad.alloc_workspace(B, H, N, d); clean.zero_()
+    dirty = torch.full_like(clean, 0xFF)
+    for fn in (lambda ws, st: salad.salad_linear_attn_fwd(q, k, v, workspace=ws, status=st),
+               lambda ws, st: salad.salad_fused_fwd(q, k, v, rp_d, ci_d, 1, lam, s, workspace=ws, status=st),
+               lambda ws, st: salad.salad_sparse_attn_fwd(q, k, v, rp_d, ci_d, 1, workspace=ws, status=st)):
+        st_a = torch.full((1,), 77, dtype=torch.int32, device="cuda"); st_b = st_a.clone()
+        a = fn(clean, st_a); b = fn(dirty, st_b)
+        torch.cuda.synchronize()
+        assert int(st_a.item()) == 0 and int(st_b.item()) == 0
+        assert torch.equal(a, b)
