@@ -223,8 +223,9 @@ ORACLE_API void oracle_linear_state(const float* k, const float* v, int B, int H
 /*
  * oracle_linear_attn: Eq. 3 for selected rows, from the state,
  *     O_l[n] = ReLU(Q_n) KV / (ReLU(Q_n) . Z + eps).
- * The paper's denominator has no eps; eps > 0 only defines the 0/0 case (all ReLU(Q_n)
- * zero gives O_l = 0).
+ * The paper's denominator has no eps; eps only defines the 0/0 case: a row whose ReLU(Q_n) . Z is
+ * zero (then the numerator is zero too: Z bounds every column of KV's weights) gives O_l = 0, also
+ * with eps = 0, where the quotient would be 0/0.
  */
 ORACLE_API void oracle_linear_attn(const float* q, const double* kv, const double* z,
                                    int B, int H, int N, int d, double eps,
@@ -244,7 +245,7 @@ ORACLE_API void oracle_linear_attn(const float* q, const double* kv, const doubl
         for (int c = 0; c < d; ++c) {
             double num = 0.0;
             for (int a = 0; a < d; ++a) num += relu((double)qn[a]) * kvb[(int64_t)a * d + c];
-            on[c] = num / (den + eps);
+            on[c] = (den + eps > 0.0) ? num / (den + eps) : 0.0;   /* 0/0 (eps = 0, ReLU(Q_n) . Z = 0) is taken as 0 */
         }
     }
 }
@@ -490,7 +491,7 @@ ORACLE_API void oracle_linear_attn_rope(const float* q, const float* rope, const
         for (int c = 0; c < d; ++c) {
             double num = 0.0;
             for (int a = 0; a < d; ++a) num += fr[a] * kvb[(int64_t)a * d + c];
-            on[c] = num / (den + eps);
+            on[c] = (den + eps > 0.0) ? num / (den + eps) : 0.0;   /* 0/0 (eps = 0, ReLU(Q_n) . Z = 0) is taken as 0 */
         }
         free(f); free(fr);
     }

@@ -1,7 +1,7 @@
 """Seeded synthetic inputs for the SALAD attention path.
 
-This module only *generates inputs* (tensors, scale parameters, rotation tables, irregular block
-lists, trivial all-kept lists).  It contains none of the method's arithmetic, and it is the one
+This module only *generates inputs* (tensors, scale parameters, irregular block lists, trivial
+all-kept lists).  It contains none of the method's arithmetic, and it is the one
 module that both the CPU oracle's callers and the GPU library's callers may use, so that
 both sides see bit-identical operands.  It needs numpy and torch (CPU) only.
 
@@ -119,29 +119,6 @@ def make_scales(wl: Workload):
     lam = rng.uniform(0.0, 1.0, size=wl.H).astype(np.float32)
     s = (1.0 / (1.0 + np.exp(-rng.standard_normal(wl.B)))).astype(np.float32)
     return lam, s
-
-
-def rope_table(grid, d: int, base: float = 10000.0) -> np.ndarray:
-    """Rotation table of a 3-D rotary position embedding, an INPUT of the rotary linear branch (the
-    vectorised twin of the oracle's token-by-token definition, bit-identical to it, so that full-size
-    tables need no minutes of Python loops; the library's own producer is checked against the oracle):
-    float16 [N, d/2, 2] (the dtype of the library's table argument; the oracle widens the same values)
-    holding the cosine and sine of the angle of every token and channel pair.
-    The d/2 channel pairs are shared out among the t, h and w axes of the latent grid (the last two
-    get floor(d/6) pairs each, t the rest, as video DiTs of the Wan family do); pair j of an axis with
-    P pairs turns by position * base**(-j / P) for a token at that position along the axis.  Tokens are
-    numbered with time slowest, n = (t*Hs + h)*Ws + w.  Angles are formed in float64."""
-    T, Hs, Ws = grid
-    pairs = d // 2
-    p_hw = pairs // 3
-    p_t = pairs - 2 * p_hw
-    t, h, w = np.meshgrid(np.arange(T), np.arange(Hs), np.arange(Ws), indexing="ij")
-    parts = []
-    for pos, P in ((t, p_t), (h, p_hw), (w, p_hw)):
-        freq = base ** (-np.arange(P, dtype=np.float64) / max(P, 1))
-        parts.append(pos.reshape(-1, 1).astype(np.float64) * freq[None, :])
-    ang = np.concatenate(parts, axis=1)                      # [N, d/2]
-    return np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float16)
 
 
 def irregular_csr(wl: Workload, lo_frac: float = 0.05, hi_frac: float = 0.15):

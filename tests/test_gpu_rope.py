@@ -79,7 +79,7 @@ def test_fused_rope_tiny_config_with_the_3d_table(salad):
     T, Hs, Ws = wl.grid
     rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
     lam, s = wlmod.make_scales(wl)
-    rope = wlmod.rope_table(wl.grid, wl.d)
+    rope = orc.rope3d_table_vectorized(wl.grid, wl.d)
     rp_d, ci_d = dev_csr(rp, ci)
     args = (q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, wl.Hm, torch.from_numpy(lam).cuda(), torch.from_numpy(s).cuda(),
             torch.from_numpy(rope).cuda())
@@ -103,7 +103,7 @@ def test_fused_rope_wan13b_90_sampled(salad):
     q, k, v = wlmod.make_qkv(wl)
     T, Hs, Ws = wl.grid
     lam, s = wlmod.make_scales(wl)
-    rope = wlmod.rope_table(wl.grid, wl.d)
+    rope = orc.rope3d_table_vectorized(wl.grid, wl.d)
     rp_d, ci_d = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
     rp, ci = rp_d.cpu().numpy(), ci_d.cpu().numpy()
     status = torch.ones(1, dtype=torch.int32, device="cuda")
@@ -154,7 +154,7 @@ def test_fused_rope_drops_per_batch_item(salad):
 def test_fused_rope_call_in_a_cuda_graph_and_repeatable(salad):
     B, H, N, d = 1, 4, 2048, 128
     q, k, v = (t.cuda() for t in rand_qkv(B, H, N, d, 911))
-    rope = torch.from_numpy(wlmod.rope_table((4, 16, 32), d)).cuda()
+    rope = torch.from_numpy(orc.rope3d_table_vectorized((4, 16, 32), d)).cuda()
     rp, ci = salad.salad_mask_build(4, 16, 32, 128, 64, [(1, 3, 8)])
     lam = torch.rand(H, device="cuda"); s = torch.rand(B, device="cuda")
     ws = salad.alloc_workspace(B, H, N, d)
@@ -200,5 +200,5 @@ def test_rope3d_table_wan13b_shape_sampled_and_feeds_the_fused_call(salad):
     # the device-built table is the one the rotary calls take
     q, k, v = (t.cuda() for t in wlmod.make_qkv(wl, heads=[0, 1]))
     a = salad.salad_linear_attn_rope_fwd(q, k, v, table)
-    b = salad.salad_linear_attn_rope_fwd(q, k, v, torch.from_numpy(wlmod.rope_table(wl.grid, wl.d)).cuda())
+    b = salad.salad_linear_attn_rope_fwd(q, k, v, torch.from_numpy(orc.rope3d_table_vectorized(wl.grid, wl.d)).cuda())
     assert torch.equal(a, b)

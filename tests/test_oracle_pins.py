@@ -243,6 +243,12 @@ def test_linear_closed_forms():
     # Q <= 0 everywhere -> numerator and denominator vanish -> 0 (eps defines 0/0)
     o = orc.linear_attn(-np.abs(q), k, v, eps=1e-6)
     assert (o == 0).all()
+    # ... and without eps the quotient 0/0 is taken as 0 as well, never NaN; rows with a positive
+    # denominator are untouched by that rule
+    qz = q.copy(); qz[:, :, ::3] = -np.abs(qz[:, :, ::3])
+    o0 = orc.linear_attn(qz, k, v, eps=0.0).reshape(B, H, N, d)
+    assert np.isfinite(o0).all() and (o0[:, :, ::3] == 0).all()
+    np.testing.assert_array_equal(o0[:, :, 1::3], orc.linear_attn(q, k, v, eps=0.0).reshape(B, H, N, d)[:, :, 1::3])
     # homogeneity: phi(a K) = a phi(K) for a > 0 cancels between numerator and denominator
     o1 = orc.linear_attn(q, k, v, eps=0.0)
     o2 = orc.linear_attn(q, 4.0 * k, v, eps=0.0)
@@ -613,7 +619,7 @@ def test_rope_fused_pins():
     rp, ci = orc.mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
     lam, s = wlmod.make_scales(wl)
     sel = wlmod.sample_rows(wl, 64, seed=3)
-    rope = wlmod.rope_table(wl.grid, wl.d)
+    rope = orc.rope3d_table_vectorized(wl.grid, wl.d)
     # zero angles: Algorithm 1 as before
     ident = _angles_table(np.zeros((wl.N, wl.d // 2)))
     a = orc.salad_fused_rope(q, k, v, ident, wl.Bq, wl.Bk, rp, ci, wl.Hm, lam, s, sel=sel)
@@ -656,11 +662,11 @@ def test_rope3d_table_pins():
     # the first pair of every axis turns by one radian per position (frequency base**0 = 1)
     np.testing.assert_allclose(r[n(2, 3, 4), [0, p_t, p_t + p_hw], 0], np.cos([2.0, 3.0, 4.0]), atol=5e-4)
     np.testing.assert_allclose(r[n(2, 3, 4), [0, p_t, p_t + p_hw], 1], np.sin([2.0, 3.0, 4.0]), atol=5e-4)
-    # rows on request, and the vectorised input generator the tests feed to both sides is the same table
+    # rows on request, and the vectorised form the full-size tests use is the same table
     sel = [0, 7, 33, N - 1]
     assert np.array_equal(orc.rope3d_table(grid, d, tokens=sel).view(np.uint16), r16[sel].view(np.uint16))
-    assert np.array_equal(wlmod.rope_table(grid, d).view(np.uint16), r16.view(np.uint16))
+    assert np.array_equal(orc.rope3d_table_vectorized(grid, d).view(np.uint16), r16.view(np.uint16))
     big = wlmod.C2.grid
     tok = np.random.default_rng(3).integers(0, wlmod.C2.N, size=200)
-    assert np.array_equal(wlmod.rope_table(big, 128)[tok].view(np.uint16),
+    assert np.array_equal(orc.rope3d_table_vectorized(big, 128)[tok].view(np.uint16),
                           orc.rope3d_table(big, 128, tokens=tok).view(np.uint16))
