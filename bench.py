@@ -11,7 +11,9 @@ built once before the timed region (it is a per-model constant); its build time 
 separately.  `value` is kept-block TFLOP/s over all ranks (4 * valid_q * valid_k * d flops
 per kept block, nothing else counted).  With N > 1 every rank runs the full layer on its own
 tensors (heads and batch items are independent: no collective on the data path) and the
-time is the maximum over ranks: weak scaling.
+time is the maximum over ranks: weak scaling.  `--shard heads` splits ONE layer over the ranks
+by contiguous head ranges instead (strong scaling, still no collective).  Started as plain
+`python bench.py --gpus N` (no launcher in the environment) the script starts the N ranks itself.
 
 `--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same
 workload on the host cores (rank 0 only).
@@ -19,8 +21,11 @@ workload on the host cores (rank 0 only).
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -44,6 +49,41 @@ def load_peaks():
         return {"source": "measured", "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "hbm_gbs": p["hbm_gbs"]}
     return {"source": "fallback", "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def kernel_source_hash():
+    """sha256 over the sources of the attention kernel: a DRAM-traffic figure captured under ncu is only
+    quoted while the kernel it was captured from is the one that runs."""
+    h = hashlib.sha256()
+    for name in ("fused_kernel.cuh", "ptx.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2601_16515_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic(workload):
+    """DRAM bytes per launch of the attention kernel from the committed ncu capture of this workload, or
+    None when there is none or the kernel has changed since.  Table: lines `workload bytes source-hash`."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None, "no capture"
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 3 and not line.startswith("#") and f[0] == workload:
+            if f[2] == kernel_source_hash():
+                return float(f[1]), "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch"
+            return None, "the kernel source has changed since the ncu capture"
+    return None, "no capture of this workload"
+
+
+def self_launch(args):
+    """`python bench.py --gpus N` without a launcher: start N ranks (one per GPU) through torch's launcher
+    and pass the command line on.  Returns the exit code."""
+    with socket.socket() as sck:
+        sck.bind(("127.0.0.1", 0))
+        port = sck.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def kept_block_flops(wl, row_ptr, col_idx, Hm):
@@ -174,9 +214,15 @@ def main():
     ap.add_argument("--workload", default="wan1.3b-90", choices=sorted(wlmod.ALL))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the dense-run and per-branch timings")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: every rank its own layer (weak scaling) or one layer split by heads (strong)")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the extra back-to-back loop that shows the power-capped behaviour (0: skip)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "salad" else args.warmup
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "salad":
+        raise SystemExit(self_launch(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -199,10 +245,21 @@ def main():
     T, Hs, Ws = wl.grid
     K, W = args.steps, args.warmup
 
-    # ---------------- inputs (seeded, synthetic; every rank its own replica of the layer)
-    q_h, k_h, v_h = (t.pin_memory() for t in wlmod.make_qkv(wl))
+    # ---------------- inputs (seeded, synthetic; every rank its own replica of the layer, or with
+    # --shard heads its contiguous range of the heads of one layer)
+    shard_heads = args.shard == "heads" and world > 1
+    full_wl = wl
+    h0, h1 = dist_util.head_range(wl.H, world, rank) if shard_heads else (0, wl.H)
+    if shard_heads:
+        if h1 == h0:
+            raise SystemExit("--shard heads needs at least one head per rank")
+        wl = wlmod.replace(wl, H=h1 - h0)
+        if len(wl.windows) == full_wl.H and full_wl.H > 1:           # one window per head: this rank's
+            wl = wlmod.replace(wl, windows=wl.windows[h0:h1])
+    q_h, k_h, v_h = (t.pin_memory() for t in wlmod.make_qkv(full_wl, heads=list(range(h0, h1))))
     q, k, v = (t.to(dev, non_blocking=True) for t in (q_h, k_h, v_h))
-    lam, s = wlmod.make_scales(wl)
+    lam, s = wlmod.make_scales(full_wl)
+    lam = lam[h0:h1].copy()
     lam_d, s_d = torch.from_numpy(lam).to(dev), torch.from_numpy(s).to(dev)
     out = torch.empty_like(q)
     out_h = torch.empty(q_h.shape, dtype=q_h.dtype).pin_memory()
@@ -211,7 +268,8 @@ def main():
 
     # ---------------- static mask, built once (step a1), timed on its own
     if wl.irregular:
-        rp_np, ci_np = wlmod.irregular_csr(wl)
+        rp_np, ci_np = wlmod.irregular_csr(full_wl)
+        rp_np, ci_np = dist_util.slice_head_lists(rp_np, ci_np, wl.nQb, h0, h1)     # this rank's heads
         rp, ci, Hm = torch.from_numpy(rp_np).to(dev), torch.from_numpy(ci_np).to(dev), wl.H
         mask_ms = None
     else:
@@ -273,10 +331,40 @@ def main():
     head_ms_per_step = t_start.elapsed_time(t_mid) / K_head
     state_ms = float(np.mean([g[0].elapsed_time(g[1]) for g in evs]))
     attn_ms = float(np.mean([g[2].elapsed_time(g[3]) for g in evs]))
-    # every rank did `flops` of work; the job took the slowest rank's time (weak scaling)
-    flops_per_s, total_ms_max = dist_util.aggregate_throughput(flops * K, total_ms, dev)
+    # replicas: every rank did `flops` of work (weak scaling); head shards: the ranks' shares add up to one
+    # layer (strong scaling).  Either way the job took the slowest rank's time.
+    if shard_heads:
+        total_flops = dist_util.sum_over_ranks(flops, dev)
+        total_ms_max = dist_util.max_over_ranks(total_ms, dev)
+        flops_per_s = total_flops * K / (total_ms_max * 1e-3)
+    else:
+        flops_per_s, total_ms_max = dist_util.aggregate_throughput(flops * K, total_ms, dev)
     ms_per_step = total_ms_max / K
     value = flops_per_s / 1e12
+
+    # ---------------- sustained: the same call back to back for seconds, into the power cap
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(K, int(args.sustained_seconds * 1.1 / (total_ms / K * 1e-3)))
+        sus_sampler = ClockSampler(physical_gpu_index(local_rank))
+        barrier()
+        sus_sampler.start()
+        t_start.record()
+        for _ in range(n_sus):
+            step()
+        t_stop.record()
+        sus_sampler.sample()
+        barrier()
+        sus_sampler.stop_flag.set()
+        sus_ms = dist_util.max_over_ranks(t_start.elapsed_time(t_stop), dev)
+        sus_tflops = flops / (sus_ms / n_sus * 1e-3) / 1e12           # per GPU
+        clk = sus_sampler.result()
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "tflops_per_gpu": sus_tflops, "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"],
+                     "peak": peaks.get("bf16_tflops_sustained"),
+                     "frac_of_measured_bf16_sustained": (sus_tflops / peaks["bf16_tflops_sustained"]
+                                                         if peaks.get("bf16_tflops_sustained") else None),
+                     "frac_of_measured_bf16_burst": sus_tflops / peaks["bf16_tflops"]}
 
     # ---------------- end to end: host buffers in, host buffer out, every step.
     # Every step copies its Q, K, V from pinned host memory and its O back.  The copies of neighbouring
@@ -340,11 +428,12 @@ def main():
     if int(status.item()) != 0:
         raise SystemExit("a kernel reported an expired wait; no number is valid")
     tensor_bytes = q_h.numel() * q_h.element_size()
-    e2e = {"value": flops * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+    job_flops = dist_util.sum_over_ranks(flops, dev) if shard_heads else flops * world
+    e2e = {"value": job_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": 3 * tensor_bytes, "d2h_bytes_per_step": tensor_bytes,
            "how": "copies of neighbouring steps overlap compute (two buffer sets, three streams)",
            "serial_ms_per_step": e2e_serial_ms,
-           "serial_value": flops * world / (e2e_serial_ms * 1e-3) / 1e12}
+           "serial_value": job_flops / (e2e_serial_ms * 1e-3) / 1e12}
     del bufs, outs_h, ws2
 
     # ---------------- extras (rank 0): per-branch calls and the 0 %-sparsity run of the same kernel
@@ -366,11 +455,13 @@ def main():
         extras["linear_only_ms"] = timed(lambda: salad.salad_linear_attn_fwd(q, k, v, out=out, workspace=ws), 20)
         # the whole linear branch as one call: K, V read (state), Q read and O written (apply)
         lin_bytes = 4 * q_h.numel() * q_h.element_size()
-        extras["linear_branch"] = {"ms": extras["linear_only_ms"], "algorithmic_bytes": lin_bytes,
-                                   "achieved_gbs": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9,
-                                   "peak_gbs": peaks["hbm_gbs"],
-                                   "frac": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                   "frac_of_nominal_8tbs": lin_bytes / (extras["linear_only_ms"] * 1e-3) / 1e9 / 8000.0}
+        def hbm_record(kernel, ms, nbytes):
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            return {"kernel": kernel, "bound": "hbm", "ms": ms, "algorithmic_bytes": nbytes, "achieved": gbs,
+                    "unit": "GB/s", "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+                    "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8tbs": gbs / 8000.0}
+        extras["linear_branch"] = hbm_record("salad_linear_attn_fwd: state, finalize and apply kernels (K, V, Q read, O written)",
+                                             extras["linear_only_ms"], lin_bytes)
         drp, dci = wlmod.dense_csr(wl.nQb, wl.nKb, 1)
         drp_d, dci_d = torch.from_numpy(drp).to(dev), torch.from_numpy(dci).to(dev)
         dense_ms = timed(lambda: salad.salad_fused_fwd(q, k, v, drp_d, dci_d, 1, lam_d, s_d, Bq=wl.Bq, Bk=wl.Bk,
@@ -391,11 +482,8 @@ def main():
         salad.salad_set_profile_events(None)
         torch.cuda.synchronize(dev)
         lin_state_ms = float(np.mean([g[0].elapsed_time(g[1]) for g in lin_evs[3:]]))
-        extras["linear_state"] = {"ms": lin_state_ms, "algorithmic_bytes": kv_bytes,
-                                  "achieved_gbs": kv_bytes / (lin_state_ms * 1e-3) / 1e9,
-                                  "peak_gbs": peaks["hbm_gbs"],
-                                  "frac": kv_bytes / (lin_state_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                  "frac_of_nominal_8tbs": kv_bytes / (lin_state_ms * 1e-3) / 1e9 / 8000.0}
+        extras["linear_state"] = hbm_record("salad_linear_state_kernel + salad_linear_finalize_kernel (K, V read once)",
+                                            lin_state_ms, kv_bytes)
 
         # dynamic-scale producer (Alg. 1 Level 2) on hidden states of the DiT this workload comes from:
         # a CFG pair of [N, D = H*d] token matrices (larger than L2), read once
@@ -405,9 +493,7 @@ def main():
         dyn_ws = torch.empty(salad.DYN_SCALE_WS_BYTES, dtype=torch.uint8, device=dev)
         dyn_ms = timed(lambda: salad.salad_dynamic_scale(xt, w_dyn, 0.0, out=s_out, workspace=dyn_ws), 20)
         x_bytes = xt.numel() * 2
-        extras["dynamic_scale"] = {"ms": dyn_ms, "algorithmic_bytes": x_bytes,
-                                   "achieved_gbs": x_bytes / (dyn_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
-                                   "frac": x_bytes / (dyn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        extras["dynamic_scale"] = hbm_record("dynamic_scale_partial_kernel + finalize (X_t read once)", dyn_ms, x_bytes)
         del xt
         # full D x D projection of the linear branch + residual sum (Alg. 1 level 1): a tensor-core GEMM
         Dm = wl.H * wl.d
@@ -423,9 +509,7 @@ def main():
         flags = [1] * wl.H
         perm_out = torch.empty_like(q)
         perm_ms = timed(lambda: salad.salad_permute_tokens(q, wl.grid, flags, out=perm_out), 20)
-        extras["permute_tokens"] = {"ms": perm_ms, "algorithmic_bytes": 2 * tensor_bytes,
-                                    "achieved_gbs": 2 * tensor_bytes / (perm_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
-                                    "frac": 2 * tensor_bytes / (perm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        extras["permute_tokens"] = hbm_record("permute_tokens_kernel (one read, one write)", perm_ms, 2 * tensor_bytes)
         del perm_out
         # Top-K mask producer (App. A.1 steps 1-2) at this shape, k chosen for the same 90 % sparsity:
         # block means read Q and K once (the HBM-bound part), then scores and selection
@@ -436,9 +520,8 @@ def main():
         tk_ci = torch.empty(wl.B * wl.H * wl.nQb * topk, dtype=torch.int32, device=dev)
         tk_ms = timed(lambda: salad.salad_topk_mask_build(q, k, topk, Bq=wl.Bq, Bk=wl.Bk, row_ptr=tk_rp,
                                                           col_idx=tk_ci, workspace=tk_ws), 20)
-        extras["topk_mask"] = {"k": topk, "ms": tk_ms, "algorithmic_bytes": 2 * tensor_bytes,
-                               "achieved_gbs": 2 * tensor_bytes / (tk_ms * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
-                               "frac": 2 * tensor_bytes / (tk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        extras["topk_mask"] = hbm_record("salad_topk_mask_build (Q, K read once)", tk_ms, 2 * tensor_bytes)
+        extras["topk_mask"]["k"] = topk
         tk_fused_ms = timed(lambda: salad.salad_fused_fwd(q, k, v, tk_rp, tk_ci, wl.B * wl.H, lam_d, s_d, Bq=wl.Bq,
                                                           Bk=wl.Bk, out=out, workspace=ws), 10)
         extras["topk_mask"]["fused_on_topk_lists_ms"] = tk_fused_ms
@@ -460,20 +543,26 @@ def main():
     if rank == 0:
         achieved = flops / (attn_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops"]
+        traffic, traffic_source = captured_traffic(full_wl.name if not shard_heads else "")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms_per_step, "ms_per_call": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": ms_per_step, "ms_per_call": ms_per_step, "higher_is_better": True,
+            "scaling": "strong" if shard_heads else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "d": wl.d, "grid": list(wl.grid),
                        "blocks": f"{wl.Bq}x{wl.Bk}", "windows": [list(w) for w in wl.windows],
                        "block_sparsity": sparsity, "kept_blocks": nnz_total,
                        "kept_block_tflop_per_call": flops / 1e12,
                        "l2": "inputs (Q,K,V,O = %.0f MB) larger than the 126 MB L2; no flush" % (4 * tensor_bytes / 1e6),
-                       "parallelism": "replicas" if world > 1 else "single"},
+                       "parallelism": ("heads" if shard_heads else "replicas") if world > 1 else "single",
+                       "heads_of_rank_0": [h0, h1]},
             "pct_of_measured_bf16_peak": 100.0 * value / world / peak,
             "pct_of_nominal_bf16_peak": 100.0 * value / world / 2250.0,
-            "pct_of_measured_bf16_sustained": (100.0 * value / world / peaks["bf16_tflops_sustained"]
-                                               if peaks.get("bf16_tflops_sustained") else None),
+            # the seconds-long loop against the seconds-long GEMM figure (a short region runs at the burst clock
+            # and belongs beside the burst peak above)
+            "pct_of_measured_bf16_sustained": (100.0 * sustained["frac_of_measured_bf16_sustained"]
+                                               if sustained and sustained["frac_of_measured_bf16_sustained"] else None),
+            "sustained": sustained,
             "first_steps": {"steps": K_head, "ms_per_step": head_ms_per_step,
                             "value": flops / (head_ms_per_step * 1e-3) / 1e12,
                             "note": "the first calls of the timed region on this rank; a long region runs into the "
@@ -481,10 +570,10 @@ def main():
             "mask_build_ms": mask_ms,
             "roofline": {"kernel": "salad_fused_kernel<128>", "bound": "tensor", "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "peak_source": peaks["source"] + " (burst)",
-                         # DRAM bytes of one launch from the ncu capture of this workload
-                         # (profiles/salad_fused_kernel_wan1.3b-90.md); algorithmic bytes are 402.6 MB
-                         "traffic": 393.7e6 if wl.name == "wan1.3b-90" else None,
-                         "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, see profiles/",
+                         # DRAM bytes of one launch from the committed ncu capture of this workload, quoted only
+                         # while the kernel source is the captured one; algorithmic bytes: Q, K, V read, O written once
+                         "traffic": traffic, "traffic_source": traffic_source,
+                         "algorithmic_bytes": 4 * tensor_bytes,
                          "kernel_ms": attn_ms, "state_kernels_ms": state_ms,
                          "timed_how": "CUDA events around the launch, %d steps directly before the timed region" % KP},
             "cpu_baseline": cpu_baseline,

@@ -30,8 +30,18 @@
  *     before anything is launched.  There is no CPU fallback: without a usable CUDA device
  *     the compute entry points return SALAD_ERR_CUDA.
  *   - d_status (optional, device int32): set to 0 by a successful launch and to a non-zero
- *     code by a kernel whose bounded internal wait expired (the kernel then returns early
- *     instead of hanging; outputs are undefined).  Read it after synchronising the stream.
+ *     code by a kernel whose bounded internal wait expired (SALAD_ERR_TIMEOUT; the kernel then
+ *     returns early instead of hanging) or by the mask checks (SALAD_ERR_BAD_MASK, below); the
+ *     remaining kernels of the call then return at once and the outputs are undefined.  Read it
+ *     after synchronising the stream.
+ *   - Mask checks.  The lists are device data, so the host cannot check them before the launch.
+ *     Every call with a sparse branch checks, in its first kernel, that the row offsets are
+ *     non-negative and non-decreasing (it reads them anyway).  The full contract (offsets
+ *     start at 0 and end within col_idx, block ids strictly ascending and in range) is checked
+ *     by salad_csr_validate, on request; salad_set_mask_validation makes the attention entry
+ *     points run it first.  Without that opt-in, offsets that point past the end of col_idx
+ *     make the attention kernel read outside the caller's array.
+ *   - SALAD_LOG=1 in the environment prints one line per kernel launch on stderr.
  *   - Supported shapes: d in {64, 128}; Bq in {64, 128}; Bk = 64; softmax_scale > 0.
  */
 #ifndef SALAD_H_
@@ -51,6 +61,7 @@ extern "C" {
 #define SALAD_ERR_CAPACITY (-4)    /* col_idx capacity smaller than nnz (nnz still returned) */
 #define SALAD_ERR_CUDA (-5)        /* a CUDA runtime/driver call or a launch failed          */
 #define SALAD_ERR_TIMEOUT (-6)     /* value written to d_status by a kernel that gave up     */
+#define SALAD_ERR_BAD_MASK (-7)    /* value written to d_status: the CSR lists break the contract */
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* salad_status_string(int status);
@@ -72,12 +83,34 @@ size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk);
  *   d_col_idx      device int32 [col_capacity], written ascending per row; may be NULL with
  *                  col_capacity 0 to obtain only row_ptr and nnz.
  *   h_nnz          HOST int64, written with the total number of kept blocks (optional).
- * Synchronises `stream`.  Returns SALAD_ERR_CAPACITY (row_ptr and *h_nnz valid, col_idx
+ * Synchronises `stream` (once to return nnz, once more after the fill when d_col_idx is given; the
+ * count pass runs in both of the usual two calls, "size, then fill": the mask is built once per
+ * model, so this costs a fraction of a millisecond in total).  Returns SALAD_ERR_CAPACITY (row_ptr and *h_nnz valid, col_idx
  * untouched) if col_capacity < nnz and d_col_idx != NULL.
  */
 int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm, const int32_t* h_windows,
                      int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
                      int64_t* h_nnz, void* stream);
+
+/*
+ * salad_csr_validate -- checks block lists against the contract above (the mask M of Eq. 2 in its
+ * block-granular CSR form):  row_ptr[0] == 0;  row_ptr non-decreasing;  row_ptr[rows] <=
+ * col_capacity;  inside every row the block ids strictly ascending (sorted, unique) and in [0, nKb).
+ *   row_ptr        device int32 [rows + 1];   col_idx  device int32 [col_capacity] (may be NULL
+ *                  with capacity 0);   rows = Hm * nQb;   nKb = ceil(N / Bk).
+ *   d_status       device int32, required: 0 if the lists are valid, SALAD_ERR_BAD_MASK if not.
+ * Reads nothing outside row_ptr[0..rows] and col_idx[0..col_capacity), whatever the lists hold, so
+ * it is safe on corrupted input.  Asynchronous on `stream` (a memset and one small kernel).
+ *
+ * salad_set_mask_validation -- col_capacity > 0: every later call of salad_sparse_attn_fwd and the
+ * salad_fused_* entry points made by this host thread first runs the check above on its lists, with
+ * col_idx holding col_capacity entries; a failure is reported as SALAD_ERR_BAD_MASK in d_status,
+ * and the attention kernels of that call do nothing.  0 switches it off (the default).  A debugging
+ * aid: it adds a memset and a kernel to every call.
+ */
+int salad_csr_validate(const int32_t* row_ptr, const int32_t* col_idx, int64_t col_capacity,
+                       int64_t rows, int nKb, int32_t* d_status, void* stream);
+int salad_set_mask_validation(int64_t col_capacity);
 
 /*
  * salad_sparse_attn_fwd -- block-sparse softmax attention, Eq. 2:
@@ -100,7 +133,8 @@ int salad_sparse_attn_fwd(const void* q, const void* k, const void* v, void* o, 
  *   o_l            bf16 [B,H,N,d], written.
  *   kv_out         optional fp32 [B,H,d,d] (row = key channel, column = value channel).
  *   z_out          optional fp32 [B,H,d].
- *   eps            >= 0; only defines the 0/0 case (a row with ReLU(Q_n) = 0 gives 0).
+ *   eps            >= 0; only defines the 0/0 case: a row with ReLU(Q_n) = 0 gives 0, also
+ *                  with eps = 0 (the quotient 0/0 is taken as 0, never NaN).
  */
 int salad_linear_attn_fwd(const void* q, const void* k, const void* v, void* o_l,
                           float* kv_out, float* z_out, int B, int H, int N, int d, float eps,
@@ -283,6 +317,8 @@ int salad_selftest_bounded_wait(int32_t* d_status, unsigned long long* d_waited_
  *   array keeps the previous call's contents; the call itself re-initialises everything it
  *   reads (the status word is cleared, every partial it sums is rewritten first).
  *   No cudaMalloc, cudaFree or other allocating routine is called.
+ *   The looked-up address (like the library's other once-per-device set-up) is kept for the life of
+ *   the process: after cudaDeviceReset on a device, do not call the library on that device again.
  */
 #define SALAD_NOALLOC_MAX_HEADS 16
 #define SALAD_NOALLOC_SCRATCH_BYTES 4759808

@@ -17,7 +17,7 @@ LIB = os.path.join(HERE, "libsalad.so")
 SOURCES = ["salad_api.cu"]
 HEADERS = ["ptx.cuh", "tmap.cuh", "mask_kernels.cuh", "linear_state_kernel.cuh", "fused_kernel.cuh",
            "dynamic_scale_kernel.cuh", "linear_apply_kernel.cuh", "topk_mask_kernels.cuh", "permute_kernel.cuh", "proj_gemm_kernel.cuh",
-           "rope_table_kernel.cuh",
+           "rope_table_kernel.cuh", "selftest_kernel.cuh", "work_order_kernel.cuh",
            os.path.join("..", "..", "include", "salad.h")]
 
 
@@ -27,9 +27,6 @@ def nvcc_command(out: str, verbose: bool = False):
            "-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
-    extra = os.environ.get("SALAD_NVCC_FLAGS")       # e.g. -DSALAD_TRACE for the cycle trace points
-    if extra:
-        cmd[1:1] = extra.split()
     return cmd
 
 

@@ -41,14 +41,6 @@
 
 namespace salad {
 
-#ifdef SALAD_TRACE
-#define TRACE(role, step, k) do { if (blockIdx.x == 700 && (step) < 64) reinterpret_cast<long long*>(p.lse)[((role) * 64 + (step)) * 8 + (k)] = clock64(); } while (0)
-#define TRACE_CTA(k) do { reinterpret_cast<long long*>(p.lse)[4096 + blockIdx.x * 8 + (k)] = (long long)global_timer_ns(); } while (0)
-#else
-#define TRACE(role, step, k) do {} while (0)
-#define TRACE_CTA(k) do {} while (0)
-#endif
-
 enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
 
 struct FusedParams {
@@ -143,8 +135,9 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     // ------------------------------------------------------------------ set-up
     if (tid == 0) {
-        TRACE_CTA(0);
-        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+        // 2: an earlier kernel of this call has already reported a failure (a rejected mask, an expired wait):
+        // this CTA starts nothing and reports nothing; 1 (set by a bounded wait of this CTA): a time-out
+        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 2 : 0;
         mbar_init(smem_u32(&bars.q_full), 1);
         mbar_init(smem_u32(&bars.st_full), 1);
         mbar_init(smem_u32(&bars.o_final), 1);
@@ -179,10 +172,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_slot;
     volatile int* abortp = &abort_flag;
-    if (tid == 0) TRACE_CTA(1);
     const int len = le - ls;
+    const bool inherited_abort = abort_flag != 0;      // uniform: read after the barrier above, before any wait
 
-    if (abort_flag == 0) {
+    if (!inherited_abort) {
     if (warp == 0) {
         // ============================================================== TMA producer: Q, the K ring, the state tile
         bool ok = true;
@@ -212,10 +205,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // From here on the linear state is needed: wait for the kernels that make it (whole warp: the
             // other lanes fetch the normaliser Z of this head for the softmax warps meanwhile).
             __syncwarp();
-            if (lane == 0) TRACE_CTA(2);
             grid_dependency_wait();
-            if (lane == 0) TRACE_CTA(3);
-            if (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) *abortp = 1;     // the state kernel gave up
+            if (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0 && *abortp == 0) *abortp = 2;   // the state kernel gave up (and said so)
             for (int a = lane; a < D; a += 32) z_s[a] = __ldcg(p.z + size_t(bh) * D + a);
             mbar_arrive(smem_u32(&bars.z_full));
             if (lane == 0 && ok) {
@@ -264,7 +255,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 // score buffer t & 1 held P of block t - 2: its P V product must have read it
                 if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.pv_done[t & 1]), ((t >> 1) - 1) & 1, abortp);
                 if (!ok) break;
-                TRACE(2, t, 0);
                 tc_fence_after_sync();
                 const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
@@ -274,7 +264,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                                 kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
                 tc_commit(smem_u32(&bars.s_full[t & 1]));
                 tc_commit(smem_u32(&bars.k_empty[s]));
-                TRACE(2, t, 3);
             }
         }
     } else if (warp == 3) {
@@ -291,7 +280,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ok = mbar_wait(smem_u32(&bars.v_full[s]), (t / C::NV) & 1, abortp);
                 if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[t & 1]), (t >> 1) & 1, abortp);
                 if (!ok) break;
-                TRACE(2, t, 1);
                 tc_fence_after_sync();
                 const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
                 const uint32_t p_col = tmem + C::COL_SP + (t & 1) * C::SP_STRIDE;
@@ -302,7 +290,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tc_commit(smem_u32(&bars.v_empty[s]));
                 tc_commit(smem_u32(&bars.pv_done[t & 1]));
                 if (t + 1 == len) tc_commit(smem_u32(&bars.o_final));
-                TRACE(2, t, 2);
             }
             if (ok && linear) {
                 ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
@@ -350,18 +337,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
         const bool ragged_keys = (p.N % C::BK) != 0;
         for (int t = 0; t < len && ok; ++t) {
-            if (ra == 0 && q4 == 0) TRACE(0, t, 0);
             // only the last key block can be short; its id is needed only then
             const int col = ragged_keys ? __ldg(p.col_idx + ls + t) : 0;
             ok = wait_uniform(&bars.s_full[t & 1], (t >> 1) & 1);
             if (!ok) break;
-            if (ra == 0 && q4 == 0) TRACE(0, t, 1);
             tc_fence_after_sync();
             // x[4n], x[4n+1] = S(row a, keys 8n + 2 q4, + 1);  x[4n+2], x[4n+3] = the same keys of row b
             uint32_t xr[32];
             tmem_ld_16x256b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, xr);
             tmem_wait_ld();
-            if (ra == 0 && q4 == 0) TRACE(0, t, 2);
             float* x = reinterpret_cast<float*>(xr);
             const int valid = p.N - col * C::BK;              // keys of this block that exist
             if (ragged_keys && valid < C::BK) {
@@ -412,7 +396,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 tmem_wait_st();
             }
-            if (ra == 0 && q4 == 0) TRACE(0, t, 3);
             // P = exp2(x * scale - m), packed bf16: word 2n = row a, keys (8n + 2 q4, + 1) = packed
             // column 4n + q4 of the P tile, word 2n + 1 the same of row b -- the 16x128b layout
             uint32_t pk[16];
@@ -435,14 +418,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 unpack_f32x2(acc_a, s0, s1); l_a += s0 + s1;
                 unpack_f32x2(acc_b, s0, s1); l_b += s0 + s1;
             }
-            if (ra == 0 && q4 == 0) TRACE(0, t, 4);
             // P goes over the scores it was computed from (this warp's own lanes, already in registers)
             tmem_st_16x128b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.p_ready[t & 1]));   // one arrival per warp
-            if (ra == 0 && q4 == 0) TRACE(0, t, 5);
         }
         float coef_a = 0.f, coef_b = 0.f;
         if (ok && linear) {
@@ -502,8 +483,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 float c_scale = 1.f;
                 if (p.static_scale) c_scale *= __ldg(p.static_scale + h);
                 if (p.dyn_scale) c_scale *= __ldg(p.dyn_scale + b);
-                coef_a = c_scale / (den_a + p.eps);
-                coef_b = c_scale / (den_b + p.eps);
+                // a row with ReLU(Q_n) = 0 and eps = 0 is 0/0: defined as 0 (the numerator is 0 as well)
+                const float da = den_a + p.eps, db = den_b + p.eps;
+                coef_a = da > 0.f ? c_scale / da : 0.f;
+                coef_b = db > 0.f ? c_scale / db : 0.f;
                 fence_proxy_async_smem();
                 mbar_arrive(smem_u32(&bars.lin_ready));
             }
@@ -557,7 +540,6 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 // writes are complete, like all of the kernel's, when the grid is
                 tma_store_wait_read_all();
             }
-#ifndef SALAD_TRACE
             if (p.lse != nullptr && q4 == 0) {
 #pragma unroll
                 for (int e2 = 0; e2 < 2; ++e2) {
@@ -568,25 +550,24 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             (len > 0) ? ((e2 ? m_b : m_a) + log2f(e2 ? lt_b : lt_a)) * 0.6931471805599453f : -INFINITY;
                 }
             }
-#endif
         }
     }
-    }  // abort_flag == 0
+    }  // !inherited_abort
 
     // ------------------------------------------------------------------ tear-down
     tc_fence_before_sync();
     __syncthreads();
-    if (abort_flag != 0) {
-        // a bounded wait expired somewhere: report, give copies in flight time to land, leave
-        if (tid == 0) {
-            atomicExch(p.ws_status, 1);
-            if (p.user_status) atomicExch(p.user_status, -6);
+    if (abort_flag != 0 && !inherited_abort) {
+        // a bounded wait expired somewhere (1: in this CTA, reported here; 2: in the state kernels, which
+        // reported it themselves): give copies in flight time to land, leave
+        if (tid == 0 && abort_flag == 1) {
+            atomicExch(p.ws_status, SALAD_ERR_TIMEOUT);
+            if (p.user_status) atomicExch(p.user_status, SALAD_ERR_TIMEOUT);
         }
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
         __syncthreads();
     }
-    if (tid == 0) TRACE_CTA(5);
     if (warp == 2) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

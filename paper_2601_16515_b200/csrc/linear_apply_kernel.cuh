@@ -85,7 +85,7 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     grid_dependency_wait();
     grid_launch_dependents();
     if (tid == 0) {
-        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+        abort_flag = (*reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 2 : 0;    // 2: reported by an earlier kernel
         for (int s = 0; s < C::NQ; ++s) {
             mbar_init(smem_u32(&bars.q_full[s]), 1);
             mbar_init(smem_u32(&bars.q_empty[s]), 1);
@@ -225,7 +225,8 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                     *ptr = v;
                 }
             }
-            coef_s[j % C::NCOEF][row] = c_scale / (den + p.eps);
+            // a row with ReLU(Q_n) = 0 and eps = 0 is 0/0: defined as 0 (the numerator is 0 as well)
+            coef_s[j % C::NCOEF][row] = (den + p.eps > 0.f) ? c_scale / (den + p.eps) : 0.f;
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bars.relu_done[s]));
         }
@@ -291,9 +292,9 @@ salad_linear_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     tc_fence_before_sync();
     __syncthreads();
     if (abort_flag != 0) {
-        if (tid == 0) {
-            atomicExch(p.ws_status, 1);
-            if (p.user_status) atomicExch(p.user_status, -6);
+        if (tid == 0 && abort_flag == 1) {            // a bounded wait of this CTA ran out
+            atomicExch(p.ws_status, SALAD_ERR_TIMEOUT);
+            if (p.user_status) atomicExch(p.user_status, SALAD_ERR_TIMEOUT);
         }
         const uint64_t ts = global_timer_ns();
         while (global_timer_ns() - ts < 200000ull) { __nanosleep(1000); }

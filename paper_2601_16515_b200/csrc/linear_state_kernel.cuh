@@ -127,9 +127,15 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         reinterpret_cast<uint32_t*>(smem + C::OFF_ONES)[i] = 0x3F803F80u;
     fence_proxy_async_smem();
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_slot), C::TMEM_COLS); tmem_relinquish(); }
+    // Invariant the attention kernel of a fused call relies on: this kernel releases its dependents only AFTER
+    // its own dependency wait (here, and in the early exit of a dropped batch item above).  The attention
+    // kernel reads the launch order and the status word, both written by the first kernel of the call,
+    // without a wait of its own; it can be placed only once every CTA of the finalize kernel has started,
+    // which needs every CTA of this kernel to have got here, i.e. past the wait for that first kernel.
     grid_dependency_wait();            // the status word is cleared by the kernel before
     grid_launch_dependents();
-    if (tid == 0) abort_flag = (!p.clear_status && *reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 1 : 0;
+    // 2: the first kernel of the call has reported a failure (a rejected mask): do nothing, report nothing
+    if (tid == 0) abort_flag = (!p.clear_status && *reinterpret_cast<volatile int32_t*>(p.ws_status) != 0) ? 2 : 0;
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -272,9 +278,9 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     tc_fence_before_sync();
     __syncthreads();
     if (abort_flag != 0) {
-        if (tid == 0) {
-            atomicExch(p.ws_status, 1);
-            if (p.user_status) atomicExch(p.user_status, -6);
+        if (tid == 0 && abort_flag == 1) {            // a bounded wait of this CTA ran out
+            atomicExch(p.ws_status, SALAD_ERR_TIMEOUT);
+            if (p.user_status) atomicExch(p.user_status, SALAD_ERR_TIMEOUT);
         }
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }

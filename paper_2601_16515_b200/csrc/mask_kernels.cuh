@@ -99,65 +99,4 @@ __global__ void __launch_bounds__(1024) mask_scan_kernel(int32_t* __restrict__ r
     }
 }
 
-// Diagnostic: one thread waits, with a 2 ms limit, on an mbarrier that nothing ever arrives on, and
-// reports the expiry the way the compute kernels do (status word = -6).  It exercises the bounded
-// wait and the status path without any fault: the kernel returns normally.
-__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int32_t* __restrict__ status,
-                                                                   unsigned long long* __restrict__ waited_ns) {
-    __shared__ uint64_t bar;
-    __shared__ int abort_flag;
-    if (threadIdx.x == 0) {
-        abort_flag = 0;
-        mbar_init(smem_u32(&bar), 1);
-        fence_mbar_init();
-        const uint64_t t0 = global_timer_ns();
-        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, 2000000ull);
-        if (waited_ns) *waited_ns = global_timer_ns() - t0;
-        *status = ok ? 0 : -6;
-    }
-}
-
-// Launch order of the attention kernel's work items: for every mask head, the query blocks
-// sorted by decreasing length of their kept list, so that the long items start first and the
-// short ones fill the tail.  Counting sort in shared memory; one CTA per mask head.  The order
-// among equal costs is arbitrary (it only affects scheduling).
-// It is the first kernel of a call, so it also clears the status words the later kernels test.
-__global__ void __launch_bounds__(1024) work_order_kernel(const int32_t* __restrict__ row_ptr, int nQb,
-                                                          int32_t* __restrict__ order,
-                                                          int32_t* __restrict__ ws_status,
-                                                          int32_t* __restrict__ user_status) {
-    grid_launch_dependents();         // the next kernel of the call may be placed now; it waits for this one
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        *ws_status = 0;
-        if (user_status) *user_status = 0;
-    }
-    constexpr int BINS = 2048;
-    __shared__ int hist[BINS];
-    const int hm = blockIdx.x, tid = threadIdx.x;
-    const int32_t* rp = row_ptr + size_t(hm) * nQb;
-    auto cost_of = [&](int qb) { return min(BINS - 1, rp[qb + 1] - rp[qb]); };
-    for (int i = tid; i < BINS; i += blockDim.x) hist[i] = 0;
-    __syncthreads();
-    for (int qb = tid; qb < nQb; qb += blockDim.x) atomicAdd(&hist[cost_of(qb)], 1);
-    __syncthreads();
-    // start position of every cost, largest cost first: an exclusive suffix sum over the bins,
-    // two bins per thread, Hillis-Steele over the per-thread totals
-    __shared__ int part[1024];
-    const int h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
-    part[tid] = h0 + h1;
-    __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-        const int add = (tid + off < 1024) ? part[tid + off] : 0;
-        __syncthreads();
-        part[tid] += add;
-        __syncthreads();
-    }
-    const int above = part[tid] - (h0 + h1);      // items with a cost in a higher pair of bins
-    hist[2 * tid + 1] = above;
-    hist[2 * tid] = above + h1;
-    __syncthreads();
-    for (int qb = tid; qb < nQb; qb += blockDim.x)
-        order[size_t(hm) * nQb + atomicAdd(&hist[cost_of(qb)], 1)] = qb;
-}
-
 }  // namespace salad

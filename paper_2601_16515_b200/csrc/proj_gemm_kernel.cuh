@@ -166,7 +166,7 @@ salad_proj_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     tc_fence_before_sync();
     __syncthreads();
     if (abort_flag != 0) {
-        if (tid == 0 && p.status) atomicExch(p.status, -6);
+        if (tid == 0 && p.status) atomicExch(p.status, SALAD_ERR_TIMEOUT);
         const uint64_t ts = global_timer_ns();
         while (global_timer_ns() - ts < 200000ull) { __nanosleep(1000); }
         __syncthreads();

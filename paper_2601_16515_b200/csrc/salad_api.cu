@@ -5,6 +5,8 @@
 
 #include <cuda_runtime.h>
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include <mutex>
 
@@ -16,8 +18,10 @@
 #include "permute_kernel.cuh"
 #include "proj_gemm_kernel.cuh"
 #include "rope_table_kernel.cuh"
+#include "selftest_kernel.cuh"
 #include "tmap.cuh"
 #include "topk_mask_kernels.cuh"
+#include "work_order_kernel.cuh"
 
 using namespace salad;
 
@@ -30,6 +34,16 @@ constexpr int kPartialSlots = 512;     // upper bound on (batch*heads) x chunks 
 constexpr int kMaxMaskHeads = 256;
 
 thread_local cudaEvent_t g_profile_events[4] = {nullptr, nullptr, nullptr, nullptr};
+// > 0: the attention entry points called by this host thread validate their lists first, col_idx holding
+// this many entries (salad_set_mask_validation)
+thread_local int64_t g_validate_capacity = 0;
+
+// SALAD_LOG=1 in the environment: one line per launch on stderr (host side only; read once).
+bool log_enabled() {
+    static const bool on = [] { const char* e = getenv("SALAD_LOG"); return e && e[0] && e[0] != '0'; }();
+    return on;
+}
+#define SALAD_LOGF(...) do { if (log_enabled()) { fprintf(stderr, "[salad] " __VA_ARGS__); fputc('\n', stderr); } } while (0)
 
 inline void record_profile(int idx, cudaStream_t st) {
     if (g_profile_events[idx]) cudaEventRecord(g_profile_events[idx], st);
@@ -257,10 +271,6 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     return check_launch();
 }
 
-#ifdef SALAD_TRACE
-float* g_trace_buffer = nullptr;
-#endif
-
 template <int D>
 int launch_fused(const Problem& P, const Workspace& w) {
     const int BH = P.B * P.H;
@@ -281,9 +291,6 @@ int launch_fused(const Problem& P, const Workspace& w) {
     fp.static_scale = P.static_scale; fp.dyn_scale = P.dyn_scale;
     fp.z = reinterpret_cast<const float*>(ws + w.off_z);
     fp.lse = P.lse;
-#ifdef SALAD_TRACE
-    if (!fp.lse) fp.lse = g_trace_buffer;      // trace builds only: time stamps go where the LSE would
-#endif
     const float sc = (P.softmax_scale > 0.f) ? P.softmax_scale : 1.0f / sqrtf(float(D));
     fp.scale_log2 = sc * 1.4426950408889634f;
     fp.eps = P.eps;
@@ -333,6 +340,23 @@ int launch_apply(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     return check_launch();
 }
 
+// Clears the status words in stream order, then checks the lists (see work_order_kernel.cuh).
+int launch_csr_validate(const int32_t* row_ptr, const int32_t* col_idx, int64_t col_capacity, int64_t rows, int nKb,
+                        int32_t* status_a, int32_t* status_b, cudaStream_t st) {
+    if (rows <= 0 || rows > (1ll << 26)) return SALAD_ERR_UNSUPPORTED;
+    if ((status_a && cudaMemsetAsync(status_a, 0, sizeof(int32_t), st) != cudaSuccess) ||
+        (status_b && cudaMemsetAsync(status_b, 0, sizeof(int32_t), st) != cudaSuccess)) {
+        cudaGetLastError();
+        return SALAD_ERR_CUDA;
+    }
+    const unsigned blocks = unsigned((rows * 32 + 255) / 256);
+    SALAD_LOGF("csr_validate_kernel grid %u block 256 (rows %lld, capacity %lld)", blocks, (long long)rows,
+               (long long)col_capacity);
+    csr_validate_kernel<<<blocks, 256, 0, st>>>(row_ptr, col_idx, (long long)col_capacity, int(rows), nKb, status_a,
+                                                status_b);
+    return check_launch();
+}
+
 int run(const Problem& P) {
     int rc = validate(P);
     if (rc != SALAD_OK) return rc;
@@ -345,9 +369,19 @@ int run(const Problem& P) {
         // first kernel of the call: longest work items first (the mask is an input of every call,
         // so is its order); it also clears the status words
         const int nQb = (P.N + P.Bq - 1) / P.Bq;
-        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb,
-                                                      reinterpret_cast<int32_t*>(ws + w.off_order),
-                                                      reinterpret_cast<int32_t*>(ws + w.off_status), P.d_status);
+        int32_t* ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
+        int clear_status = 1;
+        if (g_validate_capacity > 0) {
+            // opt-in check of the lists (salad_set_mask_validation): it owns the status words of this call
+            rc = launch_csr_validate(P.row_ptr, P.col_idx, g_validate_capacity, int64_t(P.Hm) * nQb, (P.N + 63) / 64,
+                                     ws_status, P.d_status, P.stream);
+            if (rc != SALAD_OK) return rc;
+            clear_status = 0;
+        }
+        SALAD_LOGF("work_order_kernel grid %d block 1024 (nQb %d)%s", P.Hm, nQb, clear_status ? "" : " after csr_validate_kernel");
+        work_order_kernel<<<P.Hm, 1024, 0, P.stream>>>(P.row_ptr, nQb, P.Hm,
+                                                      reinterpret_cast<int32_t*>(ws + w.off_order), ws_status,
+                                                      P.d_status, clear_status);
         if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     }
     if (P.mode & MODE_LINEAR) {
@@ -422,6 +456,7 @@ SALAD_EXPORT const char* salad_status_string(int status) {
         case SALAD_ERR_CAPACITY: return "SALAD_ERR_CAPACITY";
         case SALAD_ERR_CUDA: return "SALAD_ERR_CUDA";
         case SALAD_ERR_TIMEOUT: return "SALAD_ERR_TIMEOUT";
+        case SALAD_ERR_BAD_MASK: return "SALAD_ERR_BAD_MASK";
         default: return "SALAD_ERR_UNKNOWN";
     }
 }
@@ -430,6 +465,23 @@ SALAD_EXPORT int salad_set_profile_events(void* const* h_events) {
     for (int i = 0; i < 4; ++i)
         g_profile_events[i] = h_events ? static_cast<cudaEvent_t>(h_events[i]) : nullptr;
     return SALAD_OK;
+}
+
+SALAD_EXPORT int salad_set_mask_validation(int64_t col_capacity) {
+    if (col_capacity < 0) return SALAD_ERR_INVALID_ARG;
+    g_validate_capacity = col_capacity;
+    return SALAD_OK;
+}
+
+SALAD_EXPORT int salad_csr_validate(const int32_t* row_ptr, const int32_t* col_idx, int64_t col_capacity,
+                                    int64_t rows, int nKb, int32_t* d_status, void* stream) {
+    if (!row_ptr || !d_status || rows <= 0 || nKb <= 0 || col_capacity < 0 || (!col_idx && col_capacity > 0))
+        return SALAD_ERR_INVALID_ARG;
+    DeviceInfo dev{};
+    int rc = prepare_device(&dev);
+    if (rc != SALAD_OK) return rc;
+    return launch_csr_validate(row_ptr, col_idx, col_capacity, rows, nKb, d_status, nullptr,
+                               static_cast<cudaStream_t>(stream));
 }
 
 SALAD_EXPORT size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, int Bk) {
@@ -770,7 +822,3 @@ SALAD_EXPORT int salad_linear_attn_fwd_noalloc(const void* q, const void* k, con
     if (rc != SALAD_OK) return rc;
     return (d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
 }
-
-#ifdef SALAD_TRACE
-extern "C" __attribute__((visibility("default"))) void salad_trace_set_buffer(float* d_buf) { g_trace_buffer = d_buf; }
-#endif

@@ -23,13 +23,14 @@ SALAD_ERR_WORKSPACE = -3
 SALAD_ERR_CAPACITY = -4
 SALAD_ERR_CUDA = -5
 SALAD_ERR_TIMEOUT = -6
+SALAD_ERR_BAD_MASK = -7
 
 EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_sparse_attn_fwd", "salad_linear_attn_fwd", "salad_fused_fwd",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
            "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
            "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd",
-           "salad_rope3d_table_build")
+           "salad_rope3d_table_build", "salad_csr_validate", "salad_set_mask_validation")
 
 
 class SaladError(RuntimeError):
@@ -81,6 +82,10 @@ def _load() -> ctypes.CDLL:
     lib.salad_rope3d_table_build.argtypes = [i32, i32, i32, i32, f32, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
+    lib.salad_csr_validate.restype = i32
+    lib.salad_csr_validate.argtypes = [p, p, i64, i64, i32, p, p]
+    lib.salad_set_mask_validation.restype = i32
+    lib.salad_set_mask_validation.argtypes = [i64]
     return lib
 
 
@@ -140,6 +145,24 @@ def salad_mask_build(T: int, Hs: int, Ws: int, Bq: int, Bk: int,
         _check(_lib.salad_mask_build(T, Hs, Ws, Bq, Bk, Hm, h_win, _ptr(row_ptr), _ptr(col_idx),
                                      col_idx.numel(), ctypes.byref(nnz), _stream(stream)), "salad_mask_build")
     return row_ptr, col_idx[:nnz.value]
+
+
+def salad_csr_validate(row_ptr, col_idx, nKb: int, status=None, stream=None):
+    """Checks CSR block lists (row_ptr int32 [rows+1], col_idx int32) against the library's contract.
+    Returns the device status tensor: 0 = valid, SALAD_ERR_BAD_MASK = rejected (read it after a sync)."""
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=row_ptr.device)
+    with torch.cuda.device(row_ptr.device):
+        _check(_lib.salad_csr_validate(_ptr(row_ptr), _ptr(col_idx), col_idx.numel(), row_ptr.numel() - 1, int(nKb),
+                                       _ptr(status), _stream(stream)), "salad_csr_validate")
+    return status
+
+
+def salad_set_mask_validation(col_capacity: int = 0):
+    """col_capacity > 0: the attention calls of this host thread validate their lists first (col_idx holding
+    that many entries); 0: off."""
+    _check(_lib.salad_set_mask_validation(int(col_capacity)), "salad_set_mask_validation")
 
 
 def salad_set_profile_events(events=None):

@@ -34,7 +34,7 @@ def test_header_symbols_are_exported(lib):
 def test_status_strings(lib):
     assert lib.status_string(0) == "SALAD_OK"
     for code, name in [(-1, "INVALID_ARG"), (-2, "UNSUPPORTED"), (-3, "WORKSPACE"), (-4, "CAPACITY"),
-                       (-5, "CUDA"), (-6, "TIMEOUT")]:
+                       (-5, "CUDA"), (-6, "TIMEOUT"), (-7, "BAD_MASK")]:
         assert lib.status_string(code) == "SALAD_ERR_" + name
     assert lib.status_string(-99) == "SALAD_ERR_UNKNOWN"
 
@@ -90,6 +90,21 @@ def test_host_side_argument_checks(lib):
     assert L.salad_mask_build(4, 4, 4, 64, 64, 1000, win, fake, None, 0, None, None) == lib.SALAD_ERR_UNSUPPORTED
     neg = (ctypes.c_int32 * 3)(1, -1, 1)
     assert L.salad_mask_build(4, 4, 4, 64, 64, 1, neg, fake, None, 0, None, None) == lib.SALAD_ERR_INVALID_ARG
+
+
+def test_mask_validator_argument_checks(lib):
+    L = lib._lib
+    P = ctypes.c_void_p
+    fake = P(0x1000)
+    assert L.salad_csr_validate(None, fake, 10, 4, 8, fake, None) == lib.SALAD_ERR_INVALID_ARG     # no row_ptr
+    assert L.salad_csr_validate(fake, fake, 10, 4, 8, None, None) == lib.SALAD_ERR_INVALID_ARG     # no status word
+    assert L.salad_csr_validate(fake, None, 10, 4, 8, fake, None) == lib.SALAD_ERR_INVALID_ARG     # capacity without a list
+    assert L.salad_csr_validate(fake, fake, -1, 4, 8, fake, None) == lib.SALAD_ERR_INVALID_ARG
+    assert L.salad_csr_validate(fake, fake, 10, 0, 8, fake, None) == lib.SALAD_ERR_INVALID_ARG
+    assert L.salad_csr_validate(fake, fake, 10, 4, 0, fake, None) == lib.SALAD_ERR_INVALID_ARG
+    assert L.salad_set_mask_validation(-5) == lib.SALAD_ERR_INVALID_ARG
+    assert L.salad_set_mask_validation(100) == lib.SALAD_OK
+    assert L.salad_set_mask_validation(0) == lib.SALAD_OK
 
 
 def test_no_gpu_means_error_not_fallback(lib):

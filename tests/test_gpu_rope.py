@@ -6,7 +6,7 @@ import torch
 
 from oracle import salad_oracle as orc
 from paper_2601_16515_b200 import workloads as wlmod
-from test_gpu_parity import assert_close, dev_csr, f32, rand_qkv, random_csr, status_ok
+from test_gpu_parity import assert_close, dev_csr, f32, rand_qkv, random_csr, status_ok, stratified_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -99,7 +99,6 @@ def test_fused_rope_tiny_config_with_the_3d_table(salad):
 
 def test_fused_rope_wan13b_90_sampled(salad):
     wl = wlmod.C2
-    heads = [0, 6, 11]
     q, k, v = wlmod.make_qkv(wl)
     T, Hs, Ws = wl.grid
     lam, s = wlmod.make_scales(wl)
@@ -111,12 +110,10 @@ def test_fused_rope_wan13b_90_sampled(salad):
                                      torch.from_numpy(s).cuda(), torch.from_numpy(rope).cuda(), Bq=wl.Bq,
                                      status=status).cpu()
     status_ok(status)
-    qs, ks, vs = (f32(t[:, heads].contiguous()) for t in (q, k, v))
-    sub = wlmod.Workload("sub", wl.B, len(heads), wl.d, wl.grid, wl.Bq, wl.Bk, wl.windows, wl.seed)
-    sel = wlmod.sample_rows(sub, 1200)
-    ref = orc.salad_fused_rope(qs, ks, vs, rope, wl.Bq, wl.Bk, rp, ci, 1, lam[heads], s, sel=sel)
-    got = f32(out[:, heads].contiguous()).reshape(-1, wl.d)[sel]
-    assert_close(got, ref, "fused rope wan1.3b-90")
+    sel = stratified_rows(wl, rp, 1)                     # every head; four of them with a row in every query block
+    ref = orc.salad_fused_rope(f32(q), f32(k), f32(v), rope, wl.Bq, wl.Bk, rp, ci, 1, lam, s, sel=sel)
+    got = f32(out).reshape(-1, wl.d)[sel]
+    assert_close(got, ref, "fused rope wan1.3b-90", tight=True)
 
 
 def test_rope_argument_checks(salad):

@@ -32,10 +32,12 @@ def close(a, b, what):
 
 
 def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
+    from oracle import salad_oracle as orc
     from paper_2601_16515_b200 import salad
 
-    # first call: 2 x 4 heads of 128 channels, ragged length; second call: other sizes, other data
-    for call, (B, H, N, d) in enumerate([(2, 4, 3000, 128), (1, 3, 1100, 64)]):
+    # first call: 2 x 4 heads of 128 channels, ragged length; second call: other sizes, other data; third
+    # call: the largest problem the fixed array holds (16 heads of 128 channels)
+    for call, (B, H, N, d) in enumerate([(2, 4, 3000, 128), (1, 3, 1100, 64), (2, 8, 2000, 128)]):
         q, k, v = (bf16_randn((B, H, N, d), 10 * call + j) for j in range(3))
         ref_kv = torch.empty((B, H, d, d), dtype=torch.float32, device="cuda")
         ref_z = torch.empty((B, H, d), dtype=torch.float32, device="cuda")
@@ -45,11 +47,19 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
         kv = torch.empty_like(ref_kv)
         z = torch.empty_like(ref_z)
         status = torch.ones(1, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        allocations = torch.cuda.memory_stats()["allocation.all.allocated"]     # running count of allocations made
         got = salad.salad_linear_attn_fwd_noalloc(q, k, v, eps=1e-6, out=out, kv_out=kv, z_out=z, status=status)
         torch.cuda.synchronize()
+        # with `out` passed in, the binding asks torch's allocator for nothing either
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == allocations
         assert int(status.item()) == 0
         assert got.data_ptr() == out.data_ptr()
         close(got, ref, f"call {call}: output")
+        # ... and against the CPU oracle (Eq. 3), like every other entry point
+        want = torch.from_numpy(orc.linear_attn(q.float().cpu().numpy(), k.float().cpu().numpy(),
+                                                v.float().cpu().numpy(), eps=1e-6)).reshape(B, H, N, d)
+        close(got, want, f"call {call}: output against the oracle")
         np.testing.assert_allclose(z.cpu().numpy(), ref_z.cpu().numpy(), rtol=1e-4, atol=1e-3)
         np.testing.assert_allclose(kv.cpu().numpy(), ref_kv.cpu().numpy(), rtol=1e-3,
                                    atol=float(ref_kv.abs().max()) * 1e-4)
