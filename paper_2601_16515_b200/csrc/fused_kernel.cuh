@@ -8,8 +8,12 @@
 //   warp 0        TMA producer of the Q tile, the K ring and (at the end) the linear-state tile
 //   warp 1        TMA producer of the V ring (independent of the K ring, so neither ring can
 //                 stall the other)
-//   warp 2        tcgen05 issuer of S = Q K^T (one thread); owns the TMEM allocation
-//   warp 3        tcgen05 issuer of O += P V and of the linear numerator (one thread)
+//   warp 2        tcgen05 issuer of S = Q K^T; owns the TMEM allocation
+//   warp 3        tcgen05 issuer of O += P V and of the linear numerator
+//                 (an issuing warp walks its loop as a whole, every lane polling the barriers, and one
+//                 elected lane issues: the operands of a product are then warp-uniform values, which
+//                 keeps the cost of issuing one low -- measured 27 against 45 cycles per instruction
+//                 when a single lane runs the loop alone)
 //   warps 4-11    softmax + epilogue warps: a warp works on 16 query rows (TMEM lanes) with the
 //                 16-lane load/store shapes, four threads share a row and each thread serves two
 //                 rows; row maxima and sums are combined with two shuffles
@@ -21,8 +25,12 @@
 // as soon as the P V product of block t - 1 has read it, so both products of the neighbouring
 // blocks overlap the softmax of block t.  The running max lives in the log2 domain; exponentials
 // start against the max of the earlier blocks and the O accumulator is rescaled only when the max
-// grows by more than 2^8.  The two products have their own issuing threads: each waits only for
-// what its next MMA series needs, so it reacts as soon as that arrives.
+// grows by more than 2^8.  The two products have their own issuing warps: each waits only for
+// what its next MMA series needs, so it reacts as soon as that arrives.  One commit per series: the
+// barrier that announces the scores of block t also frees the K-ring stage for block t + 2, the one
+// that announces the completion of P V the V-ring stage.
+// The four producer / issuer warps (one warpgroup) hand registers to the eight softmax warps
+// (setmaxnreg: 40 against 96 per thread), which keeps the softmax loop free of spills.
 // After the last block the softmax warps apply ReLU to the Q rows in shared memory and compute the
 // linear denominator with plain FMAs; the linear state (bf16, transposed) is loaded over the K
 // ring, which is idle by then; the issuing thread multiplies ReLU(Q) with it, and the epilogue
@@ -87,7 +95,7 @@ static_assert(FusedCfg<128>::ST_BYTES == FusedCfg<128>::NK * FusedCfg<128>::KV_B
 static_assert(FusedCfg<64>::ST_BYTES <= FusedCfg<64>::NK * FusedCfg<64>::KV_BYTES, "the state tile fits in the K ring");
 
 struct FusedBarriers {
-    uint64_t q_full, st_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
+    uint64_t q_full, st_full, k_full[2], v_full[2];
     uint64_t s_full[2], p_ready[2], pv_done[2], o_final, lin_ready, lin_done, out_staged, z_full;
 };
 
@@ -150,9 +158,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_init(smem_u32(&bars.p_ready[j]), 8);          // one arrival per softmax warp
             mbar_init(smem_u32(&bars.pv_done[j]), 1);
             mbar_init(smem_u32(&bars.k_full[j]), 1);
-            mbar_init(smem_u32(&bars.k_empty[j]), 1);
             mbar_init(smem_u32(&bars.v_full[j]), 1);
-            mbar_init(smem_u32(&bars.v_empty[j]), 1);
         }
         fence_mbar_init();
     }
@@ -175,7 +181,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int len = le - ls;
     const bool inherited_abort = abort_flag != 0;      // uniform: read after the barrier above, before any wait
 
+    // a bounded wait taken by a whole warp: warp-uniform outcome
+    auto wait_warp = [&](uint64_t* bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, abortp));
+    };
+
     if (!inherited_abort) {
+    if (warp < 4) {
+    // the four producer / issuer warps (one warpgroup) give registers up, the eight softmax warps take them
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     if (warp == 0) {
         // ============================================================== TMA producer: Q, the K ring, the state tile
         bool ok = true;
@@ -191,13 +205,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             for (int t = 0; t < len; ++t) {
                 const int s = t % C::NK;
-                ok = mbar_wait(smem_u32(&bars.k_empty[s]), ((t / C::NK) & 1) ^ 1, abortp);
+                // stage s = t & 1 is free once Q K^T of block t - 2 has completed: the barrier that hands its
+                // scores to the softmax warps says so (one commit serves both)
+                if (t >= C::NK) ok = mbar_wait(smem_u32(&bars.s_full[s]), ((t >> 1) - 1) & 1, abortp);
                 if (!ok) break;
                 const int col = __ldg(p.col_idx + ls + t);
                 const uint32_t bar = smem_u32(&bars.k_full[s]);
                 mbar_arrive_expect_tx(bar, C::KV_BYTES);
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(s_base + C::OFF_K + s * C::KV_BYTES + ch * C::KV_CHUNK, &map_k, bar, ch * 64,
+                for (int ch = 0; ch < C::CH; ++ch)       // chunk-major: the two stages of a chunk are adjacent
+                    tma_load_3d(s_base + C::OFF_K + ch * (C::NK * C::KV_CHUNK) + s * C::KV_CHUNK, &map_k, bar, ch * 64,
                                 col * C::BK, bh);
             }
         }
@@ -228,7 +244,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             prefetch_tmap(&map_v);
             for (int t = 0; t < len; ++t) {
                 const int s = t % C::NV;
-                if (!mbar_wait(smem_u32(&bars.v_empty[s]), ((t / C::NV) & 1) ^ 1, abortp)) break;
+                // stage s = t & 1 is free once P V of block t - 2 has completed
+                if (t >= C::NV && !mbar_wait(smem_u32(&bars.pv_done[s]), ((t >> 1) - 1) & 1, abortp)) break;
                 const int col = __ldg(p.col_idx + ls + t);
                 const uint32_t bar = smem_u32(&bars.v_full[s]);
                 mbar_arrive_expect_tx(bar, C::KV_BYTES);
@@ -239,63 +256,67 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp == 2) {
         // ============================================================== issuer of S = Q K^T
-        if (lane == 0) {
-            const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
-            constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
-            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
-            const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
-            bool ok = true;
-            if (len > 0) {
-                ok = mbar_wait(smem_u32(&bars.q_full), 0, abortp);
-                tc_fence_after_sync();
-            }
+        // The whole warp walks the loop (every lane polls the barriers) and one elected lane issues: the
+        // operands of the products are then warp-uniform values, which is what keeps the cost of issuing
+        // a product low (measured: 27 against 45 cycles per instruction when one lane runs the loop alone).
+        const uint32_t idesc_qk = make_idesc_bf16(128, C::BK, 0, 0);
+        constexpr uint32_t HI = sdesc_hi_sw128(1024);   // the high descriptor word is one constant here
+        const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
+        const uint32_t k_lo0 = sdesc_lo(s_base + C::OFF_K, 16);
+        bool ok = true;
+        {
+            if (len > 0) ok = wait_warp(&bars.q_full, 0);
             for (int t = 0; t < len && ok; ++t) {
                 const int s = t % C::NK;
-                ok = mbar_wait(smem_u32(&bars.k_full[s]), (t / C::NK) & 1, abortp);
+                ok = wait_warp(&bars.k_full[s], (t / C::NK) & 1);
                 // score buffer t & 1 held P of block t - 2: its P V product must have read it
-                if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.pv_done[t & 1]), ((t >> 1) - 1) & 1, abortp);
+                if (ok && t >= 2) ok = wait_warp(&bars.pv_done[t & 1], ((t >> 1) - 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t kb_lo = k_lo0 + s * (C::KV_BYTES >> 4);
+                if (elect_one()) {
+                    const uint32_t kb_lo = k_lo0 + s * (C::KV_CHUNK >> 4);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
-                    mma_ss_lohi(tmem + C::COL_SP + (t & 1) * C::SP_STRIDE,
-                                q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
-                                kb_lo + (((k / 4) * C::KV_CHUNK + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
-                tc_commit(smem_u32(&bars.s_full[t & 1]));
-                tc_commit(smem_u32(&bars.k_empty[s]));
+                    for (int k = 0; k < D / 16; ++k)   // 16 channels: 32 bytes of each Q and K row, chunk k/4
+                        mma_ss_lohi(tmem + C::COL_SP + (t & 1) * C::SP_STRIDE,
+                                    q_lo + (((k / 4) * C::Q_CHUNK + (k % 4) * 32) >> 4), HI,
+                                    kb_lo + (((k / 4) * (C::NK * C::KV_CHUNK) + (k % 4) * 32) >> 4), HI, idesc_qk, k > 0);
+                    tc_commit(smem_u32(&bars.s_full[t & 1]));
+                }
+                __syncwarp();
             }
         }
     } else if (warp == 3) {
         // ============================================================== issuer of O += P V and of the linear numerator
-        if (lane == 0) {
-            const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
-            const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
-            constexpr uint32_t HI = sdesc_hi_sw128(1024);
-            const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
-            const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
-            bool ok = true;
-            for (int t = 0; t < len && ok; ++t) {
-                const int s = t % C::NV;
-                ok = mbar_wait(smem_u32(&bars.v_full[s]), (t / C::NV) & 1, abortp);
-                if (ok) ok = mbar_wait(smem_u32(&bars.p_ready[t & 1]), (t >> 1) & 1, abortp);
-                if (!ok) break;
-                tc_fence_after_sync();
+        const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+        const uint32_t idesc_lin = make_idesc_bf16(128, D, 0, 0);
+        constexpr uint32_t HI = sdesc_hi_sw128(1024);
+        const uint32_t q_lo = sdesc_lo(s_base + C::OFF_Q, 16);
+        const uint32_t v_lo0 = sdesc_lo(s_base + C::OFF_V, C::KV_CHUNK);
+        bool ok = true;
+        for (int t = 0; t < len && ok; ++t) {
+            const int s = t % C::NV;
+            ok = wait_warp(&bars.v_full[s], (t / C::NV) & 1);
+            if (ok) ok = wait_warp(&bars.p_ready[t & 1], (t >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (elect_one()) {
                 const uint32_t vb_lo = v_lo0 + s * (C::KV_BYTES >> 4);
                 const uint32_t p_col = tmem + C::COL_SP + (t & 1) * C::SP_STRIDE;
 #pragma unroll
                 for (int k = 0; k < C::BK / 16; ++k)      // 16 keys = 16 rows of 128 bytes
                     mma_ts_lohi(tmem + C::COL_O, p_col + k * 8, vb_lo + ((k * 2048) >> 4), HI, idesc_pv,
                                 (t > 0 || k > 0) ? 1u : 0u);
-                tc_commit(smem_u32(&bars.v_empty[s]));
                 tc_commit(smem_u32(&bars.pv_done[t & 1]));
                 if (t + 1 == len) tc_commit(smem_u32(&bars.o_final));
             }
-            if (ok && linear) {
-                ok = mbar_wait(smem_u32(&bars.st_full), 0, abortp);
-                if (ok) ok = mbar_wait(smem_u32(&bars.lin_ready), 0, abortp);
-                if (ok) {
-                    tc_fence_after_sync();
+            __syncwarp();
+        }
+        if (ok && linear) {
+            ok = wait_warp(&bars.st_full, 0);
+            if (ok) ok = wait_warp(&bars.lin_ready, 0);
+            if (ok) {
+                tc_fence_after_sync();
+                if (elect_one()) {
                     const uint32_t st_lo = sdesc_lo(s_base + C::OFF_ST, 16);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k)
@@ -303,9 +324,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                                     st_lo + (((k / 4) * C::ST_CHUNK + (k % 4) * 32) >> 4), HI, idesc_lin, k > 0);
                     tc_commit(smem_u32(&bars.lin_done));
                 }
+                __syncwarp();
             }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
         // ============================================================== softmax + epilogue
         // Eight warps.  A warp works on 16 TMEM lanes (query rows) with the 16-lane
         // load/store shapes: four threads share a row, each holding a quarter of its columns,
@@ -335,10 +359,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             return v + __shfl_xor_sync(0xffffffffu, v, 2);
         };
 
-        const bool ragged_keys = (p.N % C::BK) != 0;
+        // Only the last key block of the sequence can be short (N not a multiple of 64), and in an ascending
+        // list it can only be the last entry: one look at that entry, before the loop, settles which block
+        // needs its missing keys masked.
+        const int valid_last = (len > 0 && (p.N % C::BK) != 0 && __ldg(p.col_idx + le - 1) == p.nKb - 1)
+                                   ? p.N - (p.nKb - 1) * C::BK : C::BK;
         for (int t = 0; t < len && ok; ++t) {
-            // only the last key block can be short; its id is needed only then
-            const int col = ragged_keys ? __ldg(p.col_idx + ls + t) : 0;
             ok = wait_uniform(&bars.s_full[t & 1], (t >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
@@ -347,8 +373,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_ld_16x256b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, xr);
             tmem_wait_ld();
             float* x = reinterpret_cast<float*>(xr);
-            const int valid = p.N - col * C::BK;              // keys of this block that exist
-            if (ragged_keys && valid < C::BK) {
+            if (valid_last < C::BK && t + 1 == len) {         // keys of this block that exist
+                const int valid = valid_last;
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     const int key = 8 * n + 2 * q4;

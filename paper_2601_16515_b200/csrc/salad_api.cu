@@ -272,7 +272,7 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
 }
 
 template <int D>
-int launch_fused(const Problem& P, const Workspace& w) {
+int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     const int BH = P.B * P.H;
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
     CUtensorMap mq, mk, mv, mo, ms;
@@ -301,6 +301,8 @@ int launch_fused(const Problem& P, const Workspace& w) {
     const int64_t grid = int64_t(fp.nQb) * BH;
     if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
     record_profile(2, P.stream);
+    SALAD_LOGF("salad_fused_kernel<%d> grid %lld block %d smem %d (mode %d)", D, (long long)grid, FusedCfg<D>::THREADS,
+               FusedCfg<D>::SMEM_BYTES, P.mode);
     launch_dependent(salad_fused_kernel<D>, dim3(unsigned(grid)), dim3(FusedCfg<D>::THREADS),
                      FusedCfg<D>::SMEM_BYTES, P.stream, mq, mk, mv, mo, ms, fp);
     record_profile(3, P.stream);
@@ -391,7 +393,7 @@ int run(const Problem& P) {
     // linear-only calls: the stand-alone apply kernel
     if (P.mode == MODE_LINEAR)
         return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
-    return (P.d == 128) ? launch_fused<128>(P, w) : launch_fused<64>(P, w);
+    return (P.d == 128) ? launch_fused<128>(P, w, dev) : launch_fused<64>(P, w, dev);
 }
 
 // ---------------------------------------------------------------------------------------
