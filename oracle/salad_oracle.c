@@ -416,6 +416,45 @@ ORACLE_API void oracle_proj_combine(const float* o_s, const float* o_l, const fl
 }
 
 /*
+ * oracle_salad_fused_blockproj: Algorithm 1 with a block-diagonal Level-1 projection (Sec. 4.2): the
+ * projection layer of the linear branch restricted to one d x d block per head, no mixing between heads,
+ *     O'_l[b,h,n,:] = W_h O_l[b,h,n,:]         (W_h[c_out][a_in], the diagonal block h of Proj's weight)
+ *     O~[b,h,n,:]   = O_s[b,h,n,:] + [s_b >= tau] * s_b * O'_l[b,h,n,:].
+ * W_h = lambda_h I gives oracle_salad_fused; a full weight matrix that is zero off the diagonal blocks
+ * gives oracle_proj_combine.
+ *   w_blocks [H][d][d]
+ */
+ORACLE_API void oracle_salad_fused_blockproj(const float* q, const float* k, const float* v,
+                                             int B, int H, int N, int d, int Bq, int Bk,
+                                             const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                             const float* w_blocks, const double* s_b, double tau,
+                                             double scale, double eps,
+                                             const int64_t* sel, int64_t nsel, double* o)
+{
+    if (!sel) nsel = (int64_t)B * H * N;
+    int64_t BH = (int64_t)B * H;
+    double* kv = (double*)malloc(sizeof(double) * (size_t)(BH * d * d));
+    double* z = (double*)malloc(sizeof(double) * (size_t)(BH * d));
+    double* ol = (double*)malloc(sizeof(double) * (size_t)(nsel * d));
+    oracle_sparse_attn(q, k, v, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, scale, sel, nsel, o, NULL);
+    oracle_linear_state(k, v, B, H, N, d, kv, z);
+    oracle_linear_attn(q, kv, z, B, H, N, d, eps, sel, nsel, ol);
+    for (int64_t s = 0; s < nsel; ++s) {
+        int64_t bh; int n;
+        decode_row(sel, s, N, &bh, &n);
+        double sb = s_b[bh / H];
+        if (!(sb >= tau)) continue;                      /* dropped branch: the sparse output alone */
+        const float* wh = w_blocks + (bh % H) * (int64_t)d * d;
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int a = 0; a < d; ++a) acc += (double)wh[(int64_t)c * d + a] * ol[s * d + a];
+            o[s * d + c] += sb * acc;
+        }
+    }
+    free(kv); free(z); free(ol);
+}
+
+/*
  * Linear branch with rotary position embedding.  Sec. 4.1 states that the linear branch carries a
  * 3-D rotary embedding and gives no formula; the form taken here is the one the rotary-embedding
  * paper it cites defines for linear attention: the rotation enters the numerator only,

@@ -53,6 +53,9 @@ def _load():
         lib.oracle_salad_fused_drop.restype = None
         lib.oracle_salad_fused_drop.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
                                                                          p, i64, p])
+        lib.oracle_salad_fused_blockproj.restype = None
+        lib.oracle_salad_fused_blockproj.argtypes = ([p, p, p] + [i32] * 6 + [p, p, i32, p, p, f64, f64, f64,
+                                                                               p, i64, p])
         lib.oracle_proj_combine.restype = None
         lib.oracle_proj_combine.argtypes = [p, p, p, p, p, i32, i32, i32, i32, p]
         lib.oracle_topk_mask.restype = None
@@ -207,6 +210,26 @@ def salad_fused_drop(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, lambda_h, s_b, tau, 
         scale = 1.0 / np.sqrt(d)
     lib.oracle_salad_fused_drop(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, lam.ctypes.data,
                                 sb.ctypes.data, float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
+    return o
+
+
+def salad_fused_blockproj(q, k, v, Bq, Bk, row_ptr, col_idx, Hm, w_blocks, s_b, tau=-np.inf, scale=None,
+                          eps=1e-6, sel=None):
+    """Algorithm 1 with one d x d projection block per head on the linear branch:
+    O_s + [s_b >= tau] * s_b * W_h O_l, w_blocks [H, d, d] = W_h[c_out][a_in].  [rows, d] float64."""
+    lib = _load()
+    q, qp = _f32(q); k, kp = _f32(k); v, vp = _f32(v)
+    B, H, N, d = q.shape
+    rp, rpp = _i32(row_ptr); ci, cip = _i32(col_idx if len(col_idx) else np.zeros(1, np.int32))
+    w, wp = _f32(w_blocks); assert w.shape == (H, d, d)
+    sb = np.ascontiguousarray(s_b, dtype=np.float64); assert sb.size == B
+    s, sp, nsel = _sel(sel)
+    rows = nsel if s is not None else B * H * N
+    o = np.empty((rows, d), dtype=np.float64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    lib.oracle_salad_fused_blockproj(qp, kp, vp, B, H, N, d, Bq, Bk, rpp, cip, Hm, wp, sb.ctypes.data,
+                                     float(tau), float(scale), float(eps), sp, nsel, o.ctypes.data)
     return o
 
 

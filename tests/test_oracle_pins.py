@@ -526,6 +526,45 @@ def test_proj_combine_block_diagonal_is_the_fused_path():
     np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
 
 
+def test_blockproj_pins():
+    # One d x d projection block per head (Alg. 1 Level 1 without head mixing), pinned from both sides:
+    # against the full projection with a block-diagonal weight, and against the per-head scalar.
+    B, H, N, d = 2, 3, 48, 8
+    q, k, v = rand_qkv(B, H, N, d, 105)
+    rng = np.random.default_rng(7)
+    rp, ci = wlmod.dense_csr(3, 6, 1)                     # 16 x 8 blocks, everything kept
+    s = np.array([0.4, 0.9])
+    wb = (rng.standard_normal((H, d, d)) * 0.4).astype(np.float32)
+    assert not np.allclose(wb, np.swapaxes(wb, 1, 2))     # a transposed block must not pass
+    got = orc.salad_fused_blockproj(q, k, v, 16, 8, rp, ci, 1, wb, s).reshape(B, H, N, d)
+    o_s = orc.sparse_attn(q, k, v, 16, 8, rp, ci, 1)[0].reshape(B, H, N, d)
+    o_l = orc.linear_attn(q, k, v).reshape(B, H, N, d)
+    # ... written out with numpy: y[c] = sum_a W_h[c][a] x[a]
+    want = o_s + s[:, None, None, None] * np.einsum("hca,bhna->bhnc", wb.astype(np.float64), o_l)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    # ... the full projection layer whose weight is zero outside the diagonal blocks (o_s, o_l pass through
+    # fp32 in that wrapper: compared at that precision)
+    W = np.zeros((H * d, H * d), np.float32)
+    for h in range(H):
+        W[h * d:(h + 1) * d, h * d:(h + 1) * d] = wb[h]
+    np.testing.assert_allclose(got, orc.proj_combine(o_s, o_l, W, s), rtol=1e-5, atol=1e-6)
+    # ... W_h = lambda_h I: the per-head static scale of the fused call
+    lam = np.array([0.7, 0.2, 1.3])
+    wl_ = np.stack([l * np.eye(d) for l in lam]).astype(np.float32)
+    np.testing.assert_allclose(orc.salad_fused_blockproj(q, k, v, 16, 8, rp, ci, 1, wl_, s),
+                               orc.salad_fused(q, k, v, 16, 8, rp, ci, 1, lam.astype(np.float32), s), rtol=1e-6, atol=1e-7)
+    # zero blocks (the zero-initialised layer): the sparse branch exactly; and the drop threshold
+    zero = orc.salad_fused_blockproj(q, k, v, 16, 8, rp, ci, 1, np.zeros_like(wb), s).reshape(B, H, N, d)
+    assert np.array_equal(zero, o_s)
+    drop = orc.salad_fused_blockproj(q, k, v, 16, 8, rp, ci, 1, wb, s, tau=0.5).reshape(B, H, N, d)
+    assert np.array_equal(drop[0], o_s[0])
+    np.testing.assert_allclose(drop[1], got[1], rtol=0, atol=0)
+    # row selection
+    sel = np.array([0, 17, N + 5, B * H * N - 1], dtype=np.int64)
+    np.testing.assert_array_equal(orc.salad_fused_blockproj(q, k, v, 16, 8, rp, ci, 1, wb, s, sel=sel),
+                                  got.reshape(-1, d)[sel])
+
+
 # ----------------------------------------------------------------------------------------
 # Linear branch with the rotary embedding (Sec. 4.1: the linear branch carries a 3-D rotary
 # embedding; rotation in the numerator only, the normaliser un-rotated)
