@@ -176,6 +176,52 @@ int salad_fused_drop_fwd(const void* q, const void* k, const void* v, void* o,
                          int32_t* d_status, void* stream);
 
 /*
+ * salad_linear_state_fwd / salad_fused_prepared_fwd -- salad_fused_drop_fwd in two calls, for callers who
+ * have K and V before Q (or a free stream): the two reductions of Eq. 3,
+ *     KV = sum_j ReLU(K_j)^T V_j ,   Z = sum_j ReLU(K_j) ,
+ * are one pass over K and V that needs nothing else, so it can run early or beside other work; the
+ * attention call then finds the state in the workspace and runs without the reduction kernels.
+ *   salad_linear_state_fwd(k, v, ...)     leaves the state in `workspace`; kv_out (fp32 [B,H,d,d]) and
+ *                                         z_out (fp32 [B,H,d]) receive copies when not NULL.
+ *   salad_fused_prepared_fwd(q, k, v, ..) arguments as salad_fused_drop_fwd; `workspace` must be the one a
+ *                                         completed salad_linear_state_fwd call on the same K, V, B, H, N, d
+ *                                         wrote (order the two calls with the stream or an event).  The result
+ *                                         equals salad_fused_drop_fwd bit for bit.
+ * Branch dropping happens in the second call (the state is computed for every batch item).
+ */
+int salad_linear_state_fwd(const void* k, const void* v, float* kv_out, float* z_out, int B, int H, int N, int d,
+                           void* workspace, size_t workspace_bytes, int32_t* d_status, void* stream);
+int salad_fused_prepared_fwd(const void* q, const void* k, const void* v, void* o,
+                             int B, int H, int N, int d, int Bq, int Bk,
+                             const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                             const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                             float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                             int32_t* d_status, void* stream);
+
+/*
+ * salad_fused_proj_fwd -- salad_fused_drop_fwd with a block-diagonal Level-1 projection (Algorithm 1,
+ * "Level 1: layer-wise static scaling"; Sec. 4.2, the zero-initialised projection of the linear branch)
+ * in place of the per-head scalar: one d x d block per head, no mixing between heads,
+ *     O[b,h,n,:] = O_s[b,h,n,:] + [d_dyn_scale[b] >= drop_tau] * d_dyn_scale[b] * W_h O_l[b,h,n,:].
+ * The block folds into the linear state, W_h (ReLU(Q_n) KV)^T = (KV W_h^T)^T ReLU(Q_n)^T: the state of
+ * every head is multiplied with its block once (a d x d x d product in fp32, rounded once to bf16) and
+ * the attention kernel runs unchanged, so the call still reads Q, K, V once and writes O once.  The
+ * normaliser Z is applied before the projection, as in Algorithm 1.
+ *   d_proj_blocks  device bf16 [H, d, d], 16-byte aligned: W_h[c_out][a_in], i.e. the diagonal blocks of
+ *                  the weight matrix salad_proj_combine_fwd takes; lambda of Eq. 5 multiplied in by the
+ *                  caller.  W_h = lambda_h I reproduces salad_fused_fwd; zero blocks (the layer before
+ *                  tuning) reproduce salad_sparse_attn_fwd.
+ *   drop_tau       -INFINITY: no branch is dropped.
+ * A projection that mixes heads cannot be folded in this way: see salad_proj_combine_fwd.
+ */
+int salad_fused_proj_fwd(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int N, int d, int Bq, int Bk,
+                         const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                         const void* d_proj_blocks, const float* d_dyn_scale, float drop_tau,
+                         float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                         int32_t* d_status, void* stream);
+
+/*
  * salad_fused_rope_fwd / salad_linear_attn_rope_fwd -- the same two calls with a rotary position
  * embedding in the linear branch (Sec. 4.1 states that the linear branch carries a 3-D rotary embedding
  * and gives no formula; the rotation enters the numerator only, as the rotary-embedding paper it cites

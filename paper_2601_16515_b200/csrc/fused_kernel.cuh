@@ -65,6 +65,7 @@ struct FusedParams {
     float eps;
     float drop_tau;              // linear branch of batch item b skipped when dyn_scale[b] < drop_tau
     const __half* rope;          // [N][D] fp16: (cos, sin) per token and channel pair of the rotary linear branch, or null
+    int wait_at_top;             // 1: wait for the kernel before this one at once (calls without state kernels)
     int32_t* ws_status;          // library status word (never null)
     int32_t* user_status;        // optional
 };
@@ -119,7 +120,7 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     // before this one.  With one, the state kernels lie between, and this kernel does not wait for them
     // here: it runs beside them (each of their CTAs has passed its own wait for the first kernel before
     // a CTA of this one is placed) and waits only where it first touches the state, in the epilogue.
-    if ((p.mode & MODE_LINEAR) == 0) grid_dependency_wait();
+    if ((p.mode & MODE_LINEAR) == 0 || p.wait_at_top) grid_dependency_wait();
     grid_launch_dependents();
 
     // work item: head by head (K/V of one head stay hot in L2: ordering the cheapest items of all

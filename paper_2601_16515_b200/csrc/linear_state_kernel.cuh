@@ -290,14 +290,16 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 }
 
 // Sum the partials of each head in chunk order; emit
-//   kv_out  fp32 [BH][D][D]  (optional)      z fp32 [BH][D]  (+ optional user copy)
+//   kv_out  fp32 [BH][D][D]  (optional; kv_ws: a second, workspace copy for the projection kernel)
+//   z       fp32 [BH][D]  (+ optional user copy)
 //   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
 //           num = ReLU(Q) KV in the fused kernel.
 template <int D, int ROWS>
 __global__ void __launch_bounds__(32 * ROWS)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
-                             float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
-                             __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
+                             float* __restrict__ kv_out, float* __restrict__ kv_ws, float* __restrict__ z_ws,
+                             float* __restrict__ z_out, __nv_bfloat16* __restrict__ kvt,
+                             const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
     // The kernel after this one may be placed at once (it waits for this one before it touches the
     // state).  In fused calls ROWS = 8: a block is small, 256 threads and few registers, so that while it
@@ -333,6 +335,7 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
         }
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
+        if (kv_ws) kv_ws[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;        // for the projection kernel below
         tile[ty + ROWS * r][tx] = s;
     }
     __syncthreads();
@@ -347,6 +350,46 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
             z_ws[size_t(bh) * D + a] = s;
             if (z_out) z_out[size_t(bh) * D + a] = s;
         }
+    }
+}
+
+// Block-diagonal Level-1 projection (Algorithm 1; Sec. 4.2), folded into the linear state: with one d x d
+// block W_h per head on the linear branch,
+//     W_h (ReLU(Q_n) KV)^T = (KV W_h^T)^T ReLU(Q_n)^T ,   i.e.   num' = ReLU(Q_n) KV'  with  KV' = KV W_h^T,
+// so projecting the state once per head (a d x d x d product) projects every output row for free; the
+// normaliser Z is applied before the projection and stays as it is.  This kernel overwrites the bf16
+// transposed state the attention kernel multiplies with:
+//     kvt[c][a'] = KV'[a'][c] = sum_a KV[a'][a] * W_h[c][a]
+// from the fp32 state kv_ws[BH][D][D] and w[H][D][D] (bf16, W_h[c_out][a_in]), in fp32, one rounding.
+// grid (D/32, D/32, BH), 256 threads: a 32 (c) x 32 (a') tile per block, operands through shared memory.
+template <int D>
+__global__ void __launch_bounds__(256)
+salad_state_project_kernel(const float* __restrict__ kv_ws, const __nv_bfloat16* __restrict__ w,
+                           __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
+{
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int bh = blockIdx.z;
+    if (branch_dropped(dyn_scale, drop_tau, bh / H)) return;
+    __shared__ float ws[32][D + 1], ks[32][D + 1];
+    const int c0 = blockIdx.x * 32, a0 = blockIdx.y * 32;
+    const int tid = threadIdx.x;
+    const __nv_bfloat16* wh = w + size_t(bh % H) * D * D;
+    const float* kvh = kv_ws + size_t(bh) * D * D;
+    for (int i = tid; i < 32 * D; i += 256) {
+        const int r = i / D, a = i % D;
+        ws[r][a] = __bfloat162float(wh[size_t(c0 + r) * D + a]);
+        ks[r][a] = kvh[size_t(a0 + r) * D + a];
+    }
+    __syncthreads();
+    const int ap = tid % 32;                         // a' within the tile: consecutive threads, consecutive bf16
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int c = tid / 32 + 8 * u;
+        float acc = 0.f;
+#pragma unroll 8
+        for (int a = 0; a < D; ++a) acc = fmaf(ks[ap][a], ws[c][a], acc);
+        kvt[size_t(bh) * D * D + size_t(c0 + c) * D + a0 + ap] = __float2bfloat16(acc);
     }
 }
 

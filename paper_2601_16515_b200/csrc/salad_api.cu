@@ -52,7 +52,7 @@ inline void record_profile(int idx, cudaStream_t st) {
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
-    size_t off_status, off_kvt, off_z, off_kvp, off_zp, off_order, total;
+    size_t off_status, off_kvt, off_z, off_kvp, off_zp, off_order, off_kvf, total;
     int slots;
 };
 
@@ -67,7 +67,8 @@ Workspace carve(int B, int H, int N, int d, int Bq) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = w.off_zp + align_up(size_t(w.slots) * d * 4);
-    w.total = w.off_order + align_up(BH * nItems * 4);              // launch order, per mask (at most B*H)
+    w.off_kvf = w.off_order + align_up(BH * nItems * 4);            // launch order, per mask (at most B*H)
+    w.total = w.off_kvf + align_up(BH * d * d * 4);                 // fp32 state, for the block projection
     return w;
 }
 
@@ -189,14 +190,22 @@ struct Problem {
     float softmax_scale, eps, drop_tau;
     float *kv_out, *z_out;
     const void* rope;             // fp16 [N, d/2, 2] cosine and sine per token and channel pair, or null
+    const void* proj_blocks;      // bf16 [H, d, d]: one projection block per head on the linear branch, or null
+    bool state_only;              // salad_linear_state_fwd: the two reductions of Eq. 3 and nothing else
+    bool prepared;                // salad_fused_prepared_fwd: the workspace already holds the linear state
     void* ws; size_t ws_bytes; int32_t* d_status; cudaStream_t stream;
 };
 
 int validate(const Problem& P) {
-    if (!P.q || !P.k || !P.v || !P.o) return SALAD_ERR_INVALID_ARG;
+    if (P.state_only) {
+        if (!P.k || !P.v || !aligned16(P.k) || !aligned16(P.v)) return SALAD_ERR_INVALID_ARG;
+    } else if (!P.q || !P.k || !P.v || !P.o) {
+        return SALAD_ERR_INVALID_ARG;
+    }
     if (P.B <= 0 || P.H <= 0 || P.N <= 0 || P.d <= 0 || P.Bq <= 0 || P.Bk <= 0) return SALAD_ERR_INVALID_ARG;
     if (!shape_supported(P.d, P.Bq, P.Bk)) return SALAD_ERR_UNSUPPORTED;
-    if (!aligned16(P.q) || !aligned16(P.k) || !aligned16(P.v) || !aligned16(P.o)) return SALAD_ERR_INVALID_ARG;
+    if (!P.state_only && (!aligned16(P.q) || !aligned16(P.k) || !aligned16(P.v) || !aligned16(P.o)))
+        return SALAD_ERR_INVALID_ARG;
     if (int64_t(P.B) * P.H > 65535) return SALAD_ERR_UNSUPPORTED;
     if (P.mode & MODE_SPARSE) {
         if (!P.row_ptr || !P.col_idx) return SALAD_ERR_INVALID_ARG;
@@ -207,7 +216,8 @@ int validate(const Problem& P) {
         if (!(P.eps >= 0.f) || !isfinite(P.eps)) return SALAD_ERR_INVALID_ARG;
         if (P.rope && !aligned16(P.rope)) return SALAD_ERR_INVALID_ARG;
     }
-    if (P.mode == MODE_FUSED && (!P.static_scale || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
+    if (P.mode == MODE_FUSED && ((!P.static_scale && !P.proj_blocks) || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
+    if (P.proj_blocks && !aligned16(P.proj_blocks)) return SALAD_ERR_INVALID_ARG;
     const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
     if (!P.ws || (reinterpret_cast<uintptr_t>(P.ws) % kAlign) != 0 || P.ws_bytes < w.total)
         return SALAD_ERR_WORKSPACE;
@@ -261,12 +271,20 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     float* z_ws = reinterpret_cast<float*>(ws + w.off_z);
     __nv_bfloat16* kvt = reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt);
+    float* kv_ws = P.proj_blocks ? reinterpret_cast<float*>(ws + w.off_kvf) : nullptr;
     if ((P.mode & MODE_SPARSE) && !P.rope)
         launch_dependent(salad_linear_finalize_kernel<D, 8>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
-                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, kv_ws, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
     else
         launch_dependent(salad_linear_finalize_kernel<D, 32>, dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream,
-                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, kv_ws, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+    if (P.proj_blocks) {
+        // block-diagonal projection folded into the state: the attention kernel multiplies with KV W_h^T
+        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
+        SALAD_LOGF("salad_state_project_kernel<%d> grid (%d, %d, %d)", D, D / 32, D / 32, BH);
+        launch_dependent(salad_state_project_kernel<D>, dim3(D / 32, D / 32, BH), dim3(256), 0, P.stream, kv_ws,
+                         static_cast<const __nv_bfloat16*>(P.proj_blocks), kvt, P.dyn_scale, P.drop_tau, P.H);
+    }
     record_profile(1, P.stream);
     return check_launch();
 }
@@ -298,6 +316,7 @@ int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     fp.rope = static_cast<const __half*>(P.rope);
     fp.ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
     fp.user_status = P.d_status;
+    fp.wait_at_top = P.prepared ? 1 : 0;      // no state kernels in this call: the kernel before is the first one
     const int64_t grid = int64_t(fp.nQb) * BH;
     if (grid > 2147483647ll) return SALAD_ERR_UNSUPPORTED;
     record_profile(2, P.stream);
@@ -386,10 +405,11 @@ int run(const Problem& P) {
                                                       P.d_status, clear_status);
         if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     }
-    if (P.mode & MODE_LINEAR) {
+    if ((P.mode & MODE_LINEAR) && !P.prepared) {
         rc = (P.d == 128) ? launch_state<128>(P, w, dev) : launch_state<64>(P, w, dev);
         if (rc != SALAD_OK) return rc;
     }
+    if (P.state_only) return SALAD_OK;
     // linear-only calls: the stand-alone apply kernel
     if (P.mode == MODE_LINEAR)
         return (P.d == 128) ? launch_apply<128>(P, w, dev) : launch_apply<64>(P, w, dev);
@@ -425,6 +445,7 @@ Workspace carve_noalloc(int B, int H, int d) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = 0;                                  // linear attention has no kept lists to order
+    w.off_kvf = 0;                                    // (no projection in the linear-only calls)
     w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
     return w;
 }
@@ -591,6 +612,58 @@ SALAD_EXPORT int salad_fused_fwd(const void* q, const void* k, const void* v, vo
     // no threshold: every branch is kept, whatever the value of its scale
     return salad_fused_drop_fwd(q, k, v, o, B, H, N, d, Bq, Bk, row_ptr, col_idx, Hm, d_static_scale, d_dyn_scale,
                                 -INFINITY, softmax_scale, eps, workspace, workspace_bytes, d_status, stream);
+}
+
+SALAD_EXPORT int salad_linear_state_fwd(const void* k, const void* v, float* kv_out, float* z_out, int B, int H, int N,
+                                        int d, void* workspace, size_t workspace_bytes, int32_t* d_status,
+                                        void* stream) {
+    Problem P{};
+    P.drop_tau = -INFINITY;
+    P.k = k; P.v = v;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = 1; P.mode = MODE_LINEAR;
+    P.state_only = true;
+    P.kv_out = kv_out; P.z_out = z_out;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_fused_prepared_fwd(const void* q, const void* k, const void* v, void* o,
+                                          int B, int H, int N, int d, int Bq, int Bk,
+                                          const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                          const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                                          float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                                          int32_t* d_status, void* stream) {
+    if (isnan(drop_tau)) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
+    P.prepared = true;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
+    P.softmax_scale = softmax_scale; P.eps = eps;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_fused_proj_fwd(const void* q, const void* k, const void* v, void* o,
+                                      int B, int H, int N, int d, int Bq, int Bk,
+                                      const int32_t* row_ptr, const int32_t* col_idx, int Hm,
+                                      const void* d_proj_blocks, const float* d_dyn_scale, float drop_tau,
+                                      float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                                      int32_t* d_status, void* stream) {
+    if (isnan(drop_tau) || !d_proj_blocks) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = nullptr; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
+    P.proj_blocks = d_proj_blocks;
+    P.softmax_scale = softmax_scale; P.eps = eps;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
 }
 
 SALAD_EXPORT int salad_fused_rope_fwd(const void* q, const void* k, const void* v, void* o,

@@ -30,7 +30,8 @@ EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_set_profile_events", "salad_linear_attn_fwd_noalloc", "salad_fused_drop_fwd",
            "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
            "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd",
-           "salad_rope3d_table_build", "salad_csr_validate", "salad_set_mask_validation")
+           "salad_rope3d_table_build", "salad_csr_validate", "salad_set_mask_validation",
+           "salad_fused_proj_fwd", "salad_linear_state_fwd", "salad_fused_prepared_fwd")
 
 
 class SaladError(RuntimeError):
@@ -82,6 +83,12 @@ def _load() -> ctypes.CDLL:
     lib.salad_rope3d_table_build.argtypes = [i32, i32, i32, i32, f32, p, p]
     lib.salad_set_profile_events.restype = i32
     lib.salad_set_profile_events.argtypes = [p]
+    lib.salad_fused_proj_fwd.restype = i32
+    lib.salad_fused_proj_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, f32, p, sz, p, p]
+    lib.salad_linear_state_fwd.restype = i32
+    lib.salad_linear_state_fwd.argtypes = [p, p, p, p] + [i32] * 4 + [p, sz, p, p]
+    lib.salad_fused_prepared_fwd.restype = i32
+    lib.salad_fused_prepared_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, f32, p, sz, p, p]
     lib.salad_csr_validate.restype = i32
     lib.salad_csr_validate.argtypes = [p, p, i64, i64, i32, p, p]
     lib.salad_set_mask_validation.restype = i32
@@ -277,6 +284,63 @@ def salad_fused_rope_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_s
                                          _ptr(rope), tau, float(softmax_scale), float(eps), _ptr(workspace),
                                          workspace.numel(), _ptr(status), _stream(stream)),
                "salad_fused_rope_fwd")
+    return out
+
+
+def salad_linear_state_fwd(k, v, workspace, kv_out=None, z_out=None, status=None, stream=None):
+    """The linear state (KV, Z of Eq. 3) of K, V into `workspace`, for a later salad_fused_prepared_fwd call on
+    the same workspace; kv_out fp32 [B,H,d,d] and z_out fp32 [B,H,d] receive copies when given."""
+    for name, t in (("k", k), ("v", v)):
+        _bf16_4d(name, t)
+    if k.shape != v.shape:
+        raise ValueError("k and v must have the same shape")
+    B, H, N, d = k.shape
+    with torch.cuda.device(k.device):
+        _check(_lib.salad_linear_state_fwd(_ptr(k), _ptr(v), _ptr(kv_out), _ptr(z_out), B, H, N, d, _ptr(workspace),
+                                           workspace.numel(), _ptr(status), _stream(stream)), "salad_linear_state_fwd")
+    return workspace
+
+
+def salad_fused_prepared_fwd(q, k, v, row_ptr, col_idx, Hm: int, static_scale, dyn_scale, workspace, Bq: int = 128,
+                             Bk: int = 64, softmax_scale: float = 0.0, eps: float = 1e-6, out=None, status=None,
+                             stream=None, drop_tau: Optional[float] = None):
+    """salad_fused_fwd on a workspace that already holds the linear state (salad_linear_state_fwd)."""
+    B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    for name, t, n in (("static_scale", static_scale, H), ("dyn_scale", dyn_scale, B)):
+        if t.dtype != torch.float32 or not t.is_cuda or t.numel() != n or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor with {n} elements")
+    if out is None:
+        out = torch.empty_like(q)
+    tau = float("-inf") if drop_tau is None else float(drop_tau)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_fused_prepared_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                             _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(static_scale), _ptr(dyn_scale), tau,
+                                             float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
+                                             _ptr(status), _stream(stream)), "salad_fused_prepared_fwd")
+    return out
+
+
+def salad_fused_proj_fwd(q, k, v, row_ptr, col_idx, Hm: int, proj_blocks, dyn_scale, Bq: int = 128, Bk: int = 64,
+                         softmax_scale: float = 0.0, eps: float = 1e-6, out=None, workspace=None, status=None,
+                         stream=None, drop_tau: Optional[float] = None):
+    """O = O_sparse + dyn_scale[b] * W_h O_linear with one d x d projection block per head
+    (proj_blocks bf16 [H, d, d], W_h[c_out][a_in]), one bf16 write."""
+    B, H, N, d, workspace = _common(q, k, v, Bq, Bk, workspace)
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    if (proj_blocks.dtype != torch.bfloat16 or not proj_blocks.is_cuda or not proj_blocks.is_contiguous()
+            or tuple(proj_blocks.shape) != (H, d, d)):
+        raise ValueError(f"proj_blocks must be a contiguous CUDA bf16 tensor [{H}, {d}, {d}]")
+    if dyn_scale.dtype != torch.float32 or not dyn_scale.is_cuda or dyn_scale.numel() != B or not dyn_scale.is_contiguous():
+        raise ValueError(f"dyn_scale must be a contiguous CUDA fp32 tensor with {B} elements")
+    if out is None:
+        out = torch.empty_like(q)
+    tau = float("-inf") if drop_tau is None else float(drop_tau)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_fused_proj_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, Bq, Bk,
+                                         _ptr(row_ptr), _ptr(col_idx), Hm, _ptr(proj_blocks), _ptr(dyn_scale), tau,
+                                         float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
+                                         _ptr(status), _stream(stream)), "salad_fused_proj_fwd")
     return out
 
 

@@ -666,6 +666,64 @@ def test_full_projection_pipeline_matches_fused_for_block_diagonal(salad):
     assert_close(f32(out.cpu()).reshape(-1, wl.d), f32(fused.cpu()).reshape(-1, wl.d).astype(np.float64), "pipeline vs fused")
 
 
+@pytest.mark.parametrize("B,H,N,d,Bq", [(2, 3, 1000, 128, 128), (1, 2, 1024, 64, 64), (1, 12, 700, 128, 128)])
+def test_fused_block_projection(salad, B, H, N, d, Bq):
+    # one d x d projection block per head folded into the linear state (Alg. 1 Level 1 without head mixing)
+    wl = wlmod.Workload("t", B, H, d, (1, 1, N), Bq, 64, (), 1)
+    q, k, v = rand_qkv(B, H, N, d, 600 + N)
+    rng = np.random.default_rng(N + d)
+    rp, ci = random_csr(wl.nQb, wl.nKb, 4 + N, lo=0, hi=min(wl.nKb, 9))
+    rp_d, ci_d = dev_csr(rp, ci)
+    wb = bf16(rng.standard_normal((H, d, d)) / np.sqrt(d))
+    s = rng.uniform(0.2, 0.9, B).astype(np.float32)
+    qd, kd, vd, s_d = q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(s).cuda()
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_proj_fwd(qd, kd, vd, rp_d, ci_d, 1, wb.cuda(), s_d, Bq=Bq, status=status)
+    status_ok(status)
+    ref = orc.salad_fused_blockproj(f32(q), f32(k), f32(v), Bq, 64, rp, ci, 1, f32(wb), s.astype(np.float64))
+    assert_close(f32(out.cpu()).reshape(-1, d), ref, "block projection")
+    # W_h = lambda_h I is the per-head scalar of salad_fused_fwd (lambda representable in bf16: same bits up to
+    # the order of the roundings), zero blocks are the sparse branch bit for bit
+    lam = torch.tensor([0.5, 0.25, 1.0, 0.75] * 3)[:H]
+    wi = torch.stack([l * torch.eye(d) for l in lam]).to(torch.bfloat16).cuda()
+    a = salad.salad_fused_proj_fwd(qd, kd, vd, rp_d, ci_d, 1, wi, s_d, Bq=Bq)
+    b_ = salad.salad_fused_fwd(qd, kd, vd, rp_d, ci_d, 1, lam.float().cuda(), s_d, Bq=Bq)
+    assert_close(f32(a.cpu()).reshape(-1, d), f32(b_.cpu()).reshape(-1, d).astype(np.float64), "identity blocks vs scalar")
+    zero = salad.salad_fused_proj_fwd(qd, kd, vd, rp_d, ci_d, 1, torch.zeros_like(wi), s_d, Bq=Bq)
+    sparse = salad.salad_sparse_attn_fwd(qd, kd, vd, rp_d, ci_d, 1, Bq=Bq)
+    assert torch.equal(zero, sparse)
+    # the drop threshold
+    drop = salad.salad_fused_proj_fwd(qd, kd, vd, rp_d, ci_d, 1, wb.cuda(), s_d, Bq=Bq, drop_tau=2.0)
+    assert torch.equal(drop, sparse)
+
+
+def test_state_pass_as_its_own_call_on_a_side_stream(salad):
+    # the reductions of Eq. 3 on one stream, the attention call on another, ordered by an event: the same bits
+    # as the one-call path, and the state against the oracle
+    B, H, N, d = 2, 3, 3000, 128
+    q, k, v = rand_qkv(B, H, N, d, 41)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    rp, ci = random_csr(-(-N // 128), -(-N // 64), 6, lo=1, hi=12)
+    rp_d, ci_d = dev_csr(rp, ci)
+    lam = torch.rand(H, device="cuda"); s = torch.tensor([0.3, 0.8], device="cuda")
+    whole = salad.salad_fused_fwd(qd, kd, vd, rp_d, ci_d, 1, lam, s, drop_tau=0.5)
+    ws = salad.alloc_workspace(B, H, N, d)
+    kv = torch.empty((B, H, d, d), dtype=torch.float32, device="cuda"); z = torch.empty((B, H, d), dtype=torch.float32, device="cuda")
+    st1 = torch.ones(1, dtype=torch.int32, device="cuda"); st2 = torch.ones(1, dtype=torch.int32, device="cuda")
+    side, main = torch.cuda.Stream(), torch.cuda.current_stream()
+    side.wait_stream(main)
+    salad.salad_linear_state_fwd(kd, vd, ws, kv_out=kv, z_out=z, status=st1, stream=side)
+    done = torch.cuda.Event(); done.record(side)
+    main.wait_event(done)
+    out = salad.salad_fused_prepared_fwd(qd, kd, vd, rp_d, ci_d, 1, lam, s, ws, status=st2, drop_tau=0.5)
+    torch.cuda.synchronize()
+    assert int(st1.item()) == 0 and int(st2.item()) == 0
+    assert torch.equal(out, whole)
+    kv_ref, z_ref = orc.linear_state(f32(k), f32(v))
+    np.testing.assert_allclose(z.cpu().numpy(), z_ref, rtol=1e-4, atol=1e-3)
+    np.testing.assert_allclose(kv.cpu().numpy(), kv_ref, rtol=1e-3, atol=np.abs(kv_ref).max() * 1e-4)
+
+
 # ------------------------------------------------------------------------------ degenerate sizes
 
 @pytest.mark.parametrize("B,H,N,d,Bq", [
