@@ -342,30 +342,6 @@ def main():
     ms_per_step = total_ms_max / K
     value = flops_per_s / 1e12
 
-    # ---------------- sustained: the same call back to back for seconds, into the power cap
-    sustained = None
-    if args.sustained_seconds > 0:
-        n_sus = max(K, int(args.sustained_seconds * 1.1 / (total_ms / K * 1e-3)))
-        sus_sampler = ClockSampler(physical_gpu_index(local_rank))
-        barrier()
-        sus_sampler.start()
-        t_start.record()
-        for _ in range(n_sus):
-            step()
-        t_stop.record()
-        sus_sampler.sample()
-        barrier()
-        sus_sampler.stop_flag.set()
-        sus_ms = dist_util.max_over_ranks(t_start.elapsed_time(t_stop), dev)
-        sus_tflops = flops / (sus_ms / n_sus * 1e-3) / 1e12           # per GPU
-        clk = sus_sampler.result()
-        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
-                     "tflops_per_gpu": sus_tflops, "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"],
-                     "peak": peaks.get("bf16_tflops_sustained"),
-                     "frac_of_measured_bf16_sustained": (sus_tflops / peaks["bf16_tflops_sustained"]
-                                                         if peaks.get("bf16_tflops_sustained") else None),
-                     "frac_of_measured_bf16_burst": sus_tflops / peaks["bf16_tflops"]}
-
     # ---------------- end to end: host buffers in, host buffer out, every step.
     # Every step copies its Q, K, V from pinned host memory and its O back.  The copies of neighbouring
     # steps overlap the compute of the current one: two sets of device buffers, one stream each for
@@ -534,6 +510,31 @@ def main():
         extras["rope_linear_branch"] = {"fused_ms": rope_ms, "fused_tflops": flops / (rope_ms * 1e-3) / 1e12,
                                         "extra_ms_over_plain_call": rope_ms - ms_per_step,
                                         "linear_only_ms": rope_lin_ms}
+
+    # ---------------- sustained: the same call back to back for seconds, into the power cap (after everything
+    # else, so that the short measurements above are taken at the clock a short call sees)
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(K, int(args.sustained_seconds * 1.1 / (total_ms / K * 1e-3)))
+        sus_sampler = ClockSampler(physical_gpu_index(local_rank))
+        barrier()
+        sus_sampler.start()
+        t_start.record()
+        for _ in range(n_sus):
+            step()
+        t_stop.record()
+        sus_sampler.sample()
+        barrier()
+        sus_sampler.stop_flag.set()
+        sus_ms = dist_util.max_over_ranks(t_start.elapsed_time(t_stop), dev)
+        sus_tflops = flops / (sus_ms / n_sus * 1e-3) / 1e12           # per GPU
+        clk = sus_sampler.result()
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "tflops_per_gpu": sus_tflops, "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"],
+                     "peak": peaks.get("bf16_tflops_sustained"),
+                     "frac_of_measured_bf16_sustained": (sus_tflops / peaks["bf16_tflops_sustained"]
+                                                         if peaks.get("bf16_tflops_sustained") else None),
+                     "frac_of_measured_bf16_burst": sus_tflops / peaks["bf16_tflops"]}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -315,6 +315,40 @@ int salad_permute_tokens(const void* x, void* y, int B, int H, int N, int d, int
                          const int32_t* h_head_flags, int inverse, void* stream);
 
 /*
+ * salad_fused_stswa_fwd -- the paper's own ST-SWA (Appendix A.1) in one call, without re-ordering passes:
+ * every head gets a 1-D sliding-window mask on ITS token order, which for heads with temporal locality
+ * (h_head_flags[h] != 0) is the order that groups tokens by spatial position, m = s*T + t for token
+ * n = t*(Hs*Ws) + s.  Such a head reads Q, K, V and writes O through 4-D tensor maps over the unchanged
+ * [B,H,N,d] tensors, in which the T tokens of a spatial position are one box row; nothing is permuted in
+ * memory, and the output arrives in the original token order.  Both branches are equivariant under the
+ * re-ordering, so the result equals salad_permute_tokens -> salad_fused_drop_fwd -> salad_permute_tokens
+ * (inverse) with the block sizes below.
+ *   Blocks.  Heads in token order: 128 query x 64 key tokens, as everywhere.  Temporal heads: a key block is
+ *   the T tokens of ks = floor(64 / T) consecutive spatial positions, a query block those of kq =
+ *   floor(128 / T) positions (T = 21: 63 and 126 tokens; the rest of the 64- / 128-row tiles is masked), so
+ *   that a block is a run of consecutive tokens of the re-ordered sequence.  T <= 64.
+ *   Lists.  Hm = H.  Every head owns `rows` = max(ceil(N/128), ceil(Hs*Ws/kq)) list rows (salad_stswa_blocks
+ *   returns rows, kq, ks and the number of key blocks of a temporal head); row h*rows + i is query block i of
+ *   head h, rows beyond a head's own blocks are empty; block ids refer to the head's own key blocks.
+ *   salad_stswa_mask_build makes the lists of the 1-D windows: h_windows[h] is the half-width of head h's
+ *   window in tokens of its own order (a block pair is kept iff some token pair lies within it).
+ *   Workspace: salad_stswa_workspace_bytes.  Other arguments as salad_fused_drop_fwd; d in {64, 128},
+ *   H <= 256.  The rotary variant is not available with re-ordered heads (SALAD_ERR_UNSUPPORTED).
+ */
+int salad_stswa_blocks(int T, int Hs, int Ws, int32_t* h_list_rows, int32_t* h_q_positions,
+                       int32_t* h_k_positions, int32_t* h_key_blocks);
+size_t salad_stswa_workspace_bytes(int B, int H, int T, int Hs, int Ws, int d);
+int salad_stswa_mask_build(int T, int Hs, int Ws, int H, const int32_t* h_head_flags,
+                           const int32_t* h_windows, int32_t* d_row_ptr, int32_t* d_col_idx,
+                           int64_t col_capacity, int64_t* h_nnz, void* stream);
+int salad_fused_stswa_fwd(const void* q, const void* k, const void* v, void* o,
+                          int B, int H, int N, int d, int T, int Hs, int Ws,
+                          const int32_t* h_head_flags, const int32_t* row_ptr, const int32_t* col_idx,
+                          const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                          float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                          int32_t* d_status, void* stream);
+
+/*
  * salad_proj_combine_fwd -- Algorithm 1 with the full Level-1 projection (Sec. 4.2): a linear layer
  * on the head-concatenated output of the linear branch (zero-initialised before tuning), scaled by
  * the dynamic factor and added to the sparse branch,

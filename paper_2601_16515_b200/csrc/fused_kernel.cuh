@@ -51,8 +51,22 @@ namespace salad {
 
 enum FusedMode { MODE_SPARSE = 1, MODE_LINEAR = 2, MODE_FUSED = 3 };
 
+// Heads with temporal locality (Appendix A.1): their tokens are taken in the order that groups them by spatial
+// position, m = s * T + t for token n = t * S + s, through 4-D tensor maps, without a re-ordering pass.  A
+// key block of such a head is the T tokens of ks spatial positions (ks * T <= 64 rows of the 64-row tile), a
+// query block those of kq positions (kq * T <= 128 rows); the unused rows of the tiles hold zeros and their
+// keys are masked.
+struct TemporalHeads {
+    int T, S;                    // T == 0: no head is re-ordered
+    int kq, ks;                  // spatial positions per query / key block
+    int nQb, nKb;                // blocks per head: ceil(S / kq), ceil(S / ks)
+    uint32_t flags[8];           // bit h: head h is temporal (H <= 256)
+};
+
 struct FusedParams {
-    int N, H, nQb, nKb, Bq, Hm, mode;
+    int N, H, nQb, nKb, Bq, Hm, mode;     // nQb: list rows per mask head; nKb: key blocks of a head in token order
+    int nQb_tok;                 // query blocks of a head in token order (== nQb unless temporal heads have more)
+    TemporalHeads th;
     const int32_t* row_ptr;
     const int32_t* col_idx;
     const int32_t* order;        // [Hm][nQb] launch order of the query blocks, or null (identity)
@@ -104,7 +118,9 @@ template <int D>
 __global__ void __launch_bounds__(384, 2)
 salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
-                   const __grid_constant__ CUtensorMap map_st, const FusedParams p)
+                   const __grid_constant__ CUtensorMap map_st, const __grid_constant__ CUtensorMap map_q4,
+                   const __grid_constant__ CUtensorMap map_k4, const __grid_constant__ CUtensorMap map_v4,
+                   const __grid_constant__ CUtensorMap map_o4, const FusedParams p)
 {
     using C = FusedCfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -131,6 +147,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int h = bh % p.H, b = bh / p.H;
     const int hm = (p.Hm == 1) ? 0 : (p.Hm == p.H ? h : bh);   // one mask, one per head, or one per (batch, head)
     const int qb = p.order ? __ldg(p.order + size_t(hm) * p.nQb + rank) : rank;
+    // temporal head: blocks of spatial positions, fetched through the 4-D maps
+    const bool perm = p.th.T > 0 && ((p.th.flags[h >> 5] >> (h & 31)) & 1u);
+    const int q_rows = perm ? p.th.kq * p.th.T : p.Bq;          // rows of the 128-row tile that hold queries
+    const int k_rows = perm ? p.th.ks * p.th.T : C::BK;         // rows of a 64-row tile that hold keys
+    if (qb >= (perm ? p.th.nQb : p.nQb_tok)) return;            // (a list row beyond this head's blocks: whole CTA)
     const bool sparse = (p.mode & MODE_SPARSE) != 0;
     // post-tuning branch dropping (Sec. 4.3): no linear work at all for a dropped batch item
     const bool linear = (p.mode & MODE_LINEAR) != 0 &&
@@ -163,13 +184,19 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         fence_mbar_init();
     }
-    if (p.Bq < 128) {
-        // rows [Bq, 128) of the Q tile are never written by TMA: zero them so the unused
-        // half of the MMA tile holds finite numbers
-        for (int i = tid; i < C::CH * (128 - p.Bq) * 8; i += C::THREADS) {
-            const int chunk = i / ((128 - p.Bq) * 8), rest = i % ((128 - p.Bq) * 8);
-            *reinterpret_cast<uint4*>(smem + C::OFF_Q + chunk * C::Q_CHUNK + p.Bq * 128 + rest * 16) =
+    if (q_rows < 128 || k_rows < C::BK) {
+        // rows [q_rows, 128) of the Q tile and [k_rows, 64) of the K and V tiles are never written by TMA:
+        // zero them so that the unused part of an MMA tile holds finite numbers (zero keys are masked, zero
+        // value rows meet zero probabilities)
+        for (int i = tid; i < C::CH * (128 - q_rows) * 8; i += C::THREADS) {
+            const int chunk = i / ((128 - q_rows) * 8), rest = i % ((128 - q_rows) * 8);
+            *reinterpret_cast<uint4*>(smem + C::OFF_Q + chunk * C::Q_CHUNK + q_rows * 128 + rest * 16) =
                 make_uint4(0, 0, 0, 0);
+        }
+        const int per_tile = (C::BK - k_rows) * 8;                // 16-byte vectors per 64-row chunk of a K or V tile
+        for (int i = tid; i < (C::NK + C::NV) * C::CH * per_tile; i += C::THREADS) {
+            const int tile = i / per_tile, rest = i % per_tile;  // K: [chunk][stage], V: [stage][chunk]: all 8 KB apart
+            *reinterpret_cast<uint4*>(smem + C::OFF_K + tile * C::KV_CHUNK + k_rows * 128 + rest * 16) = make_uint4(0, 0, 0, 0);
         }
         fence_proxy_async_smem();
     }
@@ -200,9 +227,11 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // stages zeros in the Q tile without waiting for q_full, so nothing may land there.
             if (len > 0 || linear) {
                 const uint32_t bar = smem_u32(&bars.q_full);
-                mbar_arrive_expect_tx(bar, uint32_t(p.Bq) * D * 2);
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(s_base + C::OFF_Q + ch * C::Q_CHUNK, &map_q, bar, ch * 64, qb * p.Bq, bh);
+                mbar_arrive_expect_tx(bar, uint32_t(q_rows) * D * 2);
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    if (perm) tma_load_4d(s_base + C::OFF_Q + ch * C::Q_CHUNK, &map_q4, bar, ch * 64, 0, qb * p.th.kq, bh);
+                    else tma_load_3d(s_base + C::OFF_Q + ch * C::Q_CHUNK, &map_q, bar, ch * 64, qb * p.Bq, bh);
+                }
             }
             for (int t = 0; t < len; ++t) {
                 const int s = t % C::NK;
@@ -212,10 +241,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (!ok) break;
                 const int col = __ldg(p.col_idx + ls + t);
                 const uint32_t bar = smem_u32(&bars.k_full[s]);
-                mbar_arrive_expect_tx(bar, C::KV_BYTES);
-                for (int ch = 0; ch < C::CH; ++ch)       // chunk-major: the two stages of a chunk are adjacent
-                    tma_load_3d(s_base + C::OFF_K + ch * (C::NK * C::KV_CHUNK) + s * C::KV_CHUNK, &map_k, bar, ch * 64,
-                                col * C::BK, bh);
+                mbar_arrive_expect_tx(bar, uint32_t(k_rows) * D * 2);
+                for (int ch = 0; ch < C::CH; ++ch) {     // chunk-major: the two stages of a chunk are adjacent
+                    const uint32_t dst = s_base + C::OFF_K + ch * (C::NK * C::KV_CHUNK) + s * C::KV_CHUNK;
+                    if (perm) tma_load_4d(dst, &map_k4, bar, ch * 64, 0, col * p.th.ks, bh);
+                    else tma_load_3d(dst, &map_k, bar, ch * 64, col * C::BK, bh);
+                }
             }
         }
         if (linear) {
@@ -249,10 +280,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (t >= C::NV && !mbar_wait(smem_u32(&bars.pv_done[s]), ((t >> 1) - 1) & 1, abortp)) break;
                 const int col = __ldg(p.col_idx + ls + t);
                 const uint32_t bar = smem_u32(&bars.v_full[s]);
-                mbar_arrive_expect_tx(bar, C::KV_BYTES);
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_load_3d(s_base + C::OFF_V + s * C::KV_BYTES + ch * C::KV_CHUNK, &map_v, bar, ch * 64,
-                                col * C::BK, bh);
+                mbar_arrive_expect_tx(bar, uint32_t(k_rows) * D * 2);
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    const uint32_t dst = s_base + C::OFF_V + s * C::KV_BYTES + ch * C::KV_CHUNK;
+                    if (perm) tma_load_4d(dst, &map_v4, bar, ch * 64, 0, col * p.th.ks, bh);
+                    else tma_load_3d(dst, &map_v, bar, ch * 64, col * C::BK, bh);
+                }
             }
         }
     } else if (warp == 2) {
@@ -363,8 +396,15 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // Only the last key block of the sequence can be short (N not a multiple of 64), and in an ascending
         // list it can only be the last entry: one look at that entry, before the loop, settles which block
         // needs its missing keys masked.
-        const int valid_last = (len > 0 && (p.N % C::BK) != 0 && __ldg(p.col_idx + le - 1) == p.nKb - 1)
-                                   ? p.N - (p.nKb - 1) * C::BK : C::BK;
+        // (A temporal head: every block holds ks * T keys, the last one those of the positions that exist.)
+        int valid_last = k_rows;
+        if (len > 0) {
+            if (perm) {
+                if (__ldg(p.col_idx + le - 1) == p.th.nKb - 1) valid_last = (p.th.S - (p.th.nKb - 1) * p.th.ks) * p.th.T;
+            } else if ((p.N % C::BK) != 0 && __ldg(p.col_idx + le - 1) == p.nKb - 1) {
+                valid_last = p.N - (p.nKb - 1) * C::BK;
+            }
+        }
         for (int t = 0; t < len && ok; ++t) {
             ok = wait_uniform(&bars.s_full[t & 1], (t >> 1) & 1);
             if (!ok) break;
@@ -374,8 +414,8 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_ld_16x256b_x8(t_tile + C::COL_SP + (t & 1) * C::SP_STRIDE, xr);
             tmem_wait_ld();
             float* x = reinterpret_cast<float*>(xr);
-            if (valid_last < C::BK && t + 1 == len) {         // keys of this block that exist
-                const int valid = valid_last;
+            const int valid = (t + 1 == len) ? valid_last : k_rows;      // keys of this block that exist
+            if (valid < C::BK) {
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     const int key = 8 * n + 2 * q4;
@@ -559,9 +599,10 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bars.out_staged));
             if (ra == 0 && q4 == 0 && mbar_wait(smem_u32(&bars.out_staged), 0, abortp)) {
-                for (int ch = 0; ch < C::CH; ++ch)
-                    tma_store_3d(&map_o, s_base + C::OFF_Q + ch * C::Q_CHUNK, ch * 64,
-                                 qb * p.Bq, bh);
+                for (int ch = 0; ch < C::CH; ++ch) {
+                    if (perm) tma_store_4d(&map_o4, s_base + C::OFF_Q + ch * C::Q_CHUNK, ch * 64, 0, qb * p.th.kq, bh);
+                    else tma_store_3d(&map_o, s_base + C::OFF_Q + ch * C::Q_CHUNK, ch * 64, qb * p.Bq, bh);
+                }
                 tma_store_commit();
                 // only the shared-memory source must have been read before the CTA may exit; the
                 // writes are complete, like all of the kernel's, when the grid is
@@ -571,8 +612,12 @@ salad_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int e2 = 0; e2 < 2; ++e2) {
                     const int row = e2 ? rb : ra;
-                    const int n = qb * p.Bq + row;
-                    if (row < p.Bq && n < p.N)
+                    int n = qb * p.Bq + row;
+                    if (perm) {                      // row = position within the block * T + frame
+                        const int sp = qb * p.th.kq + row / p.th.T;
+                        n = (sp < p.th.S) ? (row % p.th.T) * p.th.S + sp : p.N;
+                    }
+                    if (row < q_rows && n < p.N)
                         p.lse[size_t(bh) * p.N + n] =
                             (len > 0) ? ((e2 ? m_b : m_a) + log2f(e2 ? lt_b : lt_a)) * 0.6931471805599453f : -INFINITY;
                 }

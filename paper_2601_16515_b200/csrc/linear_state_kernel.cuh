@@ -290,16 +290,14 @@ salad_linear_state_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 }
 
 // Sum the partials of each head in chunk order; emit
-//   kv_out  fp32 [BH][D][D]  (optional; kv_ws: a second, workspace copy for the projection kernel)
-//   z       fp32 [BH][D]  (+ optional user copy)
+//   kv_out  fp32 [BH][D][D]  (optional)      z fp32 [BH][D]  (+ optional user copy)
 //   kvt     bf16 [BH][D][D]  transposed: kvt[c][a] = KV[a][c], the K-major B operand of
 //           num = ReLU(Q) KV in the fused kernel.
 template <int D, int ROWS>
 __global__ void __launch_bounds__(32 * ROWS)
 salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
-                             float* __restrict__ kv_out, float* __restrict__ kv_ws, float* __restrict__ z_ws,
-                             float* __restrict__ z_out, __nv_bfloat16* __restrict__ kvt,
-                             const float* __restrict__ dyn_scale, float drop_tau, int H)
+                             float* __restrict__ kv_out, float* __restrict__ z_ws, float* __restrict__ z_out,
+                             __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
     // The kernel after this one may be placed at once (it waits for this one before it touches the
     // state).  In fused calls ROWS = 8: a block is small, 256 threads and few registers, so that while it
@@ -335,7 +333,6 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
         }
         const float s = (s0 + s1) + (s2 + s3);
         if (kv_out) kv_out[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;
-        if (kv_ws) kv_ws[size_t(bh) * D * D + size_t(a) * D + c0 + tx] = s;        // for the projection kernel below
         tile[ty + ROWS * r][tx] = s;
     }
     __syncthreads();
@@ -353,43 +350,97 @@ salad_linear_finalize_kernel(const float* __restrict__ kv_part, const float* __r
     }
 }
 
-// Block-diagonal Level-1 projection (Algorithm 1; Sec. 4.2), folded into the linear state: with one d x d
-// block W_h per head on the linear branch,
+// The finalize step with a block-diagonal Level-1 projection (Algorithm 1; Sec. 4.2) folded into the linear
+// state: with one d x d block W_h per head on the linear branch,
 //     W_h (ReLU(Q_n) KV)^T = (KV W_h^T)^T ReLU(Q_n)^T ,   i.e.   num' = ReLU(Q_n) KV'  with  KV' = KV W_h^T,
 // so projecting the state once per head (a d x d x d product) projects every output row for free; the
-// normaliser Z is applied before the projection and stays as it is.  This kernel overwrites the bf16
-// transposed state the attention kernel multiplies with:
-//     kvt[c][a'] = KV'[a'][c] = sum_a KV[a'][a] * W_h[c][a]
-// from the fp32 state kv_ws[BH][D][D] and w[H][D][D] (bf16, W_h[c_out][a_in]), in fp32, one rounding.
-// grid (D/32, D/32, BH), 256 threads: a 32 (c) x 32 (a') tile per block, operands through shared memory.
+// normaliser Z is applied before the projection and stays as it is.  The bf16 transposed state the attention
+// kernel multiplies with becomes
+//     kvt[c][a'] = KV'[a'][c] = sum_a KV[a'][a] * W_h[c][a] ,
+// KV summed from the partials in chunk order as in the plain finalize kernel, w [H][D][D] bf16 = W_h[c_out][a_in],
+// fp32 arithmetic, one rounding.  kv_out (optional) receives the un-projected fp32 state.
+// grid (D/8, BH), 256 threads: a block owns eight rows a' of the state.  It sums them from the partials once
+// (every load issued before the first add: one L2 round trip) and keeps them in shared memory; a thread then
+// forms the outputs of one output channel c for some of the rows, reading row c of W_h straight from memory
+// (32 channels = four 16-byte vectors at a time, the next four fetched while the current ones are used).
+// Blocks of this kernel wait on every SM while the state kernel runs, next to a CTA of the attention kernel
+// that has started early: 4 KB of shared memory and few registers, so that all three fit.
 template <int D>
 __global__ void __launch_bounds__(256)
-salad_state_project_kernel(const float* __restrict__ kv_ws, const __nv_bfloat16* __restrict__ w,
-                           __nv_bfloat16* __restrict__ kvt, const float* __restrict__ dyn_scale, float drop_tau, int H)
+salad_linear_finalize_proj_kernel(const float* __restrict__ kv_part, const float* __restrict__ z_part, int chunks,
+                                  const __nv_bfloat16* __restrict__ w, float* __restrict__ kv_out,
+                                  float* __restrict__ z_ws, float* __restrict__ z_out, __nv_bfloat16* __restrict__ kvt,
+                                  const float* __restrict__ dyn_scale, float drop_tau, int H)
 {
     grid_launch_dependents();
     grid_dependency_wait();
-    const int bh = blockIdx.z;
+    const int bh = blockIdx.y, a0 = blockIdx.x * 8, tid = threadIdx.x;
     if (branch_dropped(dyn_scale, drop_tau, bh / H)) return;
-    __shared__ float ws[32][D + 1], ks[32][D + 1];
-    const int c0 = blockIdx.x * 32, a0 = blockIdx.y * 32;
-    const int tid = threadIdx.x;
-    const __nv_bfloat16* wh = w + size_t(bh % H) * D * D;
-    const float* kvh = kv_ws + size_t(bh) * D * D;
-    for (int i = tid; i < 32 * D; i += 256) {
-        const int r = i / D, a = i % D;
-        ws[r][a] = __bfloat162float(wh[size_t(c0 + r) * D + a]);
-        ks[r][a] = kvh[size_t(a0 + r) * D + a];
+    __shared__ float ks[8][D + 4];
+    {
+        // the eight rows of KV: D * 8 / 256 elements per thread, the partials of the head in chunk order
+        constexpr int EPT = D * 8 / 256;
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+            const int idx = tid + 256 * e, r = idx / D, a = idx % D;
+            const float* src = kv_part + size_t(bh) * chunks * D * D + size_t(a0 + r) * D + a;
+            float s0 = 0.f, s1 = 0.f;
+            for (int ch0 = 0; ch0 < chunks; ch0 += 16) {
+                float pv[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pv[j] = (ch0 + j < chunks) ? src[size_t(ch0 + j) * D * D] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) { s0 += pv[j]; s1 += pv[j + 1]; }
+            }
+            ks[r][a] = s0 + s1;
+            if (kv_out) kv_out[size_t(bh) * D * D + size_t(a0 + r) * D + a] = s0 + s1;
+        }
     }
     __syncthreads();
-    const int ap = tid % 32;                         // a' within the tile: consecutive threads, consecutive bf16
+    // outputs of this thread: c = tid % D, rows a' = a0 + OPT * (tid / D) + (0 .. OPT-1)
+    constexpr int OPT = D * 8 / 256;
+    const int c = tid % D, r0 = (tid / D) * OPT;
+    const uint4* wrow = reinterpret_cast<const uint4*>(w + (size_t(bh % H) * D + c) * D);     // row c of W_h: D bf16
+    float acc[OPT];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const int c = tid / 32 + 8 * u;
-        float acc = 0.f;
-#pragma unroll 8
-        for (int a = 0; a < D; ++a) acc = fmaf(ks[ap][a], ws[c][a], acc);
-        kvt[size_t(bh) * D * D + size_t(c0 + c) * D + a0 + ap] = __float2bfloat16(acc);
+    for (int j = 0; j < OPT; ++j) acc[j] = 0.f;
+    uint4 cur[4], nxt[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) cur[u] = __ldg(wrow + u);
+#pragma unroll
+    for (int k0 = 0; k0 < D; k0 += 32) {
+        if (k0 + 32 < D) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) nxt[u] = __ldg(wrow + (k0 + 32) / 8 + u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&cur[u]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 wv = __bfloat1622float2(h2[e]);
+                const int a = k0 + u * 8 + e * 2;
+#pragma unroll
+                for (int j = 0; j < OPT; ++j) {
+                    acc[j] = fmaf(ks[r0 + j][a], wv.x, acc[j]);
+                    acc[j] = fmaf(ks[r0 + j][a + 1], wv.y, acc[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) cur[u] = nxt[u];
+    }
+#pragma unroll
+    for (int j = 0; j < OPT; ++j)
+        kvt[size_t(bh) * D * D + size_t(c) * D + a0 + r0 + j] = __float2bfloat16(acc[j]);
+    if (blockIdx.x == 0) {
+        for (int a = tid; a < D; a += 256) {
+            const float* src = z_part + size_t(bh) * chunks * D + a;
+            float sum = 0.f;
+            for (int ch = 0; ch < chunks; ++ch) sum += src[size_t(ch) * D];
+            z_ws[size_t(bh) * D + a] = sum;
+            if (z_out) z_out[size_t(bh) * D + a] = sum;
+        }
     }
 }
 

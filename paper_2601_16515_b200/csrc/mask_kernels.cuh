@@ -17,17 +17,22 @@ namespace salad {
 
 struct MaskGeom {
     int T, Hs, Ws, N, Bq, Bk, nQb, nKb, Hm;
+    // second block geometry, used by the mask heads whose bit is set in MaskWindows::alt (the heads with
+    // temporal locality of salad_stswa_mask_build: blocks of whole spatial positions); nQb stays the number of
+    // list rows per mask head, rows beyond a head's own blocks are empty
+    int Bq2, Bk2, nQb2, nKb2, nQb1;     // nQb1: query blocks of the heads that use (Bq, Bk)
 };
 
 // Window sizes (wt, wh, ww) per mask head, passed by value as a kernel argument so that the
 // builder needs no device scratch.
 struct MaskWindows {
     int32_t w[3 * 256];
+    uint32_t alt[8];          // bit hm: mask head hm uses the second block geometry
 };
 
-__device__ __forceinline__ bool block_pair_kept(const MaskGeom& g, int i, int j, int wt, int wh, int ww) {
-    const int q0 = i * g.Bq, q1 = min(g.N, q0 + g.Bq) - 1;    // inclusive token ranges
-    const int k0 = j * g.Bk, k1 = min(g.N, k0 + g.Bk) - 1;
+__device__ __forceinline__ bool block_pair_kept(const MaskGeom& g, int Bq, int Bk, int i, int j, int wt, int wh, int ww) {
+    const int q0 = i * Bq, q1 = min(g.N, q0 + Bq) - 1;    // inclusive token ranges
+    const int k0 = j * Bk, k1 = min(g.N, k0 + Bk) - 1;
     const int qrow0 = q0 / g.Ws, qrow1 = q1 / g.Ws;            // grid rows (t*Hs + h) touched
     const int krow0 = k0 / g.Ws, krow1 = k1 / g.Ws;
     for (int r = qrow0; r <= qrow1; ++r) {
@@ -56,11 +61,14 @@ __global__ void __launch_bounds__(256) mask_rows_kernel(const MaskGeom g, const 
     if (warp >= rows) return;
     const int hm = warp / g.nQb, i = warp - hm * g.nQb;
     const int wt = windows.w[3 * hm], wh = windows.w[3 * hm + 1], ww = windows.w[3 * hm + 2];
+    const bool alt = (windows.alt[(hm >> 5) & 7] >> (hm & 31)) & 1u;
+    const int Bq = alt ? g.Bq2 : g.Bq, Bk = alt ? g.Bk2 : g.Bk;
+    const int nKb = alt ? g.nKb2 : g.nKb, nQb_own = alt ? g.nQb2 : g.nQb1;
     int base = FILL ? row_ptr[warp] : 0;
     int count = 0;
-    for (int j0 = 0; j0 < g.nKb; j0 += 32) {
+    for (int j0 = 0; j0 < nKb && i < nQb_own; j0 += 32) {
         const int j = j0 + lane;
-        const bool keep = (j < g.nKb) && block_pair_kept(g, i, j, wt, wh, ww);
+        const bool keep = (j < nKb) && block_pair_kept(g, Bq, Bk, i, j, wt, wh, ww);
         const unsigned m = __ballot_sync(0xffffffffu, keep);
         if (FILL && keep) col_idx[base + count + __popc(m & ((1u << lane) - 1u))] = j;
         count += __popc(m);

@@ -52,14 +52,15 @@ inline void record_profile(int idx, cudaStream_t st) {
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
-    size_t off_status, off_kvt, off_z, off_kvp, off_zp, off_order, off_kvf, total;
+    size_t off_status, off_kvt, off_z, off_kvp, off_zp, off_order, total;
     int slots;
 };
 
-Workspace carve(int B, int H, int N, int d, int Bq) {
+Workspace carve(int B, int H, int N, int d, int Bq, int list_rows = 0) {
     Workspace w;
     const size_t BH = size_t(B) * H;
-    const size_t nItems = size_t(N + Bq - 1) / Bq;                 // work items of the attention kernel: query blocks
+    // work items of the attention kernel: query blocks (list rows per head, when a caller's lists have more)
+    const size_t nItems = list_rows > 0 ? size_t(list_rows) : size_t(N + Bq - 1) / Bq;
     w.slots = int(BH > size_t(kPartialSlots) ? BH : size_t(kPartialSlots));
     w.off_status = 0;
     w.off_kvt = kAlign;
@@ -67,8 +68,7 @@ Workspace carve(int B, int H, int N, int d, int Bq) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = w.off_zp + align_up(size_t(w.slots) * d * 4);
-    w.off_kvf = w.off_order + align_up(BH * nItems * 4);            // launch order, per mask (at most B*H)
-    w.total = w.off_kvf + align_up(BH * d * d * 4);                 // fp32 state, for the block projection
+    w.total = w.off_order + align_up(BH * nItems * 4);              // launch order, per mask (at most B*H)
     return w;
 }
 
@@ -182,6 +182,19 @@ int check_launch() {
     return cudaGetLastError() == cudaSuccess ? SALAD_OK : SALAD_ERR_CUDA;
 }
 
+// The temporal-head block geometry of a T x Hs x Ws grid: blocks of whole spatial positions.
+struct StswaGeom { int S, kq, ks, nQb_p, nKb_p, nQb_tok, nKb_tok, rows; };
+bool stswa_geometry(int T, int Hs, int Ws, StswaGeom* o) {
+    if (T <= 0 || Hs <= 0 || Ws <= 0 || T > 64) return false;
+    const int64_t S = int64_t(Hs) * Ws, N = S * T;
+    if (N > 2147483647ll / 2) return false;
+    o->S = int(S); o->kq = 128 / T; o->ks = 64 / T;
+    o->nQb_p = int((S + o->kq - 1) / o->kq); o->nKb_p = int((S + o->ks - 1) / o->ks);
+    o->nQb_tok = int((N + 127) / 128); o->nKb_tok = int((N + 63) / 64);
+    o->rows = o->nQb_p > o->nQb_tok ? o->nQb_p : o->nQb_tok;
+    return true;
+}
+
 struct Problem {
     const void *q, *k, *v; void* o; float* lse;
     int B, H, N, d, Bq, Bk, Hm, mode;
@@ -191,6 +204,8 @@ struct Problem {
     float *kv_out, *z_out;
     const void* rope;             // fp16 [N, d/2, 2] cosine and sine per token and channel pair, or null
     const void* proj_blocks;      // bf16 [H, d, d]: one projection block per head on the linear branch, or null
+    int st_T, st_Hs, st_Ws;       // salad_fused_stswa_fwd: the latent grid (st_T == 0 otherwise) ...
+    const int32_t* st_flags;      // ... and the host flags of the heads with temporal locality
     bool state_only;              // salad_linear_state_fwd: the two reductions of Eq. 3 and nothing else
     bool prepared;                // salad_fused_prepared_fwd: the workspace already holds the linear state
     void* ws; size_t ws_bytes; int32_t* d_status; cudaStream_t stream;
@@ -218,10 +233,23 @@ int validate(const Problem& P) {
     }
     if (P.mode == MODE_FUSED && ((!P.static_scale && !P.proj_blocks) || !P.dyn_scale)) return SALAD_ERR_INVALID_ARG;
     if (P.proj_blocks && !aligned16(P.proj_blocks)) return SALAD_ERR_INVALID_ARG;
-    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
+    int list_rows = 0;
+    if (P.st_T > 0) {
+        StswaGeom sg;
+        if (!P.st_flags || int64_t(P.st_T) * P.st_Hs * P.st_Ws != P.N) return SALAD_ERR_INVALID_ARG;
+        if (!stswa_geometry(P.st_T, P.st_Hs, P.st_Ws, &sg) || P.H > 256 || P.Bq != 128 || P.rope) return SALAD_ERR_UNSUPPORTED;
+        if (P.Hm != P.H) return SALAD_ERR_INVALID_ARG;
+        list_rows = sg.rows;
+    }
+    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq, list_rows);
     if (!P.ws || (reinterpret_cast<uintptr_t>(P.ws) % kAlign) != 0 || P.ws_bytes < w.total)
         return SALAD_ERR_WORKSPACE;
     return SALAD_OK;
+}
+
+int list_rows_of(const Problem& P) {
+    StswaGeom sg;
+    return (P.st_T > 0 && stswa_geometry(P.st_T, P.st_Hs, P.st_Ws, &sg)) ? sg.rows : 0;
 }
 
 template <int D>
@@ -271,20 +299,16 @@ int launch_state(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     float* z_ws = reinterpret_cast<float*>(ws + w.off_z);
     __nv_bfloat16* kvt = reinterpret_cast<__nv_bfloat16*>(ws + w.off_kvt);
-    float* kv_ws = P.proj_blocks ? reinterpret_cast<float*>(ws + w.off_kvf) : nullptr;
-    if ((P.mode & MODE_SPARSE) && !P.rope)
+    if (P.proj_blocks)      // block-diagonal projection folded into the state: the attention kernel multiplies with KV W_h^T
+        launch_dependent(salad_linear_finalize_proj_kernel<D>, dim3(D / 8, BH), dim3(256), 0, P.stream,
+                         sp.kv_part, sp.z_part, chunks, static_cast<const __nv_bfloat16*>(P.proj_blocks), P.kv_out, z_ws,
+                         P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+    else if ((P.mode & MODE_SPARSE) && !P.rope)
         launch_dependent(salad_linear_finalize_kernel<D, 8>, dim3(D / 32, D / 32, BH), dim3(32, 8), 0, P.stream,
-                         sp.kv_part, sp.z_part, chunks, P.kv_out, kv_ws, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
     else
         launch_dependent(salad_linear_finalize_kernel<D, 32>, dim3(D / 32, D / 32, BH), dim3(32, 32), 0, P.stream,
-                         sp.kv_part, sp.z_part, chunks, P.kv_out, kv_ws, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
-    if (P.proj_blocks) {
-        // block-diagonal projection folded into the state: the attention kernel multiplies with KV W_h^T
-        if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-        SALAD_LOGF("salad_state_project_kernel<%d> grid (%d, %d, %d)", D, D / 32, D / 32, BH);
-        launch_dependent(salad_state_project_kernel<D>, dim3(D / 32, D / 32, BH), dim3(256), 0, P.stream, kv_ws,
-                         static_cast<const __nv_bfloat16*>(P.proj_blocks), kvt, P.dyn_scale, P.drop_tau, P.H);
-    }
+                         sp.kv_part, sp.z_part, chunks, P.kv_out, z_ws, P.z_out, kvt, P.dyn_scale, P.drop_tau, P.H);
     record_profile(1, P.stream);
     return check_launch();
 }
@@ -302,6 +326,23 @@ int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     fp.N = P.N; fp.H = P.H; fp.Bq = P.Bq; fp.Hm = P.Hm; fp.mode = P.mode;
     fp.nQb = (P.N + P.Bq - 1) / P.Bq;
     fp.nKb = (P.N + 63) / 64;
+    fp.nQb_tok = fp.nQb;
+    fp.th = TemporalHeads{};
+    CUtensorMap mq4 = mq, mk4 = mk, mv4 = mv, mo4 = mo;        // unused without temporal heads
+    if (P.st_T > 0) {
+        // heads with temporal locality read and write their tokens grouped by spatial position through 4-D maps
+        StswaGeom sg;
+        stswa_geometry(P.st_T, P.st_Hs, P.st_Ws, &sg);
+        fp.th.T = P.st_T; fp.th.S = sg.S; fp.th.kq = sg.kq; fp.th.ks = sg.ks; fp.th.nQb = sg.nQb_p; fp.th.nKb = sg.nKb_p;
+        for (int h = 0; h < P.H; ++h)
+            if (P.st_flags[h]) fp.th.flags[h >> 5] |= 1u << (h & 31);
+        fp.nQb = sg.rows;
+        if (!make_tmap_bf16_4d_by_position(&mq4, P.q, D, P.st_T, sg.S, BH, sg.kq) ||
+            !make_tmap_bf16_4d_by_position(&mk4, P.k, D, P.st_T, sg.S, BH, sg.ks) ||
+            !make_tmap_bf16_4d_by_position(&mv4, P.v, D, P.st_T, sg.S, BH, sg.ks) ||
+            !make_tmap_bf16_4d_by_position(&mo4, P.o, D, P.st_T, sg.S, BH, sg.kq))
+            return SALAD_ERR_CUDA;
+    }
     fp.row_ptr = P.row_ptr; fp.col_idx = P.col_idx;
     fp.BH = BH;
     fp.order = nullptr;
@@ -323,7 +364,7 @@ int launch_fused(const Problem& P, const Workspace& w, const DeviceInfo& dev) {
     SALAD_LOGF("salad_fused_kernel<%d> grid %lld block %d smem %d (mode %d)", D, (long long)grid, FusedCfg<D>::THREADS,
                FusedCfg<D>::SMEM_BYTES, P.mode);
     launch_dependent(salad_fused_kernel<D>, dim3(unsigned(grid)), dim3(FusedCfg<D>::THREADS),
-                     FusedCfg<D>::SMEM_BYTES, P.stream, mq, mk, mv, mo, ms, fp);
+                     FusedCfg<D>::SMEM_BYTES, P.stream, mq, mk, mv, mo, ms, mq4, mk4, mv4, mo4, fp);
     record_profile(3, P.stream);
     return check_launch();
 }
@@ -384,17 +425,20 @@ int run(const Problem& P) {
     DeviceInfo dev{};
     rc = prepare_device(&dev);
     if (rc != SALAD_OK) return rc;
-    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq);
+    const Workspace w = carve(P.B, P.H, P.N, P.d, P.Bq, list_rows_of(P));
     uint8_t* ws = static_cast<uint8_t*>(P.ws);
     if (P.mode & MODE_SPARSE) {
         // first kernel of the call: longest work items first (the mask is an input of every call,
         // so is its order); it also clears the status words
-        const int nQb = (P.N + P.Bq - 1) / P.Bq;
+        const int nQb = list_rows_of(P) > 0 ? list_rows_of(P) : (P.N + P.Bq - 1) / P.Bq;
         int32_t* ws_status = reinterpret_cast<int32_t*>(ws + w.off_status);
         int clear_status = 1;
         if (g_validate_capacity > 0) {
             // opt-in check of the lists (salad_set_mask_validation): it owns the status words of this call
-            rc = launch_csr_validate(P.row_ptr, P.col_idx, g_validate_capacity, int64_t(P.Hm) * nQb, (P.N + 63) / 64,
+            int nkb_bound = (P.N + 63) / 64;
+            StswaGeom sg;                      // temporal heads have their own key-block count: the larger bounds both
+            if (P.st_T > 0 && stswa_geometry(P.st_T, P.st_Hs, P.st_Ws, &sg) && sg.nKb_p > nkb_bound) nkb_bound = sg.nKb_p;
+            rc = launch_csr_validate(P.row_ptr, P.col_idx, g_validate_capacity, int64_t(P.Hm) * nQb, nkb_bound,
                                      ws_status, P.d_status, P.stream);
             if (rc != SALAD_OK) return rc;
             clear_status = 0;
@@ -445,7 +489,6 @@ Workspace carve_noalloc(int B, int H, int d) {
     w.off_kvp = w.off_z + align_up(BH * d * 4);
     w.off_zp = w.off_kvp + align_up(size_t(w.slots) * d * d * 4);
     w.off_order = 0;                                  // linear attention has no kept lists to order
-    w.off_kvf = 0;                                    // (no projection in the linear-only calls)
     w.total = w.off_zp + align_up(size_t(w.slots) * d * 4);
     return w;
 }
@@ -512,6 +555,9 @@ SALAD_EXPORT size_t salad_workspace_bytes(int B, int H, int N, int d, int Bq, in
     return carve(B, H, N, d, Bq).total;
 }
 
+int build_mask_lists(MaskGeom g, const int32_t* h_windows, const uint32_t* alt_bits, int32_t* d_row_ptr,
+                     int32_t* d_col_idx, int64_t col_capacity, int64_t* h_nnz, void* stream);
+
 SALAD_EXPORT int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm, const int32_t* h_windows,
                                   int32_t* d_row_ptr, int32_t* d_col_idx, int64_t col_capacity,
                                   int64_t* h_nnz, void* stream) {
@@ -525,6 +571,14 @@ SALAD_EXPORT int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm,
     MaskGeom g;
     g.T = T; g.Hs = Hs; g.Ws = Ws; g.N = int(N64); g.Bq = Bq; g.Bk = Bk; g.Hm = Hm;
     g.nQb = (g.N + Bq - 1) / Bq; g.nKb = (g.N + Bk - 1) / Bk;
+    g.Bq2 = Bq; g.Bk2 = Bk; g.nQb2 = g.nQb; g.nKb2 = g.nKb; g.nQb1 = g.nQb;      // one geometry for every mask head
+    return build_mask_lists(g, h_windows, nullptr, d_row_ptr, d_col_idx, col_capacity, h_nnz, stream);
+}
+
+
+int build_mask_lists(MaskGeom g, const int32_t* h_windows, const uint32_t* alt_bits, int32_t* d_row_ptr,
+                     int32_t* d_col_idx, int64_t col_capacity, int64_t* h_nnz, void* stream) {
+    const int Hm = g.Hm;
     const int64_t rows64 = int64_t(Hm) * g.nQb;
     if (rows64 > (1 << 24)) return SALAD_ERR_UNSUPPORTED;
     const int rows = int(rows64);
@@ -534,6 +588,7 @@ SALAD_EXPORT int salad_mask_build(int T, int Hs, int Ws, int Bq, int Bk, int Hm,
     // row_ptr; row_ptr[rows] doubles as the overflow probe target before it is overwritten.
     MaskWindows win;
     for (int i = 0; i < 3 * kMaxMaskHeads; ++i) win.w[i] = (i < 3 * Hm) ? h_windows[i] : 0;
+    for (int i = 0; i < 8; ++i) win.alt[i] = alt_bits ? alt_bits[i] : 0u;
     const int blocks = (rows * 32 + 255) / 256;
     mask_rows_kernel<false><<<blocks, 256, 0, st>>>(g, win, d_row_ptr, nullptr);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
@@ -639,6 +694,67 @@ SALAD_EXPORT int salad_fused_prepared_fwd(const void* q, const void* k, const vo
     P.q = q; P.k = k; P.v = v; P.o = o;
     P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = Bq; P.Bk = Bk; P.Hm = Hm; P.mode = MODE_FUSED;
     P.prepared = true;
+    P.row_ptr = row_ptr; P.col_idx = col_idx;
+    P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
+    P.softmax_scale = softmax_scale; P.eps = eps;
+    P.ws = workspace; P.ws_bytes = workspace_bytes; P.d_status = d_status;
+    P.stream = static_cast<cudaStream_t>(stream);
+    return run(P);
+}
+
+SALAD_EXPORT int salad_stswa_blocks(int T, int Hs, int Ws, int32_t* h_list_rows, int32_t* h_q_positions,
+                                    int32_t* h_k_positions, int32_t* h_key_blocks) {
+    StswaGeom sg;
+    if (T <= 0 || Hs <= 0 || Ws <= 0) return SALAD_ERR_INVALID_ARG;
+    if (!stswa_geometry(T, Hs, Ws, &sg)) return SALAD_ERR_UNSUPPORTED;
+    if (h_list_rows) *h_list_rows = sg.rows;
+    if (h_q_positions) *h_q_positions = sg.kq;
+    if (h_k_positions) *h_k_positions = sg.ks;
+    if (h_key_blocks) *h_key_blocks = sg.nKb_p;
+    return SALAD_OK;
+}
+
+SALAD_EXPORT size_t salad_stswa_workspace_bytes(int B, int H, int T, int Hs, int Ws, int d) {
+    StswaGeom sg;
+    if (B <= 0 || H <= 0 || (d != 64 && d != 128) || !stswa_geometry(T, Hs, Ws, &sg)) return 0;
+    return carve(B, H, T * sg.S, d, 128, sg.rows).total;
+}
+
+SALAD_EXPORT int salad_stswa_mask_build(int T, int Hs, int Ws, int H, const int32_t* h_head_flags,
+                                        const int32_t* h_windows, int32_t* d_row_ptr, int32_t* d_col_idx,
+                                        int64_t col_capacity, int64_t* h_nnz, void* stream) {
+    if (T <= 0 || Hs <= 0 || Ws <= 0 || H <= 0 || !h_head_flags || !h_windows || !d_row_ptr) return SALAD_ERR_INVALID_ARG;
+    if (col_capacity < 0 || (d_col_idx == nullptr && col_capacity != 0)) return SALAD_ERR_INVALID_ARG;
+    StswaGeom sg;
+    if (H > kMaxMaskHeads || !stswa_geometry(T, Hs, Ws, &sg)) return SALAD_ERR_UNSUPPORTED;
+    for (int h = 0; h < H; ++h) if (h_windows[h] < 0) return SALAD_ERR_INVALID_ARG;
+    // a 1-D window on every head's own token order: the grid 1 x 1 x N, blocks of 128 x 64 tokens, or of the
+    // tokens of kq x ks whole spatial positions for the heads that take their tokens grouped by position
+    MaskGeom g;
+    g.T = 1; g.Hs = 1; g.Ws = T * sg.S; g.N = T * sg.S; g.Hm = H;
+    g.Bq = 128; g.Bk = 64; g.nQb1 = sg.nQb_tok; g.nKb = sg.nKb_tok;
+    g.Bq2 = sg.kq * T; g.Bk2 = sg.ks * T; g.nQb2 = sg.nQb_p; g.nKb2 = sg.nKb_p;
+    g.nQb = sg.rows;
+    int32_t win[3 * kMaxMaskHeads];
+    uint32_t alt[8] = {};
+    for (int h = 0; h < H; ++h) {
+        win[3 * h] = 0; win[3 * h + 1] = 0; win[3 * h + 2] = h_windows[h];
+        if (h_head_flags[h]) alt[h >> 5] |= 1u << (h & 31);
+    }
+    return build_mask_lists(g, win, alt, d_row_ptr, d_col_idx, col_capacity, h_nnz, stream);
+}
+
+SALAD_EXPORT int salad_fused_stswa_fwd(const void* q, const void* k, const void* v, void* o,
+                                       int B, int H, int N, int d, int T, int Hs, int Ws,
+                                       const int32_t* h_head_flags, const int32_t* row_ptr, const int32_t* col_idx,
+                                       const float* d_static_scale, const float* d_dyn_scale, float drop_tau,
+                                       float softmax_scale, float eps, void* workspace, size_t workspace_bytes,
+                                       int32_t* d_status, void* stream) {
+    if (isnan(drop_tau) || !h_head_flags || T <= 0 || Hs <= 0 || Ws <= 0) return SALAD_ERR_INVALID_ARG;
+    Problem P{};
+    P.q = q; P.k = k; P.v = v; P.o = o;
+    P.B = B; P.H = H; P.N = N; P.d = d; P.Bq = 128; P.Bk = 64; P.Hm = H; P.mode = MODE_FUSED;
+    P.st_T = T; P.st_Hs = Hs; P.st_Ws = Ws; P.st_flags = h_head_flags;
     P.row_ptr = row_ptr; P.col_idx = col_idx;
     P.static_scale = d_static_scale; P.dyn_scale = d_dyn_scale; P.drop_tau = drop_tau;
     P.softmax_scale = softmax_scale; P.eps = eps;

@@ -43,6 +43,25 @@ inline bool make_tmap_bf16_3d(CUtensorMap* out, const void* base, int d, int64_t
     return r == CUDA_SUCCESS;
 }
 
+// Map over the same bf16 tensor [outer, N, d] whose N = T * S tokens are numbered with time slowest
+// (n = t * S + s), seen as [outer, S, T, d]: a box of [1, box_s, T, 64] elements is box_s * T rows of 128
+// bytes in shared memory, row s_local * T + t -- the tokens of box_s spatial positions in the order that
+// groups tokens by spatial position (Appendix A.1), without the tensor being re-ordered in memory.
+// Spatial positions past S read as zero and are not written by stores.
+inline bool make_tmap_bf16_4d_by_position(CUtensorMap* out, const void* base, int d, int T, int64_t S,
+                                          int64_t outer, int box_s) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return false;
+    cuuint64_t dims[4] = {cuuint64_t(d), cuuint64_t(T), cuuint64_t(S), cuuint64_t(outer)};
+    cuuint64_t strides[3] = {cuuint64_t(S) * d * 2, cuuint64_t(d) * 2, cuuint64_t(T) * cuuint64_t(S) * d * 2};
+    cuuint32_t box[4] = {64, cuuint32_t(T), cuuint32_t(box_s), 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // Map over an fp16 matrix [rows, cols] (cols fastest, contiguous; cols <= 256).  One box is
 // [box_rows, cols], written to shared memory row after row without swizzle.  Rows past `rows`
 // read as zero.

@@ -31,7 +31,8 @@ EXPORTS = ("salad_status_string", "salad_workspace_bytes", "salad_mask_build",
            "salad_dynamic_scale", "salad_topk_workspace_bytes", "salad_topk_mask_build", "salad_permute_tokens", "salad_proj_combine_fwd",
            "salad_selftest_bounded_wait", "salad_fused_rope_fwd", "salad_linear_attn_rope_fwd",
            "salad_rope3d_table_build", "salad_csr_validate", "salad_set_mask_validation",
-           "salad_fused_proj_fwd", "salad_linear_state_fwd", "salad_fused_prepared_fwd")
+           "salad_fused_proj_fwd", "salad_linear_state_fwd", "salad_fused_prepared_fwd",
+           "salad_stswa_blocks", "salad_stswa_workspace_bytes", "salad_stswa_mask_build", "salad_fused_stswa_fwd")
 
 
 class SaladError(RuntimeError):
@@ -89,6 +90,14 @@ def _load() -> ctypes.CDLL:
     lib.salad_linear_state_fwd.argtypes = [p, p, p, p] + [i32] * 4 + [p, sz, p, p]
     lib.salad_fused_prepared_fwd.restype = i32
     lib.salad_fused_prepared_fwd.argtypes = [p, p, p, p] + [i32] * 6 + [p, p, i32, p, p, f32, f32, f32, p, sz, p, p]
+    lib.salad_stswa_blocks.restype = i32
+    lib.salad_stswa_blocks.argtypes = [i32, i32, i32, p, p, p, p]
+    lib.salad_stswa_workspace_bytes.restype = sz
+    lib.salad_stswa_workspace_bytes.argtypes = [i32] * 6
+    lib.salad_stswa_mask_build.restype = i32
+    lib.salad_stswa_mask_build.argtypes = [i32, i32, i32, i32, p, p, p, p, i64, p, p]
+    lib.salad_fused_stswa_fwd.restype = i32
+    lib.salad_fused_stswa_fwd.argtypes = [p, p, p, p] + [i32] * 7 + [p, p, p, p, p, f32, f32, f32, p, sz, p, p]
     lib.salad_csr_validate.restype = i32
     lib.salad_csr_validate.argtypes = [p, p, i64, i64, i32, p, p]
     lib.salad_set_mask_validation.restype = i32
@@ -409,6 +418,68 @@ def salad_permute_tokens(x, grid, head_flags, inverse: bool = False, out=None, s
     with torch.cuda.device(x.device):
         _check(_lib.salad_permute_tokens(_ptr(x), _ptr(out), B, H, N, d, T, Hs, Ws, flags, int(bool(inverse)),
                                          _stream(stream)), "salad_permute_tokens")
+    return out
+
+
+def salad_stswa_blocks(grid):
+    """Block geometry of salad_fused_stswa_fwd on a (T, Hs, Ws) grid: (list rows per head, spatial positions
+    per query block, per key block, key blocks of a temporal head)."""
+    T, Hs, Ws = grid
+    vals = [ctypes.c_int32(0) for _ in range(4)]
+    _check(_lib.salad_stswa_blocks(T, Hs, Ws, *[ctypes.byref(x) for x in vals]), "salad_stswa_blocks")
+    return tuple(int(x.value) for x in vals)
+
+
+def salad_stswa_mask_build(grid, head_flags, windows, device="cuda", stream=None):
+    """1-D sliding-window lists for salad_fused_stswa_fwd: windows[h] is the half-width of head h's window in
+    tokens of its own order (grouped by spatial position when head_flags[h]).  Returns (row_ptr, col_idx)."""
+    T, Hs, Ws = grid
+    H = len(head_flags)
+    rows = salad_stswa_blocks(grid)[0]
+    flags = (ctypes.c_int32 * H)(*[int(bool(f)) for f in head_flags])
+    win = (ctypes.c_int32 * H)(*[int(w) for w in windows])
+    row_ptr = torch.empty(H * rows + 1, dtype=torch.int32, device=device)
+    nnz = ctypes.c_int64(-1)
+    with torch.cuda.device(row_ptr.device):
+        _check(_lib.salad_stswa_mask_build(T, Hs, Ws, H, flags, win, _ptr(row_ptr), None, 0, ctypes.byref(nnz),
+                                           _stream(stream)), "salad_stswa_mask_build")
+        col_idx = torch.empty(max(1, nnz.value), dtype=torch.int32, device=device)
+        _check(_lib.salad_stswa_mask_build(T, Hs, Ws, H, flags, win, _ptr(row_ptr), _ptr(col_idx), col_idx.numel(),
+                                           ctypes.byref(nnz), _stream(stream)), "salad_stswa_mask_build")
+    return row_ptr, col_idx[:nnz.value]
+
+
+def salad_fused_stswa_fwd(q, k, v, grid, head_flags, row_ptr, col_idx, static_scale, dyn_scale, softmax_scale: float = 0.0,
+                          eps: float = 1e-6, out=None, workspace=None, status=None, stream=None,
+                          drop_tau: Optional[float] = None):
+    """The fused call with the paper's ST-SWA: flagged heads take their tokens grouped by spatial position through
+    the loads and stores themselves (no permutation pass); lists from salad_stswa_mask_build."""
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _bf16_4d(name, t)
+    if k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("q, k, v must have the same shape")
+    B, H, N, d = q.shape
+    T, Hs, Ws = grid
+    if len(head_flags) != H:
+        raise ValueError("head_flags must have one entry per head")
+    _i32("row_ptr", row_ptr); _i32("col_idx", col_idx)
+    for name, t, n in (("static_scale", static_scale, H), ("dyn_scale", dyn_scale, B)):
+        if t.dtype != torch.float32 or not t.is_cuda or t.numel() != n or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor with {n} elements")
+    flags = (ctypes.c_int32 * H)(*[int(bool(f)) for f in head_flags])
+    if workspace is None:
+        nbytes = int(_lib.salad_stswa_workspace_bytes(B, H, T, Hs, Ws, d))
+        if nbytes == 0:
+            raise SaladError(SALAD_ERR_UNSUPPORTED, "salad_stswa_workspace_bytes")
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty_like(q)
+    tau = float("-inf") if drop_tau is None else float(drop_tau)
+    with torch.cuda.device(q.device):
+        _check(_lib.salad_fused_stswa_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, d, T, Hs, Ws, flags,
+                                          _ptr(row_ptr), _ptr(col_idx), _ptr(static_scale), _ptr(dyn_scale), tau,
+                                          float(softmax_scale), float(eps), _ptr(workspace), workspace.numel(),
+                                          _ptr(status), _stream(stream)), "salad_fused_stswa_fwd")
     return out
 
 

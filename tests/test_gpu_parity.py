@@ -618,6 +618,57 @@ def test_permuted_sliding_window_pipeline(salad):
     assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "permuted ST-SWA")
 
 
+def _stswa_oracle(q, k, v, grid, flags, windows, lam, s, kq, ks):
+    """The oracle's ST-SWA pipeline: re-order the temporal heads, a 1-D window on every head's own order (blocks of
+    128 x 64 tokens, or of the tokens of kq x ks whole spatial positions), Algorithm 1, order restored."""
+    T = grid[0]
+    B, H, N, d = q.shape
+    qp, kp, vp = (orc.permute_tokens(f32(t), grid, flags) for t in (q, k, v))
+    ref_p = np.empty((B, H, N, d))
+    lists = {}
+    for h in range(H):
+        Bq, Bk = (kq * T, ks * T) if flags[h] else (128, 64)
+        rp, ci = orc.mask_build(1, 1, N, Bq, Bk, [(0, 0, windows[h])])
+        lists[h] = (rp, ci)
+        r = orc.salad_fused(qp[:, h:h + 1], kp[:, h:h + 1], vp[:, h:h + 1], Bq, Bk, rp, ci, 1,
+                            lam[h:h + 1].astype(np.float64), s.astype(np.float64))
+        ref_p[:, h] = r.reshape(B, N, d)
+    return orc.permute_tokens(ref_p, grid, flags, inverse=True), lists
+
+
+@pytest.mark.parametrize("grid,B,H,d,flags,windows", [
+    ((21, 6, 10), 1, 4, 128, [1, 0, 1, 0], [100, 200, 300, 90]),       # T = 21: blocks of 3 and 6 positions (63, 126 tokens)
+    ((8, 8, 16), 2, 3, 64, [0, 1, 1], [64, 130, 40]),                  # T = 8: 8 and 16 positions fill the tiles exactly
+    ((5, 7, 9), 1, 2, 128, [1, 1], [33, 400]),                         # 63 positions: ragged last blocks on both sides
+])
+def test_stswa_through_the_loads(salad, grid, B, H, d, flags, windows):
+    # The paper's ST-SWA with the re-ordering done by the loads and stores of the attention kernel: lists
+    # bit-exact against the oracle's 1-D window masks, output against the oracle's permute / attend / permute-back.
+    T, Hs, Ws = grid
+    N = T * Hs * Ws
+    q, k, v = rand_qkv(B, H, N, d, 1200 + N)
+    rng = np.random.default_rng(N)
+    lam = rng.uniform(0.2, 1, H).astype(np.float32); s = rng.uniform(0.2, 0.9, B).astype(np.float32)
+    rows, kq, ks, nkb_p = salad.salad_stswa_blocks(grid)
+    assert (kq, ks) == (128 // T, 64 // T)
+    rp_d, ci_d = salad.salad_stswa_mask_build(grid, flags, windows)
+    ref, lists = _stswa_oracle(q, k, v, grid, flags, windows, lam, s, kq, ks)
+    rp_g, ci_g = rp_d.cpu().numpy(), ci_d.cpu().numpy()
+    for h in range(H):
+        rp_o, ci_o = lists[h]
+        n_own = len(rp_o) - 1
+        got_rp = rp_g[h * rows:h * rows + n_own + 1] - rp_g[h * rows]
+        assert np.array_equal(got_rp, rp_o), h
+        assert np.array_equal(ci_g[rp_g[h * rows]:rp_g[h * rows + n_own]], ci_o), h
+        assert (np.diff(rp_g[h * rows + n_own:(h + 1) * rows + 1]) == 0).all()       # rows beyond the head's blocks: empty
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = torch.full_like(q.cuda(), 3.0)
+    salad.salad_fused_stswa_fwd(q.cuda(), k.cuda(), v.cuda(), grid, flags, rp_d, ci_d, torch.from_numpy(lam).cuda(),
+                                torch.from_numpy(s).cuda(), out=out, status=status)
+    status_ok(status)
+    assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "ST-SWA through the loads")
+
+
 # ------------------------------------------------------------------------------ full projection (Alg. 1 level 1)
 
 @pytest.mark.parametrize("B,H,N,d,with_bias", [

@@ -526,6 +526,38 @@ def test_proj_combine_block_diagonal_is_the_fused_path():
     np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
 
 
+def test_stswa_with_blocks_of_whole_spatial_positions():
+    # The reading behind salad_fused_stswa_fwd for heads with temporal locality (Appendix A.1): tokens grouped by
+    # spatial position, m = s*T + t; a key block = the T tokens of ks positions, a query block those of kq
+    # positions; a block pair is kept iff some token pair is within w of each other in the re-ordered sequence.
+    # The oracle's composition (permute, 1-D window mask with blocks of kq*T x ks*T tokens, Eq. 2, permute back)
+    # against the same thing written from first principles on (t, s) coordinates with a dense N x N mask.
+    T, Hs, Ws, kq, ks, w, d = 3, 2, 5, 2, 1, 4, 8
+    S, N = Hs * Ws, T * Hs * Ws
+    grid = (T, Hs, Ws)
+    q, k, v = rand_qkv(1, 1, N, d, 301)
+    qp, kp, vp = (orc.permute_tokens(t, grid, [1]) for t in (q, k, v))
+    rp, ci = orc.mask_build(1, 1, N, kq * T, ks * T, [(0, 0, w)])
+    o_p, _ = orc.sparse_attn(qp, kp, vp, kq * T, ks * T, rp, ci, 1)
+    got = orc.permute_tokens(o_p.reshape(1, 1, N, d), grid, [1], inverse=True)[0, 0]
+    # first principles: positions in the re-ordered sequence, block ids from spatial positions
+    n = np.arange(N); t, sp = n // S, n % S
+    m = sp * T + t
+    qblk, kblk = sp // kq, sp // ks
+    nQb, nKb = -(-S // kq), -(-S // ks)
+    kept = np.zeros((nQb, nKb), bool)
+    for a in range(N):
+        for b_ in range(N):
+            if abs(int(m[a]) - int(m[b_])) <= w:
+                kept[qblk[a], kblk[b_]] = True
+    allow = kept[qblk][:, kblk]                                 # [N, N] over original token ids
+    sc = (q[0, 0].astype(np.float64) @ k[0, 0].astype(np.float64).T) / np.sqrt(d)
+    sc = np.where(allow, sc, -np.inf)
+    p = np.exp(sc - sc.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
+    np.testing.assert_allclose(got, p @ v[0, 0].astype(np.float64), rtol=1e-10, atol=1e-12)
+    assert 0 < allow.mean() < 1                                 # a real mask, not all-kept
+
+
 def test_blockproj_pins():
     # One d x d projection block per head (Alg. 1 Level 1 without head mixing), pinned from both sides:
     # against the full projection with a block-diagonal weight, and against the per-head scalar.
