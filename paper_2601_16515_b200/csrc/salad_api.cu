@@ -153,6 +153,9 @@ int prepare_device(DeviceInfo* info) {
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      ProjCfg::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(salad_proj_gemm_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Proj2Cfg<256>::SMEM_BYTES);
         if (e != cudaSuccess) { cudaGetLastError(); return SALAD_ERR_CUDA; }
         sm_count[dev] = sms;
         attr_set[dev] = true;
@@ -969,7 +972,24 @@ SALAD_EXPORT int salad_proj_combine_fwd(const void* o_s, const void* o_l, const 
     pp.o_s = static_cast<const __nv_bfloat16*>(o_s);
     pp.out = static_cast<__nv_bfloat16*>(out);
     pp.bias = d_bias; pp.s_b = d_dyn_scale; pp.status = d_status;
+    // CTA pairs on 256 x 256 tiles (one pair per TPC) when the problem has at least a pair's worth of rows.
+    // (192 output columns per tile would fill the last wave of tiles better at the 1.3B width: 13.8 waves instead
+    // of 10.4; measured slower, 1048 against 1161 TFLOP/s: the narrower product costs more than the tail.)
+    const char* force_single = getenv("SALAD_PROJ_SINGLE");
+    if (dev.sms >= 2 && N > 128 && !(force_single && force_single[0] == '1')) {
+        const long long pairs_dev = dev.sms / 2, mt2 = (long long)B * ((N + 255) / 256);
+        constexpr int bn = 256;
+        const long long tiles2 = mt2 * ((D + bn - 1) / bn);
+        CUtensorMap ma2, mw2;
+        if (!make_tmap_bf16_3d(&ma2, o_l, d, N, int64_t(B) * H, 128) || !make_tmap_bf16_3d(&mw2, w, D, D, 1, bn / 2))
+            return SALAD_ERR_CUDA;
+        const long long pairs = pairs_dev < tiles2 ? pairs_dev : tiles2;
+        SALAD_LOGF("salad_proj_gemm_pair_kernel<%d> grid %lld (clusters of 2) block %d", bn, 2 * pairs, Proj2Cfg<256>::THREADS);
+        salad_proj_gemm_pair_kernel<256><<<unsigned(2 * pairs), Proj2Cfg<256>::THREADS, Proj2Cfg<256>::SMEM_BYTES, st>>>(ma2, mw2, pp);
+        return check_launch();
+    }
     const unsigned grid = unsigned(pp.tiles < dev.sms ? pp.tiles : dev.sms);
+    SALAD_LOGF("salad_proj_gemm_kernel grid %u block %d smem %d", grid, ProjCfg::THREADS, ProjCfg::SMEM_BYTES);
     salad_proj_gemm_kernel<<<grid, ProjCfg::THREADS, ProjCfg::SMEM_BYTES, st>>>(ma, mw, pp);
     return check_launch();
 }
