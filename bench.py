@@ -501,14 +501,46 @@ def main():
                                                           Bk=wl.Bk, out=out, workspace=ws), 10)
         extras["topk_mask"]["fused_on_topk_lists_ms"] = tk_fused_ms
 
+        # the fused call with one d x d Level-1 projection block per head folded into the linear state (Sec. 4.2)
+        if Hm <= wl.H:
+            blocks = (torch.randn(wl.H, wl.d, wl.d, device=dev) / wl.d ** 0.5).to(torch.bfloat16)
+            bp_ms = timed(lambda: salad.salad_fused_proj_fwd(q, k, v, rp, ci, Hm, blocks, s_d, Bq=wl.Bq, Bk=wl.Bk,
+                                                             out=out, workspace=ws), 20)
+            extras["fused_block_proj"] = {"ms": bp_ms, "tflops": flops / (bp_ms * 1e-3) / 1e12}
+            del blocks
+        # the paper's own ST-SWA (App. A.1) through the loads: half of the heads take their tokens grouped by
+        # spatial position, every head a 1-D window of a tenth of the sequence (90 % sparse); beside it the
+        # same work done with permutation passes (Q, K, V forward, O back) around the fused call
+        T_, Hs_, Ws_ = wl.grid
+        if T_ <= 64 and wl.Bq == 128 and wl.Bk == 64:
+            st_flags = [h % 2 for h in range(wl.H)]
+            st_rp, st_ci = salad.salad_stswa_mask_build(wl.grid, st_flags, [wl.N // 20] * wl.H, device=dev)
+            st_ms = timed(lambda: salad.salad_fused_stswa_fwd(q, k, v, wl.grid, st_flags, st_rp, st_ci, lam_d, s_d,
+                                                              out=out), 10)
+            pq, pk, pv, po = (torch.empty_like(q) for _ in range(4))
+
+            def passes():
+                salad.salad_permute_tokens(q, wl.grid, st_flags, out=pq)
+                salad.salad_permute_tokens(k, wl.grid, st_flags, out=pk)
+                salad.salad_permute_tokens(v, wl.grid, st_flags, out=pv)
+                salad.salad_permute_tokens(po, wl.grid, st_flags, inverse=True, out=out)
+            pass_ms = timed(passes, 10)
+            extras["fused_stswa"] = {"ms": st_ms, "kept_blocks": int(st_ci.numel()),
+                                     "temporal_heads": sum(st_flags), "window_half_width_tokens": wl.N // 20,
+                                     "four_permutation_passes_ms": pass_ms}
+            del pq, pk, pv, po, st_rp, st_ci
+
         # rotary variant of the linear branch (Sec. 4.1): the same fused call with the 3-D rotation table of
         # the workload's latent grid (fp16, 8.4 MB at this shape, shared by all heads)
         rope_d = salad.salad_rope3d_table_build(*wl.grid, wl.d, device=dev)
         rope_ms = timed(lambda: salad.salad_fused_rope_fwd(q, k, v, rp, ci, Hm, lam_d, s_d, rope_d, Bq=wl.Bq, Bk=wl.Bk,
                                                            out=out, workspace=ws), 20)
         rope_lin_ms = timed(lambda: salad.salad_linear_attn_rope_fwd(q, k, v, rope_d, out=out, workspace=ws), 20)
+        # the plain call timed the same way right beside it (the long timed region may sit at the power cap)
+        plain_ms = timed(lambda: salad.salad_fused_fwd(q, k, v, rp, ci, Hm, lam_d, s_d, Bq=wl.Bq, Bk=wl.Bk,
+                                                       out=out, workspace=ws), 20)
         extras["rope_linear_branch"] = {"fused_ms": rope_ms, "fused_tflops": flops / (rope_ms * 1e-3) / 1e12,
-                                        "extra_ms_over_plain_call": rope_ms - ms_per_step,
+                                        "plain_call_ms": plain_ms, "extra_ms_over_plain_call": rope_ms - plain_ms,
                                         "linear_only_ms": rope_lin_ms}
 
     # ---------------- sustained: the same call back to back for seconds, into the power cap (after everything
