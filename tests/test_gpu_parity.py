@@ -669,6 +669,54 @@ def test_stswa_through_the_loads(salad, grid, B, H, d, flags, windows):
     assert_close(f32(out.cpu()).reshape(-1, d), ref.reshape(-1, d), "ST-SWA through the loads")
 
 
+def test_stswa_wan13b_shape(salad):
+    # ST-SWA through the loads at the full Wan-1.3B shape, as the benchmark runs it (every second head temporal,
+    # a window of a tenth of the sequence on every head's own order): lists bit-exact for every head, output on
+    # sampled rows of every head -- first, last and random query blocks, first / last / random row of each.
+    wl = wlmod.C2
+    grid = wl.grid
+    T, Hs, Ws = grid
+    B, H, N, d = wl.B, wl.H, wl.N, wl.d
+    flags = [h % 2 for h in range(H)]
+    windows = [N // 20] * H
+    q, k, v = wlmod.make_qkv(wl)
+    lam, s = wlmod.make_scales(wl)
+    rows, kq, ks, nkb_p = salad.salad_stswa_blocks(grid)
+    rp_d, ci_d = salad.salad_stswa_mask_build(grid, flags, windows)
+    rp_g, ci_g = rp_d.cpu().numpy(), ci_d.cpu().numpy()
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = torch.full_like(q.cuda(), 3.0)
+    salad.salad_fused_stswa_fwd(q.cuda(), k.cuda(), v.cuda(), grid, flags, rp_d, ci_d, torch.from_numpy(lam).cuda(),
+                                torch.from_numpy(s).cuda(), out=out, status=status)
+    status_ok(status)
+    got_all = f32(out.cpu())
+    assert np.isfinite(got_all).all()
+    # position m of a temporal head's own order holds token order_t[m] (from the oracle's re-ordering of an index ramp)
+    ramp = np.arange(N, dtype=np.float32).reshape(1, 1, N, 1)
+    order_t = orc.permute_tokens(ramp, grid, [1]).reshape(N).astype(np.int64)
+    qp, kp, vp = (orc.permute_tokens(f32(t), grid, flags) for t in (q, k, v))
+    rng = np.random.default_rng(77)
+    worst = (0.0, 0.0)
+    for h in range(H):
+        Bq, Bk = (kq * T, ks * T) if flags[h] else (128, 64)
+        rp_o, ci_o = orc.mask_build(1, 1, N, Bq, Bk, [(0, 0, windows[h])])
+        n_own = len(rp_o) - 1
+        assert np.array_equal(rp_g[h * rows:h * rows + n_own + 1] - rp_g[h * rows], rp_o), h
+        assert np.array_equal(ci_g[rp_g[h * rows]:rp_g[h * rows + n_own]], ci_o), h
+        blocks = {0, n_own - 1} | set(rng.integers(0, n_own, 6).tolist())
+        ms = []
+        for i in blocks:
+            m0, m1 = i * Bq, min(N, (i + 1) * Bq)
+            ms += [m0, m1 - 1, int(rng.integers(m0, m1))]
+        ms = np.unique(np.asarray(ms, dtype=np.int64))
+        ref = orc.salad_fused(qp[:, h:h + 1], kp[:, h:h + 1], vp[:, h:h + 1], Bq, Bk, rp_o, ci_o, 1,
+                              lam[h:h + 1].astype(np.float64), s.astype(np.float64), sel=ms)     # B = 1: row index = m
+        toks = order_t[ms] if flags[h] else ms
+        ma, rel = assert_close(got_all[0, h, toks], ref, f"ST-SWA full size, head {h}", tight=True)
+        worst = (max(worst[0], ma), max(worst[1], rel))
+    print(f"\n[parity] ST-SWA through the loads, {wl.name}: max_abs {worst[0]:.3e} rel_l2 {worst[1]:.3e}")
+
+
 # ------------------------------------------------------------------------------ full projection (Alg. 1 level 1)
 
 @pytest.mark.parametrize("B,H,N,d,with_bias", [
@@ -746,6 +794,27 @@ def test_fused_block_projection(salad, B, H, N, d, Bq):
     # the drop threshold
     drop = salad.salad_fused_proj_fwd(qd, kd, vd, rp_d, ci_d, 1, wb.cuda(), s_d, Bq=Bq, drop_tau=2.0)
     assert torch.equal(drop, sparse)
+
+
+def test_fused_block_projection_wan13b_shape(salad):
+    # the block projection at the full Wan-1.3B shape (the benchmark's configuration), stratified rows of all heads
+    wl = wlmod.C2
+    q, k, v = wlmod.make_qkv(wl)
+    T, Hs, Ws = wl.grid
+    _, s = wlmod.make_scales(wl)
+    rng = np.random.default_rng(4242)
+    wb = bf16(rng.standard_normal((wl.H, wl.d, wl.d)) / np.sqrt(wl.d))
+    rp_d, ci_d = salad.salad_mask_build(T, Hs, Ws, wl.Bq, wl.Bk, wl.windows)
+    rp, ci = rp_d.cpu().numpy(), ci_d.cpu().numpy()
+    Hm = len(wl.windows)
+    status = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = salad.salad_fused_proj_fwd(q.cuda(), k.cuda(), v.cuda(), rp_d, ci_d, Hm, wb.cuda(), torch.from_numpy(s).cuda(),
+                                     Bq=wl.Bq, Bk=wl.Bk, status=status)
+    status_ok(status)
+    sel = stratified_rows(wl, rp, Hm, dense_heads=2)
+    ref = orc.salad_fused_blockproj(f32(q), f32(k), f32(v), wl.Bq, wl.Bk, rp, ci, Hm, f32(wb), s.astype(np.float64), sel=sel)
+    max_abs, rel = assert_close(f32(out.cpu()).reshape(-1, wl.d)[sel], ref, "block projection, full size", tight=True)
+    print(f"\n[parity] block projection, {wl.name}: {len(sel)} stratified rows: max_abs {max_abs:.3e} rel_l2 {rel:.3e}")
 
 
 def test_state_pass_as_its_own_call_on_a_side_stream(salad):
