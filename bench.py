@@ -415,20 +415,25 @@ def main():
     # ---------------- extras (rank 0): per-branch calls and the 0 %-sparsity run of the same kernel
     extras = {}
     if rank == 0 and not args.no_extras:
-        def timed(fn, iters):
+        def timed(fn, iters, reps=1):
+            """ms per call over `iters` back-to-back calls; the median of `reps` such loops (the short,
+            HBM-bound calls are timed three times: one loop of 20 lasts about a millisecond)."""
             for _ in range(2):
                 fn()
             torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(iters):
-                fn()
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) / iters
+            got = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(iters):
+                    fn()
+                b.record()
+                torch.cuda.synchronize()
+                got.append(a.elapsed_time(b) / iters)
+            return sorted(got)[len(got) // 2]
         extras["sparse_only_ms"] = timed(lambda: salad.salad_sparse_attn_fwd(
             q, k, v, rp, ci, Hm, Bq=wl.Bq, Bk=wl.Bk, out=out, workspace=ws), 20)
-        extras["linear_only_ms"] = timed(lambda: salad.salad_linear_attn_fwd(q, k, v, out=out, workspace=ws), 20)
+        extras["linear_only_ms"] = timed(lambda: salad.salad_linear_attn_fwd(q, k, v, out=out, workspace=ws), 20, reps=3)
         # the whole linear branch as one call: K, V read (state), Q read and O written (apply)
         lin_bytes = 4 * q_h.numel() * q_h.element_size()
         def hbm_record(kernel, ms, nbytes):
@@ -450,7 +455,7 @@ def main():
         # the short-ring variant of the same kernels shares its SMs with the attention kernel
         # (`roofline.state_kernels_ms`).
         kv_bytes = 2 * tensor_bytes
-        lin_state_ms = timed(lambda: salad.salad_linear_state_fwd(k, v, ws), 20)
+        lin_state_ms = timed(lambda: salad.salad_linear_state_fwd(k, v, ws), 20, reps=3)
         extras["linear_state"] = hbm_record("salad_linear_state_fwd: salad_linear_state_kernel + salad_linear_finalize_kernel (K, V read once)",
                                             lin_state_ms, kv_bytes)
         # the attention call on a workspace that already holds the state (a caller who ran the state pass
@@ -466,7 +471,7 @@ def main():
         w_dyn = torch.randn(wl.H * wl.d, device=dev, dtype=torch.float32) / (wl.H * wl.d) ** 0.5
         s_out = torch.empty(2, device=dev, dtype=torch.float32)
         dyn_ws = torch.empty(salad.DYN_SCALE_WS_BYTES, dtype=torch.uint8, device=dev)
-        dyn_ms = timed(lambda: salad.salad_dynamic_scale(xt, w_dyn, 0.0, out=s_out, workspace=dyn_ws), 20)
+        dyn_ms = timed(lambda: salad.salad_dynamic_scale(xt, w_dyn, 0.0, out=s_out, workspace=dyn_ws), 20, reps=3)
         x_bytes = xt.numel() * 2
         extras["dynamic_scale"] = hbm_record("dynamic_scale_partial_kernel + finalize (X_t read once)", dyn_ms, x_bytes)
         del xt
@@ -483,7 +488,7 @@ def main():
         # temporal-head permutation (App. A.1): one read and one write of a [B,H,N,d] tensor
         flags = [1] * wl.H
         perm_out = torch.empty_like(q)
-        perm_ms = timed(lambda: salad.salad_permute_tokens(q, wl.grid, flags, out=perm_out), 20)
+        perm_ms = timed(lambda: salad.salad_permute_tokens(q, wl.grid, flags, out=perm_out), 20, reps=3)
         extras["permute_tokens"] = hbm_record("permute_tokens_kernel (one read, one write)", perm_ms, 2 * tensor_bytes)
         del perm_out
         # Top-K mask producer (App. A.1 steps 1-2) at this shape, k chosen for the same 90 % sparsity:
