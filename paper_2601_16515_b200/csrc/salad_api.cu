@@ -149,7 +149,7 @@ int prepare_device(DeviceInfo* info) {
                                      ApplyCfg<64, true>::SMEM_BYTES);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(topk_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     128 * (kScoreRows + kScoreTile) * 4);
+                                     kScoreSmemBytes);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(salad_proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      ProjCfg::SMEM_BYTES);
@@ -892,18 +892,19 @@ SALAD_EXPORT int salad_topk_mask_build(const void* q, const void* k, int B, int 
     MeanJob jk{static_cast<const uint4*>(k), kmeanT, Bk, int(nKb), ldk};
     block_mean_kernel<<<dim3(unsigned(nQb > nKb ? nQb : nKb), unsigned(BH), 2), kMeanThreads, 0, st>>>(jq, jk, N, d);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
-    const size_t smem = size_t(d) * (kScoreRows + kScoreTile) * 4;          // 80 KB at d = 128
+    const size_t smem = kScoreSmemBytes;
     launch_dependent(topk_score_kernel, dim3(unsigned(ldk / kScoreTile), unsigned((nQb + kScoreRows - 1) / kScoreRows),
                                              unsigned(BH)),
-                     dim3(256), smem, st, qmean, kmeanT, int(nQb), int(nKb), ldk, d, score);
+                     dim3(128), smem, st, qmean, kmeanT, int(nQb), int(nKb), ldk, d, score);
     if (check_launch() != SALAD_OK) return SALAD_ERR_CUDA;
     const dim3 pgrid(unsigned((rows + 7) / 8));
-    if (nKb <= 512)
-        launch_dependent(topk_pick_kernel<16>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
-    else if (nKb <= 1024)
-        launch_dependent(topk_pick_kernel<32>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+    // a CTA per row while the row fits the threads' registers; the warp-per-two-rows kernel beyond that
+    if (nKb <= 512 && rows <= 2147483647ll)
+        launch_dependent(topk_pick_row_kernel<4>, dim3(unsigned(rows)), dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+    else if (nKb <= 1024 && rows <= 2147483647ll)
+        launch_dependent(topk_pick_row_kernel<8>, dim3(unsigned(rows)), dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
     else
-        launch_dependent(topk_pick_kernel<0>, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
+        launch_dependent(topk_pick_kernel, pgrid, dim3(128), 0, st, score, int(nKb), int(kk), d_row_ptr, d_col_idx, rows);
     return check_launch();
 }
 

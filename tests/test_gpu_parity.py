@@ -542,6 +542,24 @@ def test_topk_mask_build(salad, B, H, N, d, Bq, Bk, topk):
     assert ndiff <= max(1, (len(rp_o) - 1) // 50)            # near ties are rare
 
 
+@pytest.mark.parametrize("N,Bk,topk", [(2048, 64, 5), (6400, 16, 7), (9600, 16, 3), (19200, 16, 9)])      # 32, 400, 600, 1200 key blocks
+def test_topk_exact_ties_go_to_the_lower_block(salad, N, Bk, topk):
+    # Exact ties: groups of key blocks with identical tokens have bit-identical means and scores, so the
+    # selection must be settled by the index (lists equal to the oracle's, no near-tie allowance).  The sizes
+    # cover both selection kernels (a row in the registers of one CTA, and the longer rows).
+    B, H, d, Bq = 1, 2, 64, 128
+    rng = np.random.default_rng(N + topk)
+    nKb = N // Bk
+    base = rng.standard_normal((B, H, 4, Bk, d)).astype(np.float32)          # four distinct key blocks ...
+    which = rng.integers(0, 4, size=nKb)
+    k = torch.from_numpy(base[:, :, which].reshape(B, H, N, d)).to(torch.bfloat16)      # ... repeated in random order
+    q = torch.from_numpy(rng.standard_normal((B, H, N, d)).astype(np.float32)).to(torch.bfloat16)
+    rp_o, ci_o = orc.topk_mask(f32(q), f32(k), Bq, Bk, topk)
+    rp_g, ci_g = salad.salad_topk_mask_build(q.cuda(), k.cuda(), topk, Bq=Bq, Bk=Bk)
+    assert np.array_equal(rp_g.cpu().numpy(), rp_o)
+    assert np.array_equal(ci_g.cpu().numpy(), ci_o)
+
+
 def test_topk_mask_wan13b_shape(salad):
     # full size, the configuration the benchmark times: k = 51 of 512 key blocks (90 % block sparsity)
     wl = wlmod.C2
